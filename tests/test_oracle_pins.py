@@ -1,0 +1,299 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, a library
+attention routine in fp64, and brute force.  None of them re-uses the oracle's
+own formula; each is chosen so that a plausible mistake in the oracle (wrong
+head mapping, dropped scale, wrong source layer, off-by-one length) fails."""
+import itertools
+import math
+import os
+
+import pytest
+import torch
+
+import workloads as W
+from oracle import Oracle, cache_bytes, count_owners, group_map, mu_from_owners
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(path):
+    with open(os.path.join(GOLD, path)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def _rand_bf16(shape, seed, std=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(shape, generator=g, dtype=torch.float32) * std).to(torch.bfloat16)
+
+
+def _fill(o, L, B, n, Hkv, D, seed):
+    """Distinct random K/V for every layer; returns dict layer -> (K,V) [B,n,Hkv,D]."""
+    store = {}
+    b_idx = torch.arange(B).repeat_interleave(n)
+    t_idx = torch.arange(n).repeat(B)
+    for l in range(L):
+        K = _rand_bf16((B, n, Hkv, D), seed * 100 + 2 * l)
+        V = _rand_bf16((B, n, Hkv, D), seed * 100 + 2 * l + 1)
+        o.append(l, K.reshape(B * n, Hkv, D), V.reshape(B * n, Hkv, D), b_idx, t_idx)
+        store[l] = (K, V)
+    return store
+
+
+def _sdpa64(Q, K, V, lens, scale):
+    """torch's library attention in fp64, one sequence at a time.
+    Q [B,Hq,D]; K,V [B,n,Hkv,D]; GQA by repeat_interleave over heads."""
+    B, Hq, D = Q.shape
+    Hkv = K.shape[2]
+    G = Hq // Hkv
+    out = torch.zeros(B, Hq, D, dtype=torch.float64)
+    for b in range(B):
+        n = int(lens[b])
+        if n == 0:
+            continue
+        q = Q[b].double()[None, :, None, :]                                  # [1,Hq,1,D]
+        k = K[b, :n].double().permute(1, 0, 2).repeat_interleave(G, 0)[None]  # [1,Hq,n,D]
+        v = V[b, :n].double().permute(1, 0, 2).repeat_interleave(G, 0)[None]
+        out[b] = torch.nn.functional.scaled_dot_product_attention(q, k, v, scale=scale)[0, :, 0, :]
+    return out
+
+
+# ------------------------------------------------------------------ routing
+def test_fig4_sharing_example():
+    """Figure 4: S={1,3} of 5 layers -> layers 1-2 read KV1, 3-5 read KV3; 60 % saved."""
+    rows = {r[0]: r[1:] for r in _rows("fig4_sharing.txt")}
+    L = int(rows["n_layers"][0])
+    owners0 = [int(x) - 1 for x in rows["cached"]]
+    reads0 = [int(x) - 1 for x in rows["reads"]]
+    mu = mu_from_owners(L, owners0)
+    assert mu == reads0 == [0, 0, 2, 2, 2]
+    assert count_owners(mu) == 2
+    full = cache_bytes(list(range(L)), 8, 128, 2, 1000)
+    shared = cache_bytes(mu, 8, 128, 2, 1000)
+    assert round(100 * (1 - shared / full)) == int(rows["memory_saved_percent"][0])
+    num, den = rows["cached_fraction"][0].split("/")
+    assert shared * int(den) == full * int(num)
+
+
+def test_mu_matches_definition_on_all_small_owner_sets():
+    """Eq. (3.2) by exhaustive enumeration, against an independent set-based restatement."""
+    L = 6
+    for k in range(1, L + 1):
+        for S in itertools.combinations(range(L), k):
+            got = mu_from_owners(L, S)
+            if 0 not in S:
+                assert got is None          # mu undefined for layers below the first owner
+                continue
+            want = [l if l in S else max(j for j in S if j < l) for l in range(L)]
+            assert got == want
+            assert all(got[got[l]] == got[l] and got[l] <= l for l in range(L))
+
+
+def test_owner_reads_itself():
+    """l' = l reduces to self-attention: with S = all layers mu is the identity."""
+    assert mu_from_owners(7, range(7)) == list(range(7))
+
+
+def test_group_maps():
+    """Section 4.3 leaders: g consecutive layers share the first; 'every 4th layer' (Section 1)."""
+    assert group_map(8, 4) == [0, 0, 0, 0, 4, 4, 4, 4]
+    assert group_map(36, 4) == mu_from_owners(36, range(0, 36, 4))
+    assert count_owners(group_map(36, 4)) == 9
+    assert count_owners(group_map(36, 8)) == 5           # last group is short
+    assert group_map(5, 1) == [0, 1, 2, 3, 4]
+
+
+# ------------------------------------------------------------------ bytes
+def test_bytes_per_token_printed_values():
+    for name, L, Hkv, D, kb in _rows("kv_bytes_per_token.txt"):
+        L, Hkv, D, kb = int(L), int(Hkv), int(D), int(kb)
+        per_token = cache_bytes(list(range(L)), Hkv, D, 2, 1)
+        assert per_token == 2 * L * Hkv * D * 2
+        assert per_token // 1024 == kb and per_token % 1024 == 0
+
+
+def test_tables_4_and_5_kv_cache_column():
+    """KV-cache MB cells of Tables 4 and 5.  The tables do not print how many
+    tokens were generated; 128 (Table 4) and 63 (Table 5) are the counts that
+    reproduce every cell, with MB = 2^20 bytes and round-half-up."""
+    gen = {"4": 128, "5": 63}
+    for tab, T, batch, g, mb in _rows("table4_table5_kv_mb.txt"):
+        r = group_map(36, int(g))
+        n_tok = int(batch) * (int(T) + gen[tab])
+        got = cache_bytes(r, 8, 128, 2, n_tok) / 2 ** 20
+        assert math.floor(got + 0.5) == int(mb), (tab, T, batch, g, got)
+
+
+def test_cache_scales_as_one_over_g():
+    """'KV cache memory scales as 1/g' (Section 4.3)."""
+    base = cache_bytes(group_map(32, 1), 8, 128, 2, 4096)
+    for g in (2, 4, 8):
+        assert cache_bytes(group_map(32, g), 8, 128, 2, 4096) * g == base
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (6, 2, 32), (8, 8, 16), (8, 1, 128)])
+def test_identity_map_equals_library_attention(Hq, Hkv, D):
+    """Identity routing = standard per-layer attention (Algorithm 1)."""
+    L, B, n = 3, 3, 40
+    o = Oracle(L, list(range(L)), Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=7)
+    lens = torch.tensor([40, 1, 23], dtype=torch.int32)
+    for l in range(L):
+        Q = _rand_bf16((B, Hq, D), 900 + l)
+        for scale in (D ** -0.5, 0.37):
+            got = o.decode_attn(l, Q, lens, scale)
+            want = _sdpa64(Q, store[l][0], store[l][1], lens, scale)
+            assert torch.allclose(got, want, rtol=1e-12, atol=1e-13)
+
+
+def test_all_layers_routed_to_layer0():
+    L, B, n, Hq, Hkv, D = 4, 2, 19, 4, 2, 32
+    o = Oracle(L, [0] * L, Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=3)
+    lens = torch.tensor([19, 7], dtype=torch.int32)
+    for l in range(L):
+        Q = _rand_bf16((B, Hq, D), 50 + l)
+        want = _sdpa64(Q, store[0][0], store[0][1], lens, D ** -0.5)
+        assert torch.allclose(o.decode_attn(l, Q, lens), want, rtol=1e-12, atol=1e-13)
+
+
+def test_routed_layers_read_their_source_and_nothing_else():
+    """r=[0,0,2,2]: layer 1 must use layer 0's cache, layer 3 layer 2's; changing the
+    non-owner layers' own K/V changes no output."""
+    L, B, n, Hq, Hkv, D = 4, 2, 33, 4, 2, 64
+    r = [0, 0, 2, 2]
+    o = Oracle(L, r, Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=11)
+    lens = torch.tensor([33, 20], dtype=torch.int32)
+    Qs = [_rand_bf16((B, Hq, D), 70 + l) for l in range(L)]
+    outs = [o.decode_attn(l, Qs[l], lens) for l in range(L)]
+    for l in range(L):
+        want = _sdpa64(Qs[l], store[r[l]][0], store[r[l]][1], lens, D ** -0.5)
+        assert torch.allclose(outs[l], want, rtol=1e-12, atol=1e-13)
+        other = _sdpa64(Qs[l], store[l][0], store[l][1], lens, D ** -0.5)
+        if r[l] != l:
+            assert not torch.allclose(outs[l], other, rtol=1e-3, atol=1e-3)
+    # overwrite the non-owner layers' own stores: outputs must not move
+    b_idx = torch.arange(B).repeat_interleave(n)
+    t_idx = torch.arange(n).repeat(B)
+    for l in (1, 3):
+        o.append(l, _rand_bf16((B * n, Hkv, D), 999 + l), _rand_bf16((B * n, Hkv, D), 1999 + l), b_idx, t_idx)
+    for l in range(L):
+        assert torch.equal(o.decode_attn(l, Qs[l], lens), outs[l])
+
+
+def test_single_cached_token_returns_its_value_exactly():
+    L, B, Hq, Hkv, D = 2, 3, 6, 3, 16
+    o = Oracle(L, [0, 0], Hq, Hkv, D, B, 4)
+    store = _fill(o, L, B, 4, Hkv, D, seed=5)
+    lens = torch.ones(B, dtype=torch.int32)
+    out = o.decode_attn(1, _rand_bf16((B, Hq, D), 1), lens)
+    V0 = store[0][1][:, 0].double()                     # [B,Hkv,D]
+    assert torch.equal(out, V0.repeat_interleave(Hq // Hkv, dim=1))
+
+
+def test_softmax_weights_are_a_distribution_and_uniform_for_zero_query():
+    L, B, n, Hq, Hkv, D = 1, 2, 57, 4, 2, 32
+    o = Oracle(L, [0], Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=9)
+    Q = _rand_bf16((B, Hq, D), 2, std=2.0)
+    for b in range(B):
+        for h in range(Hq):
+            w = o.attn_weights(0, Q, b, h, n)
+            assert (w >= 0).all() and abs(w.sum().item() - 1.0) < 1e-15 * n
+    lens = torch.tensor([57, 31], dtype=torch.int32)
+    out = o.decode_attn(0, torch.zeros(B, Hq, D, dtype=torch.bfloat16), lens)
+    for b in range(B):
+        mean_v = store[0][1][b, : int(lens[b])].double().mean(0)          # [Hkv,D]
+        assert torch.allclose(out[b], mean_v.repeat_interleave(Hq // Hkv, 0), rtol=1e-13, atol=1e-14)
+
+
+def test_two_token_closed_form_sigmoid():
+    """n=2 with axis-aligned vectors: w0 = 1/(1+exp(-(s0-s1))), s_t = scale*a*k_t."""
+    D, scale, a, k0, k1 = 8, 0.25, 3.0, 2.0, -1.5
+    o = Oracle(1, [0], 1, 1, D, 1, 2)
+    K = torch.zeros(2, 1, D, dtype=torch.bfloat16)
+    V = torch.zeros(2, 1, D, dtype=torch.bfloat16)
+    K[0, 0, 0], K[1, 0, 0] = k0, k1
+    V[0, 0, :], V[1, 0, :] = 1.0, -3.0
+    o.append(0, K, V, torch.tensor([0, 0]), torch.tensor([0, 1]))
+    Q = torch.zeros(1, 1, D, dtype=torch.bfloat16)
+    Q[0, 0, 0] = a
+    w0 = 1.0 / (1.0 + math.exp(-(scale * a * (k0 - k1))))
+    out = o.decode_attn(0, Q, torch.tensor([2], dtype=torch.int32), scale)
+    assert torch.allclose(out, torch.full((1, 1, D), w0 * 1.0 + (1 - w0) * -3.0, dtype=torch.float64),
+                          rtol=1e-14, atol=0)
+
+
+def test_brute_force_tiny():
+    """Independent pure-Python loops, no max subtraction, explicit weights."""
+    L, B, n, Hq, Hkv, D = 3, 2, 5, 4, 2, 4
+    r = [0, 0, 2]
+    o = Oracle(L, r, Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=21)
+    lens = [5, 3]
+    scale = 0.5
+    for l in range(L):
+        Q = _rand_bf16((B, Hq, D), 300 + l)
+        got = o.decode_attn(l, Q, torch.tensor(lens, dtype=torch.int32), scale)
+        Ks, Vs = store[r[l]]
+        for b in range(B):
+            for h in range(Hq):
+                kv = h // (Hq // Hkv)
+                e = []
+                for t in range(lens[b]):
+                    s = sum(float(Q[b, h, d]) * float(Ks[b, t, kv, d]) for d in range(D))
+                    e.append(math.exp(scale * s))
+                z = sum(e)
+                for d in range(D):
+                    want = sum(e[t] / z * float(Vs[b, t, kv, d]) for t in range(lens[b]))
+                    assert abs(got[b, h, d].item() - want) < 1e-12
+
+
+def test_zero_length_sequence_gives_zero_row_and_length_is_respected():
+    L, B, n, Hq, Hkv, D = 1, 2, 10, 2, 1, 8
+    o = Oracle(L, [0], Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=4)
+    Q = _rand_bf16((B, Hq, D), 8)
+    out = o.decode_attn(0, Q, torch.tensor([0, 6], dtype=torch.int32))
+    assert torch.equal(out[0], torch.zeros(Hq, D, dtype=torch.float64))
+    want = _sdpa64(Q, store[0][0], store[0][1], [0, 6], D ** -0.5)
+    assert torch.allclose(out, want, rtol=1e-12, atol=1e-13)
+    full = o.decode_attn(0, Q, torch.tensor([0, 7], dtype=torch.int32))
+    assert not torch.allclose(full[1], out[1])
+
+
+def test_append_is_a_bit_copy_and_last_write_wins():
+    o = Oracle(2, [0, 0], 2, 2, 8, 2, 6)
+    K = _rand_bf16((3, 2, 8), 1)
+    V = _rand_bf16((3, 2, 8), 2)
+    o.append(1, K, V, torch.tensor([1, 0, 1]), torch.tensor([5, 2, 5]))
+    k, v = o.read(1, 1, 5)
+    assert torch.equal(k.view(torch.int16), K[2].view(torch.int16))
+    assert torch.equal(v.view(torch.int16), V[2].view(torch.int16))
+    k, v = o.read(1, 0, 2)
+    assert torch.equal(k.view(torch.int16), K[1].view(torch.int16))
+    k, _ = o.read(1, 0, 0)
+    assert torch.equal(k.view(torch.int16), torch.zeros(2, 8, dtype=torch.int16))
+    with pytest.raises(RuntimeError):
+        o.read(0, 0, 0)          # layer 0 never appended: no store
+
+
+def test_oracle_on_the_tiny_workload_matches_library_attention():
+    """The tiny workload end to end (shapes of the first benchmark config)."""
+    w = W.get_workload("tiny")
+    r = W.routing_map(w)
+    lens = W.seq_lens(w)
+    o = Oracle(w.n_layers, r, w.q_heads, w.kv_heads, w.head_dim, w.batch, int(lens.max()))
+    si, pos = W.token_index(lens)
+    dense = {}
+    for l in range(w.n_layers):
+        K, V = W.draw_kv(w, l, si, pos)
+        o.append(l, K, V, si, pos)
+        Kd = torch.zeros(w.batch, int(lens.max()), w.kv_heads, w.head_dim, dtype=torch.bfloat16)
+        Vd = torch.zeros_like(Kd)
+        Kd[si, pos], Vd[si, pos] = K, V
+        dense[l] = (Kd, Vd)
+    for l in range(w.n_layers):
+        Q = W.draw_q(w, l)
+        want = _sdpa64(Q, dense[r[l]][0], dense[r[l]][1], lens, w.head_dim ** -0.5)
+        assert torch.allclose(o.decode_attn(l, Q, lens), want, rtol=1e-12, atol=1e-13)
