@@ -1,0 +1,228 @@
+/*
+ * skv.h -- C ABI of the routed (depth-wise shared) paged KV cache and its
+ * decode-time attention step for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes, in the paper's terms ("Stochastic KV Routing:
+ * Enabling Adaptive Depth-Wise Cache Sharing", Section 3.1):
+ *
+ *   - A transformer decoder has L layers.  A cache sharing strategy S names
+ *     the layers that keep a KV cache; every layer l reads the cache of its
+ *     source layer mu(l) <= l (Eq. (3.2)).  This library takes the map itself,
+ *     r[l] (0-based), and accepts any r with r[0] = 0, r[l] <= l and
+ *     r[r[l]] = r[l]; layers with r[l] = l are the OWNERS.
+ *   - Algorithm 2, one decode step, per layer:  "Update" (append the new
+ *     token's K,V) happens only for owners; "Load" + "Attn" reads the owner's
+ *     cache:  Output_l = Attn(Q_l, K_r[l], V_r[l])   (Eq. (3.1)).
+ *     Attn is scaled dot-product softmax attention with grouped queries:
+ *     query head h reads KV head floor(h / (q_heads / kv_heads)).
+ *   - Cache memory is allocated for owners only, so its size is
+ *     2 x |owners| x kv_heads x head_dim x 2 bytes per token (Section 1
+ *     footnote with #layers -> |S|; Section 4.3: "scales as 1/g").
+ *
+ * Conventions
+ *   - Every function returns an int status: SKV_OK (0) or a negative
+ *     skv_status.  Nothing throws or aborts.  Argument errors are found on the
+ *     host before anything is launched.
+ *   - "device" pointers are CUDA device memory of the current device, owned by
+ *     the caller for the whole life of the handle; the library never allocates
+ *     or frees device memory (except where a function says otherwise).
+ *     "host" pointers are ordinary host memory.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
+ *     as void*; NULL = the default stream) and the call returns without
+ *     waiting, except skv_get_status which synchronises that stream.
+ *   - bf16 tensors are dense, row-major, last index fastest.
+ *   - Layers are 0-based (the paper counts from 1).
+ *   - There is no CPU implementation behind these calls: without a usable
+ *     CUDA device every call that needs one returns SKV_ERR_CUDA.
+ *
+ * Supported shapes: head_dim 64 or 128; page_size 16; q_heads a multiple of
+ * kv_heads with q_heads / kv_heads <= 8.
+ */
+#ifndef SKV_H
+#define SKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct skv_cache skv_cache; /* opaque host-side handle */
+
+typedef enum skv_status {
+    SKV_OK = 0,
+    SKV_ERR_ARG = -1,         /* null pointer, non-positive size, misaligned buffer */
+    SKV_ERR_ROUTING = -2,     /* r[0] != 0, r[l] > l, r[l] < 0 or r[r[l]] != r[l] */
+    SKV_ERR_UNSUPPORTED = -3, /* shape outside the supported set */
+    SKV_ERR_NOMEM = -4,       /* caller's pool or workspace is too small */
+    SKV_ERR_LAYER = -5,       /* layer index out of range, or an owner is required */
+    SKV_ERR_CUDA = -6,        /* a CUDA runtime call failed (no device, bad stream, ...) */
+    SKV_ERR_TIMEOUT = -7,     /* device status: a bounded wait inside a kernel ran out */
+    SKV_ERR_BOUNDS = -8       /* device status: a page id or slot id was out of range */
+} skv_status;
+
+const char *skv_strerror(int status);
+
+/* ---- routing maps (pure host) ------------------------------------------ */
+
+/* Eq. (3.2): r_out[l] = l if l is in owners[], else the largest owner below l.
+ * owners: host, n_owners distinct layer indices in [0, n_layers), any order;
+ * layer 0 must be among them (otherwise mu is undefined for the layers below
+ * the first owner -> SKV_ERR_ROUTING).  r_out: host, n_layers entries. */
+int skv_routing_from_owners(int n_layers, const int32_t *owners, int n_owners, int32_t *r_out);
+
+/* Section 4.3 "leaders": every g consecutive layers read the first one of
+ * their group, r_out[l] = l - (l mod g); the last group may be short. */
+int skv_routing_groups(int n_layers, int g, int32_t *r_out);
+
+/* ---- cache -------------------------------------------------------------- */
+
+/* Bytes of device memory the caller must provide for the page pool:
+ * a 256-byte header + |owners| * max_pages * page_bytes, where
+ * page_bytes = 2 (K,V) * page_size * kv_heads * head_dim * 2.
+ * max_pages is per owner layer; page ids are shared by all owner layers. */
+int skv_cache_pool_bytes(int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                         int page_size, int64_t max_pages, size_t *out_bytes);
+
+/* Create a handle (Algorithm 2's cache state for a strategy S).
+ *   r           host, n_layers entries, copied.
+ *   device_pool device, >= pool_bytes, 256-byte aligned; zero-filled on `stream`
+ *               by this call; must outlive the handle.  If device_pool is NULL
+ *               (and pool_bytes 0) the handle does accounting only: routing and
+ *               byte queries work, every call that would launch returns
+ *               SKV_ERR_ARG.  No CUDA call is made in that case.
+ * Errors: SKV_ERR_ROUTING, SKV_ERR_UNSUPPORTED, SKV_ERR_NOMEM (pool_bytes too
+ * small), SKV_ERR_ARG, SKV_ERR_CUDA. */
+int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                     int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes,
+                     void *stream);
+
+/* Frees host state only; never touches device_pool. */
+void skv_cache_destroy(skv_cache *cache);
+
+/* r[layer] (>= 0) or SKV_ERR_LAYER. */
+int skv_layer_owner(const skv_cache *cache, int layer);
+/* 1 if r[layer] == layer, 0 if not, SKV_ERR_LAYER if out of range. */
+int skv_is_owner(const skv_cache *cache, int layer);
+
+/* Byte accounting; any out pointer may be NULL.
+ *   page_bytes      bytes of one page of one owner layer
+ *   kv_bytes        |owners| * max_pages * page_bytes (the KV storage proper)
+ *   bytes_per_token 2 * |owners| * kv_heads * head_dim * 2 */
+int skv_cache_stats(const skv_cache *cache, int *n_owners, size_t *page_bytes, size_t *kv_bytes,
+                    size_t *bytes_per_token);
+
+/* ---- Algorithm 2 "Update": append ---------------------------------------- */
+
+/* Store the K,V rows of n_tokens new tokens in `layer`'s cache.  If `layer`
+ * is not an owner this is a no-op that launches nothing (its K,V are never
+ * read: Algorithm 2 updates only layers in S) and K, V may be NULL.
+ *   K, V      device bf16 [n_tokens][kv_heads][head_dim], 16-byte aligned
+ *   slot_map  device int64 [n_tokens]; slot = page * page_size + offset;
+ *             a negative slot skips the token; slots >= max_pages * page_size
+ *             are skipped and raise SKV_ERR_BOUNDS in the device status.
+ *             Duplicate slots in one call: unspecified which row is kept.
+ * The copy is bit-exact. */
+int skv_append(skv_cache *cache, int layer, const void *K, const void *V, const int64_t *slot_map,
+               int64_t n_tokens, void *stream);
+
+/* Inverse of skv_append for tests and snapshots: read rows back.
+ *   layer     must be an owner (SKV_ERR_LAYER otherwise)
+ *   slot_ids  device int64 [n]; negative -> the output row is left untouched
+ *   K_out, V_out device bf16 [n][kv_heads][head_dim] */
+int skv_gather(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t n, void *K_out,
+               void *V_out, void *stream);
+
+/* ---- Algorithm 2 "Load + Attn": decode attention -------------------------- */
+
+/* Bytes of device workspace skv_decode_attn needs for this batch / head count
+ * (split partials and a page-count prefix; independent of sequence lengths). */
+int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, size_t *out_bytes);
+
+/* Eq. (3.1) for one layer and one new token per sequence:
+ *   out[b,h,:] = sum_{t < seq_lens[b]} softmax_t(scale * <Q[b,h,:], K[b,t,kv(h),:]>) * V[b,t,kv(h),:]
+ * with K,V the cache of layer r[layer] and token t of sequence b stored at
+ * slot page_table[b][t / page_size] * page_size + t % page_size.
+ *   Q           device bf16 [batch][q_heads][head_dim], 16-byte aligned
+ *   page_table  device int32 [batch][pt_stride]; entries past a sequence's
+ *               last page are never read
+ *   seq_lens    device int32 [batch]; tokens to attend, including the one just
+ *               appended; 0 gives an all-zero output row
+ *   out         device bf16 [batch][q_heads][head_dim]
+ *   scale       <= 0 selects 1/sqrt(head_dim)
+ *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes;
+ *               may be reused by later calls on the same stream
+ * Runs two kernels on `stream`: a split-K flash-decoding pass that writes
+ * fp32 partial (max, sum, output) triples, and a log-sum-exp merge.  Slots past
+ * seq_lens[b] in the last page contribute nothing whatever they contain.
+ * No host synchronisation; sequence lengths are read on the device.
+ * Errors: SKV_ERR_ARG, SKV_ERR_LAYER, SKV_ERR_UNSUPPORTED (head ratio),
+ * SKV_ERR_NOMEM (workspace), SKV_ERR_CUDA.  Device-side problems (page id out
+ * of range, a bounded wait that ran out) are reported by skv_get_status. */
+int skv_decode_attn(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
+                    const int32_t *seq_lens, void *out, int batch, int q_heads, int pt_stride,
+                    float scale, void *workspace, size_t workspace_bytes, void *stream);
+
+/* The two halves of skv_decode_attn, separately launchable (profiling,
+ * sequence-sharded use): the split-K pass fills `workspace`; the merge turns
+ * the partials in `workspace` into `out`.  Same arguments and errors. */
+int skv_decode_splitk(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
+                      const int32_t *seq_lens, int batch, int q_heads, int pt_stride, float scale,
+                      void *workspace, size_t workspace_bytes, void *stream);
+int skv_decode_merge(skv_cache *cache, const int32_t *seq_lens, void *out, int batch, int q_heads,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* One whole decode step of Algorithm 2 from HOST buffers: copies the step's
+ * inputs to the device, runs append + decode attention for layers 0..L-1 in
+ * order, and copies the outputs back, all on `stream` (the caller
+ * synchronises).  Host buffers should be pinned for the copies to be
+ * asynchronous.
+ *   hQ          host bf16 [n_layers][batch][q_heads][head_dim]
+ *   hK, hV      host bf16 [n_owners][batch][kv_heads][head_dim], owner layers
+ *               in increasing layer order
+ *   h_slot_map  host int64 [batch]  (slot of each sequence's new token)
+ *   h_page_table host int32 [batch][pt_stride];  h_seq_lens host int32 [batch]
+ *   h_out       host bf16 [n_layers][batch][q_heads][head_dim]
+ *   staging     device, 256-byte aligned, >= skv_decode_step_staging_bytes;
+ *               holds the device copies of all of the above plus the decode
+ *               workspace */
+int skv_decode_step_staging_bytes(const skv_cache *cache, int batch, int q_heads, int pt_stride,
+                                  size_t *out_bytes);
+int skv_decode_step_host(skv_cache *cache, const void *hQ, const void *hK, const void *hV,
+                         const int64_t *h_slot_map, const int32_t *h_page_table,
+                         const int32_t *h_seq_lens, void *h_out, int batch, int q_heads,
+                         int pt_stride, float scale, void *staging, size_t staging_bytes,
+                         void *stream);
+
+/* ---- status, tuning, counters ------------------------------------------- */
+
+/* Synchronises `stream`, reads and clears the device status word.
+ * *device_status receives SKV_OK, SKV_ERR_TIMEOUT or SKV_ERR_BOUNDS. */
+int skv_get_status(skv_cache *cache, void *stream, int *device_status);
+
+/* Split-K kernel variant: 0 = automatic (CUDA-core kernel when
+ * q_heads == kv_heads, tensor-core (mma) kernel otherwise), 1 = CUDA-core
+ * kernel (only q_heads == kv_heads), 2 = tensor-core kernel. */
+int skv_set_decode_variant(skv_cache *cache, int variant);
+
+/* Launch shape of the split-K kernel: warps per CTA (1..16), pipeline stages
+ * per warp (2..8) and CTAs per SM (1..8); 0 keeps the current value.
+ * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
+int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
+
+/* Number of kernels this handle has launched so far. */
+int skv_launch_count(const skv_cache *cache, int64_t *out_count);
+
+/* The split-K work partition (pure host arithmetic, same code the kernels use):
+ * the n_blocks (sequence, kv head, page) blocks of a call are cut into
+ * n_workers contiguous ranges of equal size +-1.  skv_plan_worker_range gives
+ * worker w's [begin, end); skv_plan_worker_of gives the worker whose range
+ * holds block x, or SKV_ERR_ARG. */
+int skv_plan_worker_range(int64_t n_blocks, int n_workers, int w, int64_t *begin, int64_t *end);
+int skv_plan_worker_of(int64_t n_blocks, int n_workers, int64_t x);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKV_H */

@@ -1,0 +1,219 @@
+// Shared declarations of the skv CUDA library (sm_100a): page geometry, kernel
+// parameter blocks, PTX helpers and the host-side launcher prototypes.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace skv {
+
+// ---- page geometry ---------------------------------------------------------
+// One page holds PAGE tokens of every kv head of one owner layer.  Within the
+// page, each (kv head) owns one contiguous block [K half | V half]; a half is
+// stored "chunk-major": [D/8 chunks][PAGE tokens][8 bf16], i.e. element
+// (token t, dim d) of a half sits at byte ((d/8)*PAGE + t)*16 + (d%8)*2.
+// A 128-byte run is thus 8 tokens x 8 dims: exactly one 8x8 tensor-core
+// operand matrix, so ldmatrix reads it without bank conflicts and the whole
+// block is moved by a single linear bulk copy.
+constexpr int PAGE = 16;
+constexpr int CHUNK_ELEMS = 8;                   // bf16 per 16-byte chunk
+constexpr int HEADER_BYTES = 256;                // pool header (device status word)
+
+__host__ __device__ constexpr int half_bytes(int D) { return PAGE * D * 2; }
+__host__ __device__ constexpr int block_bytes(int D) { return 2 * half_bytes(D); }
+
+// device status bits
+constexpr int STATUS_TIMEOUT = 1;
+constexpr int STATUS_BOUNDS = 2;
+
+struct AppendParams {
+    uint8_t *layer_base;        // first page of this owner layer
+    const uint4 *K;             // [n_tokens][Hkv][D] bf16 viewed as 16-byte chunks
+    const uint4 *V;
+    const int64_t *slot_map;
+    int64_t n_tokens;
+    int64_t n_slots;            // max_pages * PAGE
+    int64_t page_stride;        // bytes between pages of one layer
+    int Hkv, D;
+    int *status;
+};
+
+struct GatherParams {
+    const uint8_t *layer_base;
+    uint4 *K_out;
+    uint4 *V_out;
+    const int64_t *slot_ids;
+    int64_t n;
+    int64_t n_slots;
+    int64_t page_stride;
+    int Hkv, D;
+    int *status;
+};
+
+struct DecodeParams {
+    const uint8_t *layer_base;  // first page of the owner layer that is read
+    int64_t page_stride;
+    int64_t max_pages;
+    const uint16_t *Q;          // [B][Hq][D] bf16 bits
+    const int32_t *page_table;  // [B][pt_stride]
+    const int32_t *seq_lens;    // [B]
+    float *part_o;              // [n_slots][G][D]
+    float *part_ml;             // [n_slots][G][2]  (running max in log2 units, sum)
+    int32_t *prefix;            // [B+1] cumulative page counts (written by CTA 0)
+    int B, Hq, Hkv, pt_stride;
+    float scale_log2;           // scale * log2(e)
+    int *status;
+};
+
+struct MergeParams {
+    const float *part_o;
+    const float *part_ml;
+    const int32_t *prefix;      // [B+1]
+    const int32_t *seq_lens;
+    uint16_t *out;              // [B][Hq][D] bf16 bits
+    int B, Hq, Hkv, D;
+    int n_workers;
+};
+
+struct DecodeTuning {
+    int variant;                // 0 auto, 1 CUDA-core (G=1), 2 tensor-core
+    int warps;                  // per CTA
+    int stages;                 // per warp
+    int ctas_per_sm;
+};
+
+// host launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
+cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
+// smem bytes the split-K kernel needs for this shape, or 0 if unsupported
+size_t decode_smem_bytes(int D, int B, int warps, int stages);
+cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid,
+                                 int warps, int stages, cudaStream_t s);
+cudaError_t launch_merge(const MergeParams &p, cudaStream_t s);
+
+// ---- worker <-> work-range arithmetic (shared by split-K and merge) --------
+// The flattened work space orders (sequence b, kv head h, page pg) b-major:
+// position x = prefix[b]*Hkv + h*pages_b + pg,  total T = prefix[B]*Hkv.
+// Worker w of W owns [w*T/W, (w+1)*T/W).
+__host__ __device__ inline int64_t worker_begin(int64_t w, int64_t T, int64_t W) { return (w * T) / W; }
+
+// first worker whose range contains position x (0 <= x < T)
+__host__ __device__ inline int worker_of(int64_t x, int64_t T, int64_t W)
+{
+    int64_t w = (x * W) / T;
+    if (w >= W) w = W - 1;
+    while (w > 0 && worker_begin(w, T, W) > x) --w;
+    while (w + 1 < W && worker_begin(w + 1, T, W) <= x) ++w;
+    return (int)w;
+}
+
+// ---- PTX helpers -------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up after about two seconds and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+// linear bulk copy global -> this CTA's shared memory, completion on an mbarrier
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+// D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// two fp32 -> packed bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+}  // namespace skv

@@ -1,0 +1,99 @@
+"""Driving code shared by the GPU tests, the smoke check and the benchmark:
+sets a workload up on the device through the binding (pool, page table, cache
+pre-fill, per-step inputs).  It draws inputs from :mod:`workloads` and calls
+the library; it contains no arithmetic of the method and never touches the
+oracle."""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List, Optional
+
+import torch
+
+import workloads as W
+
+from .binding import SkvCache
+
+
+@dataclasses.dataclass
+class DeviceWorkload:
+    w: W.Workload
+    r: List[int]
+    lens_cpu: torch.Tensor            # int32 [B], tokens attended in the decode step
+    page_table_cpu: torch.Tensor      # int32 [B, width]
+    total_pages: int
+    cache: SkvCache
+    page_table: torch.Tensor          # device copies
+    seq_lens: torch.Tensor
+    slot_new: torch.Tensor            # int64 [B] slot of each sequence's newest token (position n_b-1)
+    workspace: torch.Tensor
+    device: torch.device
+
+    @property
+    def batch(self) -> int:
+        return int(self.lens_cpu.numel())
+
+    @property
+    def owners(self) -> List[int]:
+        return [l for l in range(self.w.n_layers) if self.r[l] == l]
+
+    def kv_bytes_per_call(self) -> int:
+        """Algorithmic bytes of one decode-attention call: the owner layer's K,V of
+        every attended token, plus Q in and out out."""
+        w = self.w
+        tokens = int(self.lens_cpu.to(torch.int64).sum())
+        return tokens * w.kv_heads * w.head_dim * 2 * 2 + 2 * self.batch * w.q_heads * w.head_dim * 2
+
+    def append_bytes_per_call(self) -> int:
+        """Algorithmic bytes of one owner-layer append of one token per sequence (read + write)."""
+        w = self.w
+        return 2 * (self.batch * w.kv_heads * w.head_dim * 2 * 2)
+
+
+def setup(w: W.Workload, device="cuda", lens: Optional[torch.Tensor] = None, r: Optional[List[int]] = None,
+          extra_pages: int = 0, permute: Optional[bool] = None) -> DeviceWorkload:
+    device = torch.device(device)
+    r = W.routing_map(w) if r is None else list(r)
+    lens_cpu = (W.seq_lens(w) if lens is None else lens).to(torch.int32)
+    B = int(lens_cpu.numel())
+    table, total = W.page_layout(lens_cpu, w.page_size, w.permute_pages if permute is None else permute, w.seed,
+                                 extra_pages=extra_pages)
+    total = max(total, 1)
+    cache = SkvCache(r, w.kv_heads, w.head_dim, w.page_size, total, allocate=True)
+    ws = torch.empty(cache.skv_decode_workspace_bytes(B, w.q_heads), dtype=torch.uint8, device=device)
+    b = torch.arange(B, dtype=torch.int64)
+    last = (lens_cpu.to(torch.int64) - 1)
+    has = last >= 0
+    slot_new = torch.full((B,), -1, dtype=torch.int64)
+    if bool(has.any()):
+        slot_new[has] = W.slot_map_for(table, b[has], last[has], w.page_size)
+    return DeviceWorkload(w=w, r=r, lens_cpu=lens_cpu, page_table_cpu=table, total_pages=total, cache=cache,
+                          page_table=table.to(device), seq_lens=lens_cpu.to(device),
+                          slot_new=slot_new.to(device), workspace=ws, device=device)
+
+
+def prefill(dw: DeviceWorkload, upto_offset: int = -1, layers: Optional[List[int]] = None,
+            chunk_tokens: int = 1 << 16) -> None:
+    """Append tokens t < lens[b] + upto_offset of every owner layer (drawn on the device)."""
+    w = dw.w
+    seq_idx, pos = W.token_index(dw.lens_cpu, upto_offset)
+    slots = W.slot_map_for(dw.page_table_cpu, seq_idx, pos, w.page_size)
+    for l in (dw.owners if layers is None else layers):
+        if dw.r[l] != l:
+            continue
+        for s in range(0, seq_idx.numel(), chunk_tokens):
+            e = min(seq_idx.numel(), s + chunk_tokens)
+            K, V = W.draw_kv(w, l, seq_idx[s:e], pos[s:e], device=dw.device)
+            dw.cache.skv_append(l, K, V, slots[s:e].to(dw.device))
+    torch.cuda.synchronize(dw.device)
+
+
+def step_inputs(dw: DeviceWorkload, layer: int, device=None) -> Dict[str, torch.Tensor]:
+    """Q of `layer` and the newest token's K,V rows (position lens[b]-1) for this decode step."""
+    w = dw.w
+    device = dw.device if device is None else device
+    B = dw.batch
+    b = torch.arange(B, dtype=torch.int64)
+    last = (dw.lens_cpu.to(torch.int64) - 1).clamp(min=0)
+    K, V = W.draw_kv(w, layer, b, last, device=device)
+    return {"Q": W.draw_q(w, layer, batch=B, device=device), "K": K, "V": V}

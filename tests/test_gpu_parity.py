@@ -1,0 +1,207 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Cache contents: bit-exact.  Attention
+outputs: |out - ref| <= 1e-2 + 1e-2*|ref| (bf16 in, fp32 accumulate)."""
+import pytest
+import torch
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 1e-2, 1e-2
+
+
+def _within_tol(out_bf16, ref64):
+    out = out_bf16.detach().cpu().double()
+    err = (out - ref64).abs()
+    bound = ATOL + RTOL * ref64.abs()
+    worst = (err - bound).max().item()
+    return worst <= 0.0, err.max().item()
+
+
+def _make(w, **kw):
+    from paper_2604_22782_b200 import harness
+    return harness, harness.setup(w, **kw)
+
+
+def _oracle_for(dw, seqs, layers_needed, upto_offset=0):
+    """Oracle holding sequences `seqs` (their full lengths) for the given layers' own stores."""
+    from oracle import Oracle
+    w = dw.w
+    sub_lens = dw.lens_cpu[seqs]
+    o = Oracle(w.n_layers, dw.r, w.q_heads, w.kv_heads, w.head_dim, len(seqs), max(1, int(sub_lens.max())))
+    local, pos = W.token_index(sub_lens, upto_offset)
+    glob = torch.as_tensor(seqs, dtype=torch.int64)[local]
+    for l in layers_needed:
+        K, V = W.draw_kv(w, l, glob, pos)
+        o.append(l, K, V, local, pos)
+    return o
+
+
+def _decode_layer(dw, layer, Q=None, scale=0.0):
+    from paper_2604_22782_b200 import harness
+    w = dw.w
+    if Q is None:
+        Q = harness.step_inputs(dw, layer)["Q"]
+    out = torch.full((dw.batch, w.q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device=dw.device)
+    dw.cache.skv_decode_attn(layer, Q, dw.page_table, dw.seq_lens, out, dw.workspace, scale=scale)
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    return Q, out
+
+
+def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True):
+    """One decode step of every layer: prefill n-1 tokens, append the last one, attend; compare all."""
+    harness, dw = _make(w, lens=lens, r=r, permute=permute)
+    if poison:   # every byte of the page area becomes a bf16 NaN pattern (0x7FC1)
+        dw.pool_view = dw.cache.pool[256:].view(torch.int16)
+        dw.pool_view.fill_(0x7FC1)
+    if variant:
+        dw.cache.skv_set_decode_variant(variant)
+    if tuning:
+        dw.cache.skv_set_decode_tuning(*tuning)
+    B = dw.batch
+    harness.prefill(dw, upto_offset=-1)
+    seqs = list(range(B))
+    o = _oracle_for(dw, seqs, range(w.n_layers), upto_offset=0)    # every layer keeps its own store
+    worst = 0.0
+    for l in range(w.n_layers):
+        inp = harness.step_inputs(dw, l)
+        before = dw.cache.skv_launch_count()
+        dw.cache.skv_append(l, inp["K"], inp["V"], dw.slot_new)
+        if dw.r[l] != l:
+            assert dw.cache.skv_launch_count() == before      # non-owner: nothing launched
+        Q, out = _decode_layer(dw, l, inp["Q"])
+        ref = o.decode_attn(l, Q.cpu(), dw.lens_cpu)
+        ok, err = _within_tol(out, ref)
+        worst = max(worst, err)
+        assert ok, f"layer {l}: max abs err {err}"
+        assert torch.isfinite(out.float()).all()
+    if check_cache:
+        seq_idx, pos = W.token_index(dw.lens_cpu)
+        slots = W.slot_map_for(dw.page_table_cpu, seq_idx, pos, w.page_size).to(dw.device)
+        n = seq_idx.numel()
+        for l in dw.owners:
+            Kg = torch.zeros((n, w.kv_heads, w.head_dim), dtype=torch.bfloat16, device=dw.device)
+            Vg = torch.zeros_like(Kg)
+            dw.cache.skv_gather(l, slots, Kg, Vg)
+            torch.cuda.synchronize()
+            Kg, Vg = Kg.cpu().view(torch.int16), Vg.cpu().view(torch.int16)
+            for i in range(0, n, max(1, n // 97)):
+                k, v = o.read(l, int(seq_idx[i]), int(pos[i]))
+                assert torch.equal(k.view(torch.int16), Kg[i]) and torch.equal(v.view(torch.int16), Vg[i])
+            Kd, Vd = W.draw_kv(w, l, seq_idx, pos)            # what was appended, all rows
+            assert torch.equal(Kd.view(torch.int16), Kg) and torch.equal(Vd.view(torch.int16), Vg)
+    assert dw.cache.skv_get_status() == 0
+    return worst
+
+
+def test_tiny_config_every_layer():
+    """Config 1: 4 layers r=[0,0,2,2], 4 q / 2 kv heads, D=64, lens {37,128}, contiguous pages."""
+    w = W.get_workload("tiny")
+    assert W.routing_map(w) == [0, 0, 2, 2] and W.seq_lens(w).tolist() == [37, 128]
+    _full_step_check(w)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 4, 128), (4, 4, 64), (4, 2, 128), (8, 2, 128), (8, 2, 64), (8, 1, 128),
+                                       (6, 2, 64), (3, 1, 128)])
+def test_all_short_lengths(Hq, Hkv, D):
+    """Every length 0..3*page_size (one sequence each; odd batch) for G in {1,2,3,4,8}, D in {64,128}."""
+    lens = torch.arange(0, 3 * 16 + 1, dtype=torch.int32)
+    w = W.Workload("short", 3, Hq, Hkv, D, 16, lens.numel(), 0, 48, "explicit", explicit_r=(0, 0, 2), seed=11)
+    _full_step_check(w, lens=lens)
+
+
+def test_poisoned_pool_never_leaks():
+    """Unused slots hold NaN patterns: tokens past seq_len must contribute nothing."""
+    lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3], dtype=torch.int32)
+    for Hq, Hkv in ((8, 2), (2, 2)):
+        w = W.Workload("poison", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=5)
+        _full_step_check(w, lens=lens, poison=True, check_cache=False)
+
+
+@pytest.mark.parametrize("variant,Hq,Hkv", [(2, 4, 4), (1, 4, 4), (2, 16, 4)])
+def test_forced_variants_and_launch_shapes(variant, Hq, Hkv):
+    """Tensor-core kernel on MHA, CUDA-core kernel, and other warps/stages/CTAs-per-SM settings."""
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15], dtype=torch.int32)
+    w = W.Workload("variants", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=6)
+    for tuning in ((4, 3, 2), (1, 2, 1), (8, 2, 1), (2, 6, 2), (3, 4, 3)):
+        _full_step_check(w, lens=lens, variant=variant, tuning=tuning, check_cache=False)
+
+
+def test_page_permutation_does_not_change_outputs():
+    lens = torch.tensor([300, 77, 512, 129], dtype=torch.int32)
+    w = W.Workload("perm", 2, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=8)
+    from paper_2604_22782_b200 import harness
+    outs = []
+    for permute in (False, True):
+        dw = harness.setup(w, lens=lens, permute=permute, extra_pages=13)
+        harness.prefill(dw, upto_offset=0)
+        outs.append(_decode_layer(dw, 1)[1].cpu())
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+
+
+def test_non_owner_append_is_a_noop_and_null_inputs_are_fine():
+    from paper_2604_22782_b200 import harness
+    w = W.get_workload("tiny")
+    dw = harness.setup(w)
+    harness.prefill(dw, upto_offset=0)
+    snap = dw.cache.pool.clone()
+    count = dw.cache.skv_launch_count()
+    for l in (1, 3):
+        inp = harness.step_inputs(dw, l)
+        dw.cache.skv_append(l, inp["K"], inp["V"], dw.slot_new)
+        dw.cache.skv_append(l, None, None, None, n_tokens=dw.batch)
+    torch.cuda.synchronize()
+    assert dw.cache.skv_launch_count() == count
+    assert torch.equal(snap, dw.cache.pool)
+    with pytest.raises(Exception):
+        dw.cache.skv_append(0, None, None, dw.slot_new)       # an owner needs real K,V
+
+
+def test_out_of_range_ids_are_flagged_not_followed():
+    """Bad slot / page ids raise the device status word; nothing is read or written out of bounds."""
+    from paper_2604_22782_b200 import harness
+    from paper_2604_22782_b200.binding import SKV_ERR_BOUNDS
+    w = W.get_workload("tiny")
+    dw = harness.setup(w)
+    harness.prefill(dw, upto_offset=0)
+    inp = harness.step_inputs(dw, 0)
+    bad = dw.slot_new.clone()
+    bad[0] = dw.total_pages * w.page_size + 5
+    dw.cache.skv_append(0, inp["K"], inp["V"], bad)
+    assert dw.cache.skv_get_status() == SKV_ERR_BOUNDS
+    assert dw.cache.skv_get_status() == 0                      # reading clears it
+    pt = dw.page_table.clone()
+    pt[1, 2] = dw.total_pages + 7
+    out = torch.zeros((dw.batch, w.q_heads, w.head_dim), dtype=torch.bfloat16, device=dw.device)
+    dw.cache.skv_decode_attn(0, inp["Q"], pt, dw.seq_lens, out, dw.workspace)
+    assert dw.cache.skv_get_status() == SKV_ERR_BOUNDS
+
+
+def test_medium_llama3_shape_ragged():
+    """Llama-3-8B head shape, 12 ragged sequences spanning many pages and several workers' ranges."""
+    lens = torch.tensor([1000, 17, 640, 333, 2049, 1, 16, 999, 1500, 48, 777, 1211], dtype=torch.int32)
+    w = W.Workload("medium", 4, 32, 8, 128, 16, lens.numel(), 0, 0, "groups", group=2, seed=21)
+    _full_step_check(w, lens=lens)
+
+
+def test_medium_mha_long_sequence_split_and_merge():
+    """MHA, one 20k-token sequence + short ones: one segment is split over many workers and merged."""
+    lens = torch.tensor([20000, 5, 300], dtype=torch.int32)
+    w = W.Workload("mha_long", 2, 4, 4, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=23)
+    _full_step_check(w, lens=lens, check_cache=False)
+
+
+def test_explicit_scale_is_used():
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([200, 31], dtype=torch.int32)
+    w = W.Workload("scale", 1, 8, 2, 128, 16, 2, 0, 0, "explicit", explicit_r=(0,), seed=29)
+    dw = harness.setup(w, lens=lens)
+    harness.prefill(dw, upto_offset=0)
+    o = _oracle_for(dw, [0, 1], [0])
+    Q, out = _decode_layer(dw, 0, scale=0.031)
+    ok, err = _within_tol(out, o.decode_attn(0, Q.cpu(), dw.lens_cpu, 0.031))
+    assert ok, err
+    ok_default, _ = _within_tol(out, o.decode_attn(0, Q.cpu(), dw.lens_cpu))
+    assert not ok_default
