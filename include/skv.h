@@ -173,6 +173,19 @@ int skv_decode_splitk(skv_cache *cache, int layer, const void *Q, const int32_t 
 int skv_decode_merge(skv_cache *cache, const int32_t *seq_lens, void *out, int batch, int q_heads,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* One whole decode step of Algorithm 2 with inputs already on the device:
+ * for l = 0..L-1: append (owners only) then decode attention, on `stream`.
+ *   Q        device bf16 [n_layers][batch][q_heads][head_dim]
+ *   K, V     device bf16 [n_owners][batch][kv_heads][head_dim], owner layers in
+ *            increasing layer order
+ *   slot_map device int64 [batch]: slot of each sequence's new token
+ *   out      device bf16 [n_layers][batch][q_heads][head_dim]
+ * Other arguments as in skv_decode_attn. */
+int skv_decode_step(skv_cache *cache, const void *Q, const void *K, const void *V,
+                    const int64_t *slot_map, const int32_t *page_table, const int32_t *seq_lens,
+                    void *out, int batch, int q_heads, int pt_stride, float scale, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
 /* One whole decode step of Algorithm 2 from HOST buffers: copies the step's
  * inputs to the device, runs append + decode attention for layers 0..L-1 in
  * order, and copies the outputs back, all on `stream` (the caller

@@ -56,6 +56,7 @@ lib.skv_decode_workspace_bytes.argtypes = [_vp, _int, _int, _szp]
 lib.skv_decode_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_splitk.argtypes = [_vp, _int, _vp, _i32p, _i32p, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_merge.argtypes = [_vp, _i32p, _vp, _int, _int, _vp, _sz, _vp]
+lib.skv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_step_staging_bytes.argtypes = [_vp, _int, _int, _int, _szp]
 lib.skv_decode_step_host.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32,
                                      _vp, _sz, _vp]
@@ -241,6 +242,15 @@ class SkvCache:
         rc = lib.skv_decode_merge(self._h, _ptr(seq_lens), _ptr(out), batch, q_heads, _ptr(workspace),
                                   workspace.numel(), _stream_ptr(stream))
         _check(rc, "skv_decode_merge")
+
+    def skv_decode_step(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, slot_map: torch.Tensor,
+                        page_table: torch.Tensor, seq_lens: torch.Tensor, out: torch.Tensor,
+                        workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:
+        batch, q_heads = Q.shape[1], Q.shape[2]
+        rc = lib.skv_decode_step(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(slot_map), _ptr(page_table),
+                                 _ptr(seq_lens), _ptr(out), batch, q_heads, page_table.shape[1], scale,
+                                 _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+        _check(rc, "skv_decode_step")
 
     def skv_decode_step_staging_bytes(self, batch: int, q_heads: int, pt_stride: int) -> int:
         out = _sz(0)

@@ -362,6 +362,31 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
     return skv_decode_merge(c, seq_lens, out, batch, q_heads, workspace, workspace_bytes, stream);
 }
 
+int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, const int64_t *slot_map,
+                    const int32_t *page_table, const int32_t *seq_lens, void *out, int batch, int q_heads,
+                    int pt_stride, float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_decode_args(c, 0, batch, q_heads);
+    if (rc) return rc;
+    if (!Q || !K || !V || !slot_map || !out) return SKV_ERR_ARG;
+    const size_t q_layer = (size_t)batch * q_heads * c->head_dim * 2;
+    const size_t kv_layer = (size_t)batch * c->kv_heads * c->head_dim * 2;
+    const uint8_t *q = static_cast<const uint8_t *>(Q), *k = static_cast<const uint8_t *>(K),
+                  *v = static_cast<const uint8_t *>(V);
+    uint8_t *o = static_cast<uint8_t *>(out);
+    for (int l = 0; l < c->n_layers; ++l) {
+        const int os = c->slot[(size_t)l];
+        if (os >= 0) {
+            rc = skv_append(c, l, k + (size_t)os * kv_layer, v + (size_t)os * kv_layer, slot_map, batch, stream);
+            if (rc) return rc;
+        }
+        rc = skv_decode_attn(c, l, q + (size_t)l * q_layer, page_table, seq_lens, o + (size_t)l * q_layer, batch,
+                             q_heads, pt_stride, scale, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+    }
+    return SKV_OK;
+}
+
 // ---- whole decode step from host buffers -------------------------------------
 namespace {
 struct StagingLayout {
@@ -424,18 +449,11 @@ int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const voi
     ok &= cudaMemcpyAsync(d + s.page_table, h_page_table, (size_t)batch * pt_stride * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(d + s.seq_lens, h_seq_lens, (size_t)batch * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
-    for (int l = 0; l < c->n_layers; ++l) {
-        const int os = c->slot[(size_t)l];
-        if (os >= 0) {
-            rc = skv_append(c, l, d + s.k + (size_t)os * kv_layer, d + s.v + (size_t)os * kv_layer,
-                            reinterpret_cast<const int64_t *>(d + s.slot_map), batch, stream);
-            if (rc) return rc;
-        }
-        rc = skv_decode_attn(c, l, d + s.q + (size_t)l * q_layer, reinterpret_cast<const int32_t *>(d + s.page_table),
-                             reinterpret_cast<const int32_t *>(d + s.seq_lens), d + s.out + (size_t)l * q_layer,
-                             batch, q_heads, pt_stride, scale, d + s.ws, s.ws_bytes, stream);
-        if (rc) return rc;
-    }
+    rc = skv_decode_step(c, d + s.q, d + s.k, d + s.v, reinterpret_cast<const int64_t *>(d + s.slot_map),
+                         reinterpret_cast<const int32_t *>(d + s.page_table),
+                         reinterpret_cast<const int32_t *>(d + s.seq_lens), d + s.out, batch, q_heads, pt_stride,
+                         scale, d + s.ws, s.ws_bytes, stream);
+    if (rc) return rc;
     if (cudaMemcpyAsync(h_out, d + s.out, q_layer * c->n_layers, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;

@@ -97,3 +97,22 @@ def step_inputs(dw: DeviceWorkload, layer: int, device=None) -> Dict[str, torch.
     last = (dw.lens_cpu.to(torch.int64) - 1).clamp(min=0)
     K, V = W.draw_kv(w, layer, b, last, device=device)
     return {"Q": W.draw_q(w, layer, batch=B, device=device), "K": K, "V": V}
+
+
+def step_tensors(dw: DeviceWorkload, device=None, pin: bool = False) -> Dict[str, torch.Tensor]:
+    """Inputs of one whole decode step, stacked: Q [L,B,Hq,D]; K,V [n_owners,B,Hkv,D] (owner layers in
+    increasing order); out buffer [L,B,Hq,D]."""
+    w = dw.w
+    device = dw.device if device is None else torch.device(device)
+    qs, ks, vs = [], [], []
+    for l in range(w.n_layers):
+        inp = step_inputs(dw, l, device=device)
+        qs.append(inp["Q"])
+        if dw.r[l] == l:
+            ks.append(inp["K"])
+            vs.append(inp["V"])
+    t = {"Q": torch.stack(qs).contiguous(), "K": torch.stack(ks).contiguous(), "V": torch.stack(vs).contiguous()}
+    t["out"] = torch.zeros_like(t["Q"])
+    if pin and device.type == "cpu":
+        t = {k: v.pin_memory() for k, v in t.items()}
+    return t

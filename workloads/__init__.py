@@ -168,6 +168,11 @@ WORKLOADS = {
 }
 
 
+# the same attention call as "llama3_8b" (same batch, lengths, page permutation) with only two
+# layers, so that a profiler capture holds a few hundred MB instead of the whole model's cache
+WORKLOADS["llama3_8b_2layers"] = dataclasses.replace(WORKLOADS["llama3_8b"], name="llama3_8b_2layers", n_layers=2)
+
+
 def sweep_workload(group: int) -> Workload:
     """Sharing-ratio sweep on the Llama-3-8B shape: owner fraction 1/group."""
     return Workload(f"sweep_g{group}", 32, 32, 8, 128, 16, 128, 512, 2048, "groups",
