@@ -160,6 +160,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--tuning", default="", help="warps,stages,ctas_per_sm of the split-K kernel")
+    ap.add_argument("--merge-mode", type=int, default=-1, help="1 = merge inside the split-K kernel, 0 = merge kernel")
+    ap.add_argument("--balance", default="", help="pool_percent,min_chunk_blocks,chunks_per_worker")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = W.get_workload(args.workload)
@@ -181,10 +183,10 @@ def main():
         import dataclasses
         w = dataclasses.replace(w, seed=w.seed + 1000 * rank)
     dw = harness.setup(w, device=dev)
-    if args.variant:
-        dw.cache.skv_set_decode_variant(args.variant)
-    if args.tuning:
-        dw.cache.skv_set_decode_tuning(*[int(x) for x in args.tuning.split(",")])
+    dw.retune(variant=args.variant or None,
+              tuning=[int(x) for x in args.tuning.split(",")] if args.tuning else None,
+              merge_mode=args.merge_mode if args.merge_mode >= 0 else None,
+              balance=[int(x) for x in args.balance.split(",")] if args.balance else None)
     harness.prefill(dw, upto_offset=-1)
     t = harness.step_tensors(dw)
     L, n_own = w.n_layers, len(dw.owners)
@@ -225,7 +227,7 @@ def main():
                 a.record()
                 cache.skv_decode_splitk(l, t["Q"][l], dw.page_table, dw.seq_lens, dw.workspace)
                 b.record()
-                cache.skv_decode_merge(dw.seq_lens, t["out"][l], dw.workspace)
+                cache.skv_decode_merge(t["out"][l], dw.workspace)
                 pairs.append((a, b))
         torch.cuda.synchronize(dev)
         kern_ms = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)

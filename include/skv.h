@@ -137,7 +137,10 @@ int skv_gather(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t n, 
 /* ---- Algorithm 2 "Load + Attn": decode attention -------------------------- */
 
 /* Bytes of device workspace skv_decode_attn needs for this batch / head count
- * (split partials and a page-count prefix; independent of sequence lengths). */
+ * under the CURRENT launch shape and balance settings (ask again after
+ * skv_set_decode_tuning / skv_set_decode_balance).  Independent of sequence
+ * lengths.  It holds the split partials, a page-count prefix and a few control
+ * words. */
 int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, size_t *out_bytes);
 
 /* Eq. (3.1) for one layer and one new token per sequence:
@@ -151,27 +154,36 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
  *               appended; 0 gives an all-zero output row
  *   out         device bf16 [batch][q_heads][head_dim]
  *   scale       <= 0 selects 1/sqrt(head_dim)
- *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes;
- *               may be reused by later calls on the same stream
- * Runs two kernels on `stream`: a split-K flash-decoding pass that writes
- * fp32 partial (max, sum, output) triples, and a log-sum-exp merge.  Slots past
- * seq_lens[b] in the last page contribute nothing whatever they contain.
- * No host synchronisation; sequence lengths are read on the device.
+ *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes.  The
+ *               library keeps control words in it that are zero between calls:
+ *               it clears them whenever it sees a workspace pointer, batch or
+ *               head count it did not use in the previous call, so a workspace
+ *               may be shared by calls on one stream, but the caller must not
+ *               write to it between two calls that pass the same pointer.
+ * Work is split over the sequence (flash-decoding): every warp streams an
+ * equal share of the (sequence, kv head, page) blocks plus dynamically claimed
+ * chunks of a shared tail, and writes fp32 partial (max, sum, output) triples;
+ * the partials of a (sequence, kv head) are combined by a log-sum-exp merge,
+ * either by the warp that finishes the segment (default, one kernel) or by a
+ * separate merge kernel (skv_set_decode_merge_mode).  Slots past seq_lens[b]
+ * in the last page contribute nothing whatever they contain.  No host
+ * synchronisation; sequence lengths are read on the device.
  * Errors: SKV_ERR_ARG, SKV_ERR_LAYER, SKV_ERR_UNSUPPORTED (head ratio),
  * SKV_ERR_NOMEM (workspace), SKV_ERR_CUDA.  Device-side problems (page id out
- * of range, a bounded wait that ran out) are reported by skv_get_status. */
+ * of range, a bounded wait that ran out) are reported by skv_get_status; after
+ * SKV_ERR_TIMEOUT the outputs of that call are undefined. */
 int skv_decode_attn(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
                     const int32_t *seq_lens, void *out, int batch, int q_heads, int pt_stride,
                     float scale, void *workspace, size_t workspace_bytes, void *stream);
 
-/* The two halves of skv_decode_attn, separately launchable (profiling,
- * sequence-sharded use): the split-K pass fills `workspace`; the merge turns
- * the partials in `workspace` into `out`.  Same arguments and errors. */
+/* The two kernels separately (profiling, sequence-sharded use): the split-K
+ * pass fills `workspace` with partials; the merge kernel turns the partials in
+ * `workspace` into `out`.  Same arguments and errors. */
 int skv_decode_splitk(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
                       const int32_t *seq_lens, int batch, int q_heads, int pt_stride, float scale,
                       void *workspace, size_t workspace_bytes, void *stream);
-int skv_decode_merge(skv_cache *cache, const int32_t *seq_lens, void *out, int batch, int q_heads,
-                     void *workspace, size_t workspace_bytes, void *stream);
+int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *workspace,
+                     size_t workspace_bytes, void *stream);
 
 /* One whole decode step of Algorithm 2 with inputs already on the device:
  * for l = 0..L-1: append (owners only) then decode attention, on `stream`.
@@ -223,6 +235,24 @@ int skv_set_decode_variant(skv_cache *cache, int variant);
  * per warp (2..8) and CTAs per SM (1..8); 0 keeps the current value.
  * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
 int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
+
+/* 1 (default): skv_decode_attn merges inside the split-K kernel (the warp that
+ * completes a segment combines its partials); 0: it launches the merge kernel. */
+int skv_set_decode_merge_mode(skv_cache *cache, int fused);
+
+/* Load balance of the split-K pass: pool_percent (0..100) of the blocks are
+ * not assigned up front but claimed in chunks of at least min_chunk_blocks by
+ * warps that finish early; chunks_per_worker (1..64) bounds the number of
+ * chunks (and the workspace).  pool_percent 0 = fully static split. */
+int skv_set_decode_balance(skv_cache *cache, int pool_percent, int min_chunk_blocks, int chunks_per_worker);
+
+/* Tracing: while a device buffer of at least 32 * skv_decode_worker_count bytes
+ * is set, every split-K launch records four uint64 per worker (warp): SM id,
+ * kernel-entry time, time its first page arrived, exit time (global timer, ns).
+ * NULL switches tracing off.  skv_decode_worker_count = SMs * CTAs per SM *
+ * warps per CTA under the current tuning. */
+int skv_set_trace_buffer(skv_cache *cache, void *device_buffer, size_t bytes);
+int skv_decode_worker_count(const skv_cache *cache);
 
 /* Number of kernels this handle has launched so far. */
 int skv_launch_count(const skv_cache *cache, int64_t *out_count);

@@ -55,7 +55,7 @@ lib.skv_gather.argtypes = [_vp, _int, _i64p, _i64, _vp, _vp, _vp]
 lib.skv_decode_workspace_bytes.argtypes = [_vp, _int, _int, _szp]
 lib.skv_decode_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_splitk.argtypes = [_vp, _int, _vp, _i32p, _i32p, _int, _int, _int, _f32, _vp, _sz, _vp]
-lib.skv_decode_merge.argtypes = [_vp, _i32p, _vp, _int, _int, _vp, _sz, _vp]
+lib.skv_decode_merge.argtypes = [_vp, _vp, _int, _int, _vp, _sz, _vp]
 lib.skv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_step_staging_bytes.argtypes = [_vp, _int, _int, _int, _szp]
 lib.skv_decode_step_host.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32,
@@ -63,6 +63,10 @@ lib.skv_decode_step_host.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _v
 lib.skv_get_status.argtypes = [_vp, _vp, ctypes.POINTER(_int)]
 lib.skv_set_decode_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
+lib.skv_set_decode_merge_mode.argtypes = [_vp, _int]
+lib.skv_set_decode_balance.argtypes = [_vp, _int, _int, _int]
+lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
+lib.skv_decode_worker_count.argtypes = [_vp]
 lib.skv_launch_count.argtypes = [_vp, ctypes.POINTER(_i64)]
 lib.skv_plan_worker_range.argtypes = [_i64, _int, _int, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]
 lib.skv_plan_worker_of.argtypes = [_i64, _int, _i64]
@@ -236,10 +240,9 @@ class SkvCache:
                                    _stream_ptr(stream))
         _check(rc, "skv_decode_splitk")
 
-    def skv_decode_merge(self, seq_lens: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor,
-                         stream=None) -> None:
+    def skv_decode_merge(self, out: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
         batch, q_heads = out.shape[0], out.shape[1]
-        rc = lib.skv_decode_merge(self._h, _ptr(seq_lens), _ptr(out), batch, q_heads, _ptr(workspace),
+        rc = lib.skv_decode_merge(self._h, _ptr(out), batch, q_heads, _ptr(workspace),
                                   workspace.numel(), _stream_ptr(stream))
         _check(rc, "skv_decode_merge")
 
@@ -278,6 +281,23 @@ class SkvCache:
 
     def skv_set_decode_tuning(self, warps_per_cta: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
         _check(lib.skv_set_decode_tuning(self._h, warps_per_cta, stages, ctas_per_sm), "skv_set_decode_tuning")
+
+    def skv_set_decode_merge_mode(self, fused: int) -> None:
+        _check(lib.skv_set_decode_merge_mode(self._h, fused), "skv_set_decode_merge_mode")
+
+    def skv_set_decode_balance(self, pool_percent: int, min_chunk_blocks: int = 2, chunks_per_worker: int = 8) -> None:
+        _check(lib.skv_set_decode_balance(self._h, pool_percent, min_chunk_blocks, chunks_per_worker),
+               "skv_set_decode_balance")
+
+    def skv_set_trace_buffer(self, buf: Optional[torch.Tensor]) -> None:
+        _check(lib.skv_set_trace_buffer(self._h, _ptr(buf), 0 if buf is None else buf.numel() * buf.element_size()),
+               "skv_set_trace_buffer")
+
+    def skv_decode_worker_count(self) -> int:
+        rc = lib.skv_decode_worker_count(self._h)
+        if rc < 0:
+            raise SkvError(rc, "skv_decode_worker_count")
+        return rc
 
     def skv_launch_count(self) -> int:
         out = _i64(0)

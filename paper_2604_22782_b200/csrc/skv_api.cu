@@ -22,8 +22,14 @@ struct skv_cache {
     size_t page_bytes = 0;           // one page of one owner layer
     int sm_count = 0;
     int max_smem_optin = 0;
-    DecodeTuning tune{0, 4, 3, 2};
+    DecodeTuning tune{0, 4, 3, 2, 1, Balance{20, 2, 0}};
+    int chunks_per_worker = 8;       // pool chunk slots per worker (sizes the workspace)
+    // the decode workspace whose control words are known to be zero (see prepare_workspace)
+    const void *ws_ready = nullptr;
+    int ws_batch = 0, ws_q_heads = 0, ws_workers = 0, ws_chunks = 0;
     int64_t launches = 0;
+    unsigned long long *trace = nullptr;   // optional per-worker timestamps (device)
+    size_t trace_bytes = 0;
 
     int *status_word() const { return reinterpret_cast<int *>(pool); }
     uint8_t *layer_base(int owner_slot) const
@@ -61,23 +67,57 @@ bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t o_off, ml_off, prefix_off, total;
+    size_t ctrl_off, seg_off, prefix_off, ml_off, o_off, total, zero_bytes;
     int64_t n_slots;
 };
 
-WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int n_workers)
+// control words | per-segment block counters | page-count prefix | partial (max,sum) | partial outputs
+WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int n_workers, int max_chunks)
 {
     WorkspaceLayout w;
     const int G = q_heads / c->kv_heads;
-    w.n_slots = (int64_t)n_workers + (int64_t)batch * c->kv_heads;
-    w.o_off = 0;
-    w.ml_off = round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
-    w.prefix_off = w.ml_off + round_up((size_t)w.n_slots * G * 2 * sizeof(float), 256);
-    w.total = w.prefix_off + round_up((size_t)(batch + 1) * sizeof(int32_t), 256);
+    const int64_t n_seg = (int64_t)batch * c->kv_heads;
+    w.n_slots = (int64_t)n_workers + n_seg + (int64_t)max_chunks + n_seg;
+    w.ctrl_off = 0;
+    w.seg_off = 256;
+    w.prefix_off = w.seg_off + round_up((size_t)n_seg * sizeof(int32_t), 256);
+    w.zero_bytes = w.prefix_off;
+    w.ml_off = w.prefix_off + round_up((size_t)(batch + 1) * sizeof(int32_t), 256);
+    w.o_off = w.ml_off + round_up((size_t)w.n_slots * G * 2 * sizeof(float), 256);
+    w.total = w.o_off + round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
     return w;
 }
 
 int n_workers_of(const skv_cache *c) { return c->sm_count * c->tune.ctas_per_sm * c->tune.warps; }
+
+int max_chunks_of(const skv_cache *c) { return c->tune.bal.pool_pct > 0 ? c->chunks_per_worker * n_workers_of(c) : 0; }
+
+Balance balance_of(const skv_cache *c)
+{
+    Balance b = c->tune.bal;
+    b.max_chunks = max_chunks_of(c);
+    return b;
+}
+
+// The split-K kernel expects its control words and per-segment counters to be zero on entry and leaves
+// them zero on exit, so they are cleared only when the workspace (or the layout in it) changes.
+int prepare_workspace(skv_cache *c, void *workspace, const WorkspaceLayout &wl, int batch, int q_heads, cudaStream_t st)
+{
+    const int W = n_workers_of(c), ch = max_chunks_of(c);
+    if (c->ws_ready == workspace && c->ws_batch == batch && c->ws_q_heads == q_heads && c->ws_workers == W &&
+        c->ws_chunks == ch)
+        return SKV_OK;
+    if (cudaMemsetAsync(workspace, 0, wl.zero_bytes, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SKV_ERR_CUDA;
+    }
+    c->ws_ready = workspace;
+    c->ws_batch = batch;
+    c->ws_q_heads = q_heads;
+    c->ws_workers = W;
+    c->ws_chunks = ch;
+    return SKV_OK;
+}
 
 int check_decode_args(const skv_cache *c, int layer, int batch, int q_heads)
 {
@@ -276,28 +316,32 @@ int skv_decode_workspace_bytes(const skv_cache *c, int batch, int q_heads, size_
 {
     if (!c || !out_bytes || batch <= 0 || q_heads <= 0) return SKV_ERR_ARG;
     if (q_heads % c->kv_heads != 0 || q_heads / c->kv_heads > 8) return SKV_ERR_UNSUPPORTED;
-    // sized for the largest worker count any tuning can select, so that the
-    // workspace stays valid when the launch shape is changed later
     const int sm = c->sm_count > 0 ? c->sm_count : 148;
-    const int max_workers = sm * 64;                 // an SM holds at most 64 warps
-    *out_bytes = workspace_layout(c, batch, q_heads, max_workers).total;
+    const int W = sm * c->tune.ctas_per_sm * c->tune.warps;
+    const int ch = c->tune.bal.pool_pct > 0 ? c->chunks_per_worker * W : 0;
+    *out_bytes = workspace_layout(c, batch, q_heads, W, ch).total;
     return SKV_OK;
 }
 
-int skv_decode_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
-                      int batch, int q_heads, int pt_stride, float scale, void *workspace,
-                      size_t workspace_bytes, void *stream)
+namespace {
+// launches the split-K kernel; `out` non-null selects the fused (in-kernel) merge
+int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
+                  void *out, int batch, int q_heads, int pt_stride, float scale, void *workspace,
+                  size_t workspace_bytes, void *stream)
 {
     int rc = check_decode_args(c, layer, batch, q_heads);
     if (rc) return rc;
     if (!Q || !page_table || !seq_lens || !workspace || pt_stride <= 0) return SKV_ERR_ARG;
-    if (!aligned(Q, 16) || !aligned(workspace, 256)) return SKV_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(workspace, 256) || (out && !aligned(out, 8))) return SKV_ERR_ARG;
     const int G = q_heads / c->kv_heads;
     const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W, max_chunks_of(c));
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
     const size_t smem = decode_smem_bytes(c->head_dim, batch, c->tune.warps, c->tune.stages);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = prepare_workspace(c, workspace, wl, batch, q_heads, st);
+    if (rc) return rc;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     DecodeParams p;
     p.layer_base = c->layer_base(c->slot[(size_t)c->r[(size_t)layer]]);
@@ -309,43 +353,56 @@ int skv_decode_splitk(skv_cache *c, int layer, const void *Q, const int32_t *pag
     p.part_o = reinterpret_cast<float *>(ws + wl.o_off);
     p.part_ml = reinterpret_cast<float *>(ws + wl.ml_off);
     p.prefix = reinterpret_cast<int32_t *>(ws + wl.prefix_off);
+    p.ctrl = reinterpret_cast<int32_t *>(ws + wl.ctrl_off);
+    p.seg_count = reinterpret_cast<int32_t *>(ws + wl.seg_off);
+    p.out = static_cast<uint16_t *>(out);
     p.B = batch;
     p.Hq = q_heads;
     p.Hkv = c->kv_heads;
     p.pt_stride = pt_stride;
     const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)c->head_dim);
     p.scale_log2 = sc * 1.4426950408889634f;
+    p.bal = balance_of(c);
     p.status = c->status_word();
+    p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
     const bool tensor_core = c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
     const int grid = c->sm_count * c->tune.ctas_per_sm;
-    if (launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, c->tune.warps, c->tune.stages,
-                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, c->tune.warps, c->tune.stages, st) != cudaSuccess)
         return SKV_ERR_CUDA;
     c->launches += 1;
     return SKV_OK;
 }
+}  // namespace
 
-int skv_decode_merge(skv_cache *c, const int32_t *seq_lens, void *out, int batch, int q_heads, void *workspace,
-                     size_t workspace_bytes, void *stream)
+int skv_decode_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
+                      int batch, int q_heads, int pt_stride, float scale, void *workspace,
+                      size_t workspace_bytes, void *stream)
+{
+    return launch_splitk(c, layer, Q, page_table, seq_lens, nullptr, batch, q_heads, pt_stride, scale, workspace,
+                         workspace_bytes, stream);
+}
+
+int skv_decode_merge(skv_cache *c, void *out, int batch, int q_heads, void *workspace, size_t workspace_bytes,
+                     void *stream)
 {
     int rc = check_decode_args(c, 0, batch, q_heads);
     if (rc) return rc;
-    if (!seq_lens || !out || !workspace || !aligned(out, 8) || !aligned(workspace, 256)) return SKV_ERR_ARG;
+    if (!out || !workspace || !aligned(out, 8) || !aligned(workspace, 256)) return SKV_ERR_ARG;
     const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W, max_chunks_of(c));
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     MergeParams m;
     m.part_o = reinterpret_cast<const float *>(ws + wl.o_off);
     m.part_ml = reinterpret_cast<const float *>(ws + wl.ml_off);
     m.prefix = reinterpret_cast<const int32_t *>(ws + wl.prefix_off);
-    m.seq_lens = seq_lens;
     m.out = static_cast<uint16_t *>(out);
     m.B = batch;
     m.Hq = q_heads;
     m.Hkv = c->kv_heads;
     m.D = c->head_dim;
     m.n_workers = W;
+    m.bal = balance_of(c);
     if (launch_merge(m, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
     c->launches += 1;
     return SKV_OK;
@@ -356,10 +413,13 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
                     size_t workspace_bytes, void *stream)
 {
     if (!out) return SKV_ERR_ARG;
+    if (c && c->tune.fused_merge)
+        return launch_splitk(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, workspace,
+                             workspace_bytes, stream);
     int rc = skv_decode_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
                                workspace_bytes, stream);
     if (rc) return rc;
-    return skv_decode_merge(c, seq_lens, out, batch, q_heads, workspace, workspace_bytes, stream);
+    return skv_decode_merge(c, out, batch, q_heads, workspace, workspace_bytes, stream);
 }
 
 int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, const int64_t *slot_map,
@@ -474,6 +534,7 @@ int skv_get_status(skv_cache *c, void *stream, int *device_status)
         return SKV_ERR_CUDA;
     }
     *device_status = (word & STATUS_TIMEOUT) ? SKV_ERR_TIMEOUT : (word & STATUS_BOUNDS) ? SKV_ERR_BOUNDS : SKV_OK;
+    if (word & STATUS_TIMEOUT) c->ws_ready = nullptr;     // a worker gave up: counters may be left non-zero
     return SKV_OK;
 }
 
@@ -499,6 +560,38 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     }
     c->tune = t;
     return SKV_OK;
+}
+
+int skv_set_decode_merge_mode(skv_cache *c, int fused)
+{
+    if (!c || fused < 0 || fused > 1) return SKV_ERR_ARG;
+    c->tune.fused_merge = fused;
+    return SKV_OK;
+}
+
+int skv_set_decode_balance(skv_cache *c, int pool_percent, int min_chunk_blocks, int chunks_per_worker)
+{
+    if (!c || pool_percent < 0 || pool_percent > 100 || min_chunk_blocks < 1 || chunks_per_worker < 1 ||
+        chunks_per_worker > 64)
+        return SKV_ERR_ARG;
+    c->tune.bal.pool_pct = pool_percent;
+    c->tune.bal.min_chunk = min_chunk_blocks;
+    c->chunks_per_worker = chunks_per_worker;
+    return SKV_OK;
+}
+
+int skv_set_trace_buffer(skv_cache *c, void *device_buffer, size_t bytes)
+{
+    if (!c || (device_buffer && !aligned(device_buffer, 8))) return SKV_ERR_ARG;
+    c->trace = static_cast<unsigned long long *>(device_buffer);
+    c->trace_bytes = device_buffer ? bytes : 0;
+    return SKV_OK;
+}
+
+int skv_decode_worker_count(const skv_cache *c)
+{
+    if (!c || !c->pool) return SKV_ERR_ARG;
+    return n_workers_of(c);
 }
 
 int skv_launch_count(const skv_cache *c, int64_t *out_count)

@@ -50,6 +50,35 @@ struct GatherParams {
     int *status;
 };
 
+// How one decode call's blocks are handed to the W workers (warps).  The
+// flattened block list [0, T) is cut in two: [0, Ts) is split statically into
+// W equal contiguous ranges; the tail [Ts, T) (the "pool") is cut into chunks
+// of `chunk` blocks that workers claim one at a time from an atomic counter
+// once their static range is done, so that faster SMs take more of the work.
+struct Plan {
+    int64_t T, Ts;
+    int chunk, n_chunks;
+};
+
+struct Balance {
+    int pool_pct;       // share of the blocks that goes to the pool (0 = fully static)
+    int min_chunk;      // smallest pool chunk, in blocks
+    int max_chunks;     // upper bound on the number of pool chunks (sizes the workspace)
+};
+
+__host__ __device__ inline Plan make_plan(int64_t T, const Balance &b)
+{
+    Plan pl;
+    pl.T = T;
+    int64_t pool = b.max_chunks > 0 ? (T * b.pool_pct) / 100 : 0;
+    int64_t c = b.min_chunk > 0 ? b.min_chunk : 1;
+    if (pool > c * b.max_chunks) c = (pool + b.max_chunks - 1) / b.max_chunks;
+    pl.chunk = (int)c;
+    pl.n_chunks = (int)((pool + c - 1) / c);
+    pl.Ts = T - pool;
+    return pl;
+}
+
 struct DecodeParams {
     const uint8_t *layer_base;  // first page of the owner layer that is read
     int64_t page_stride;
@@ -60,19 +89,24 @@ struct DecodeParams {
     float *part_o;              // [n_slots][G][D]
     float *part_ml;             // [n_slots][G][2]  (running max in log2 units, sum)
     int32_t *prefix;            // [B+1] cumulative page counts (written by CTA 0)
+    int32_t *ctrl;              // [0] pool claim counter, [1] exited-worker counter (both 0 between launches)
+    int32_t *seg_count;         // [B*Hkv] blocks finished per segment (0 between launches); fused merge only
+    uint16_t *out;              // [B][Hq][D] bf16 bits: non-null = merge inside this kernel (last arriver)
     int B, Hq, Hkv, pt_stride;
     float scale_log2;           // scale * log2(e)
+    Balance bal;
     int *status;
+    unsigned long long *trace;  // optional [n_workers][4]: sm id, entry ns, first-page ns, exit ns
 };
 
 struct MergeParams {
     const float *part_o;
     const float *part_ml;
     const int32_t *prefix;      // [B+1]
-    const int32_t *seq_lens;
     uint16_t *out;              // [B][Hq][D] bf16 bits
     int B, Hq, Hkv, D;
     int n_workers;
+    Balance bal;
 };
 
 struct DecodeTuning {
@@ -80,6 +114,8 @@ struct DecodeTuning {
     int warps;                  // per CTA
     int stages;                 // per warp
     int ctas_per_sm;
+    int fused_merge;            // 1: the split-K kernel's last arriver per segment merges
+    Balance bal;
 };
 
 // host launchers (each returns a cudaError_t from the launch)

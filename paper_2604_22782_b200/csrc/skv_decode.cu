@@ -259,20 +259,130 @@ struct CudaCoreState {
 };
 
 // ---------------------------------------------------------------------------
+// Where the partials of one segment (sequence b, kv head kvh) live.  A static
+// range that meets the segment wrote slot  worker + seg;  a pool chunk that
+// meets it wrote slot  W + n_seg + chunk + seg.  Lane k of the calling warp
+// gets the k-th partial's slot (or -1); returns how many there are.  A segment
+// with more than 32 partials is walked in rounds of 32 (`round`).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ int partial_slots(const Plan &pl, int64_t W, int64_t n_seg, int64_t s0, int pages,
+                                             int64_t seg, int lane, int round, int64_t &slot)
+{
+    const int64_t s1 = s0 + pages;
+    int n_static = 0;
+    int64_t w_first = 0;
+    const bool sparse = pl.Ts < W;            // then every non-empty static range is a single block
+    if (s0 < pl.Ts) {
+        const int64_t e = s1 < pl.Ts ? s1 : pl.Ts;
+        if (sparse) {
+            n_static = (int)(e - s0);
+        } else {
+            w_first = worker_of(s0, pl.Ts, W);
+            n_static = worker_of(e - 1, pl.Ts, W) - (int)w_first + 1;
+        }
+    }
+    int n_pool = 0;
+    int64_t j_first = 0;
+    if (s1 > pl.Ts && pl.n_chunks > 0) {
+        const int64_t a = s0 > pl.Ts ? s0 : pl.Ts;
+        j_first = (a - pl.Ts) / pl.chunk;
+        n_pool = (int)((s1 - 1 - pl.Ts) / pl.chunk - j_first) + 1;
+    }
+    const int k = round * 32 + lane;
+    slot = -1;
+    if (k < n_static) slot = (sparse ? (int64_t)worker_of(s0 + k, pl.Ts, W) : w_first + k) + seg;
+    else if (k < n_static + n_pool) slot = W + n_seg + j_first + (k - n_static) + seg;
+    return n_static + n_pool;
+}
+
+// Log-sum-exp merge of one segment's partials for its G query heads, by one warp:
+// out[b, kvh*G+g, :] = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i,  M = max_i m_i.
+template <int D>
+__device__ __noinline__ void merge_segment(const float *part_o, const float *part_ml, uint16_t *out,
+                                              const Plan &pl, int64_t W, int B, int Hq, int Hkv, int b, int kvh,
+                                              int64_t s0, int pages, int lane)
+{
+    constexpr int PER = D / 32;               // consecutive output dims per lane
+    const int G = Hq / Hkv;
+    const int64_t seg = (int64_t)b * Hkv + kvh, n_seg = (int64_t)B * Hkv;
+    int64_t slot;
+    const int n = partial_slots(pl, W, n_seg, s0, pages, seg, lane, 0, slot);
+    for (int g = 0; g < G; ++g) {
+        float acc[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+        float M = -INFINITY, L = 0.f;
+        for (int r = 0; r * 32 < n; ++r) {
+            int64_t my = slot;
+            if (r > 0) partial_slots(pl, W, n_seg, s0, pages, seg, lane, r, my);
+            // this round's (max, sum) pairs, one partial per lane
+            float2 ml = make_float2(-INFINITY, 0.f);
+            if (my >= 0) ml = __ldcg(reinterpret_cast<const float2 *>(part_ml + (my * G + g) * 2));
+            float Mr = ml.x;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) Mr = fmaxf(Mr, __shfl_xor_sync(FULL, Mr, d));
+            const float M_new = fmaxf(M, Mr);
+            const float keep = exp2f(M - M_new);          // 0 on the first round
+            const float wt = (my >= 0) ? exp2f(ml.x - M_new) : 0.f;
+            float Lr = wt * ml.y;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) Lr += __shfl_xor_sync(FULL, Lr, d);
+            L = L * keep + Lr;
+            M = M_new;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) acc[i] *= keep;
+            const int cnt = (n - r * 32) < 32 ? (n - r * 32) : 32;
+            for (int i0 = 0; i0 < cnt; i0 += 4) {
+                float v[4][PER], wv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = (i0 + u) < cnt ? (i0 + u) : i0;       // clamp: weight 0 below
+                    const int64_t sl = __shfl_sync(FULL, my, i);
+                    wv[u] = (i0 + u) < cnt ? __shfl_sync(FULL, wt, i) : 0.f;
+                    const float *po = part_o + (sl * G + g) * D + lane * PER;
+                    if constexpr (PER == 4) {
+                        const float4 t = __ldcg(reinterpret_cast<const float4 *>(po));
+                        v[u][0] = t.x; v[u][1] = t.y; v[u][2] = t.z; v[u][3] = t.w;
+                    } else {
+                        const float2 t = __ldcg(reinterpret_cast<const float2 *>(po));
+                        v[u][0] = t.x; v[u][1] = t.y;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int i = 0; i < PER; ++i) acc[i] = fmaf(wv[u], v[u][i], acc[i]);
+            }
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        uint16_t *dst = out + ((int64_t)b * Hq + (int64_t)kvh * G + g) * D + lane * PER;
+#pragma unroll
+        for (int i = 0; i < PER; i += 2)
+            *reinterpret_cast<uint32_t *>(dst + i) = pack_bf16x2(acc[i] * inv, acc[i + 1] * inv);
+    }
+}
+
+// ---------------------------------------------------------------------------
 template <int D, class State>
 __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = block_bytes(D);
+    constexpr int QLEN = 8;                   // per-warp queue of range ids between producer and consumer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint64_t t_entry = p.trace ? global_timer_ns() : 0;
+    uint64_t t_first = 0;
 
-    // carve shared memory: prefix | rings | barriers   (ring base rounded up to 128 bytes)
+    // carve shared memory: prefix | rings | barriers | range queues  (ring base rounded up to 128 bytes)
     const uint32_t base = smem_u32(smem_raw);
     const uint32_t pad = (128u - (base & 127u)) & 127u;
     int32_t *prefix = reinterpret_cast<int32_t *>(smem_raw + pad);
-    const uint32_t rings = base + pad + (uint32_t)prefix_bytes(p.B);
+    const size_t rings_off = pad + prefix_bytes(p.B);
+    const uint32_t rings = base + (uint32_t)rings_off;
     const uint32_t ring = rings + (uint32_t)(warp * stages * BLOCK);
-    const uint32_t bars = rings + (uint32_t)(nwarps * stages * BLOCK) + (uint32_t)(warp * stages * 8);
+    const size_t bars_off = rings_off + (size_t)nwarps * stages * BLOCK;
+    const uint32_t bars = base + (uint32_t)bars_off + (uint32_t)(warp * stages * 8);
+    int32_t *queue = reinterpret_cast<int32_t *>(smem_raw + bars_off + (size_t)nwarps * stages * 8) + warp * QLEN;
 
     if (lane == 0) {
         for (int s = 0; s < stages; ++s) mbar_init(bars + 8 * s, 1);
@@ -299,23 +409,64 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
         if (lane == 0) prefix[0] = 0;
     }
     __syncthreads();
-    if (blockIdx.x == 0)
+    if (blockIdx.x == 0) {
         for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.prefix[i] = prefix[i];
+        if (p.out) {     // fused merge: rows of empty sequences are zero and belong to nobody else
+            const int row_words = p.Hq * D / 2;
+            for (int b = 0; b < p.B; ++b)
+                if (prefix[b + 1] == prefix[b])
+                    for (int i = threadIdx.x; i < row_words; i += blockDim.x)
+                        reinterpret_cast<uint32_t *>(p.out)[(int64_t)b * row_words + i] = 0u;
+        }
+    }
 
     const int64_t W = (int64_t)gridDim.x * nwarps, w = (int64_t)blockIdx.x * nwarps + warp;
-    const int64_t T = (int64_t)prefix[p.B] * p.Hkv;
-    if (T == 0) return;
-    const int64_t x0 = worker_begin(w, T, W), x1 = worker_begin(w + 1, T, W);
-    const int n = (int)(x1 - x0);
-    if (n <= 0) return;
+    const int64_t n_seg = (int64_t)p.B * p.Hkv;
+    const Plan pl = make_plan((int64_t)prefix[p.B] * p.Hkv, p.bal);
+    if (pl.T == 0) return;
+    const bool pooled = pl.n_chunks > 0;
 
-    Cursor prod = locate(prefix, p.B, p.Hkv, x0);
-    Cursor cons = prod;
+    // static range of this worker
+    const int64_t x0 = worker_begin(w, pl.Ts, W);
+    const int n_static = (int)(worker_begin(w + 1, pl.Ts, W) - x0);
+    // first pool claim, requested now and looked at only when the static range has been issued
+    int next_j = 0;
+    if (pooled && lane == 0) next_j = atomicAdd(p.ctrl, 1);
 
-    // producer side: page ids of the current sequence are fetched 32 at a time, one per lane
-    int win_b = -1, win_base = 0, win_ids = 0;
-    int issued = 0, p_stage = 0;
-    auto issue = [&]() {
+    // ---- producer: walks ranges (static, then claimed chunks) and keeps the ring full ----
+    Cursor prod = {0, 0, 0, 0};
+    int prod_left = 0, q_tail = 0, in_flight = 0, p_stage = 0;
+    bool static_given = false, prod_done = false;
+    int win_b = -1, win_base = 0, win_ids = 0;   // page ids of the current sequence, 32 at a time, one per lane
+    auto issue = [&]() -> bool {
+        if (prod_done) return false;
+        if (prod_left == 0) {
+            int id = -1, cnt = 0;
+            int64_t begin = 0;
+            if (!static_given) {
+                static_given = true;
+                begin = x0;
+                cnt = n_static;
+            }
+            if (cnt == 0 && pooled) {
+                const int j = __shfl_sync(FULL, next_j, 0);
+                if (j < pl.n_chunks) {
+                    if (lane == 0) next_j = atomicAdd(p.ctrl, 1);
+                    id = j;
+                    begin = pl.Ts + (int64_t)j * pl.chunk;
+                    const int64_t rest = pl.T - begin;
+                    cnt = rest < pl.chunk ? (int)rest : pl.chunk;
+                }
+            }
+            if (cnt == 0) {
+                prod_done = true;
+                return false;
+            }
+            if (lane == 0) queue[q_tail & (QLEN - 1)] = id;
+            ++q_tail;
+            prod = locate(prefix, p.B, p.Hkv, begin);
+            prod_left = cnt;
+        }
         if (prod.b != win_b || prod.pg < win_base || prod.pg >= win_base + 32) {
             win_b = prod.b;
             win_base = prod.pg;
@@ -334,18 +485,43 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
             bulk_copy_g2s(ring + (uint32_t)(p_stage * BLOCK), src, BLOCK, bar);
         }
         if (++p_stage == stages) p_stage = 0;
-        if (++issued < n) advance(prod, prefix, p.Hkv);
+        ++in_flight;
+        if (--prod_left > 0) advance(prod, prefix, p.Hkv);
+        return true;
     };
-    const int prime = n < stages ? n : stages;
-    for (int i = 0; i < prime; ++i) issue();
+    // the queue holds at most `stages`+1 ranges: a range is queued only when one of its blocks is issued
+    while (in_flight < stages && issue()) {}
 
+    // ---- consumer ----
     State st;
-    int c_stage = 0;
+    Cursor cons = {0, 0, 0, 0};
+    int cons_left = 0, q_head = 0, c_stage = 0, run_pages = 0, n_b = 0;
+    int64_t slot_base = 0;
     uint32_t parity = 0;
-    bool fresh = true;
-    for (int i = 0; i < n; ++i) {
+    bool fresh = true, first = true, failed = false;
+    while (in_flight > 0) {
+        if (cons_left == 0) {
+            __syncwarp();
+            const int id = queue[q_head & (QLEN - 1)];
+            ++q_head;
+            int64_t begin;
+            if (id < 0) {
+                begin = x0;
+                cons_left = n_static;
+                slot_base = w;
+            } else {
+                begin = pl.Ts + (int64_t)id * pl.chunk;
+                const int64_t rest = pl.T - begin;
+                cons_left = rest < pl.chunk ? (int)rest : pl.chunk;
+                slot_base = W + n_seg + id;
+            }
+            cons = locate(prefix, p.B, p.Hkv, begin);
+            fresh = true;
+        }
         if (fresh) {
             st.begin(p, cons.b, cons.h, G, lane);
+            n_b = __ldg(p.seq_lens + cons.b);
+            run_pages = 0;
             fresh = false;
         }
         const bool ok = mbar_wait_bounded(bars + 8 * c_stage, parity);
@@ -354,72 +530,83 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
             if (lane == 0) atomicOr(p.status, STATUS_TIMEOUT);
             int s = c_stage;
             uint32_t par = parity;
-            for (int k = i + 1; k < issued; ++k) {
+            for (int k = 1; k < in_flight; ++k) {
                 if (++s == stages) { s = 0; par ^= 1u; }
                 mbar_wait_bounded(bars + 8 * s, par);
             }
-            return;
+            failed = true;
+            break;
         }
+        if (p.trace && first) t_first = global_timer_ns();
+        first = false;
         const uint32_t sK = ring + (uint32_t)(c_stage * BLOCK);
-        const int n_b = __ldg(p.seq_lens + cons.b);
         const int left = n_b - cons.pg * PAGE;
         st.page(sK, sK + half_bytes(D), left < PAGE ? left : PAGE, p.scale_log2, lane);
         __syncwarp();                       // every lane is done reading this stage
-        if (issued < n) issue();            // refill it
+        --in_flight;
+        issue();                            // refill it
         if (++c_stage == stages) { c_stage = 0; parity ^= 1u; }
-        const bool seg_end = (cons.pg + 1 == cons.pages) || (i + 1 == n);
-        if (seg_end) {
-            st.finish(p, w + (int64_t)cons.b * p.Hkv + cons.h, G, lane);
+        ++run_pages;
+        --cons_left;
+        if (cons.pg + 1 == cons.pages || cons_left == 0) {
+            // this worker's run inside segment (b, h) ends: publish the partial
+            const int64_t seg = (int64_t)cons.b * p.Hkv + cons.h;
+            st.finish(p, slot_base + seg, G, lane);
+            if (p.out) {
+                // the worker that completes the segment's block count merges it
+                __threadfence();
+                __syncwarp();
+                int done = 0;
+                if (lane == 0) done = atomicAdd(p.seg_count + seg, run_pages) + run_pages;
+                done = __shfl_sync(FULL, done, 0);
+                if (done == cons.pages) {
+                    __threadfence();
+                    const int64_t s0 = (int64_t)prefix[cons.b] * p.Hkv + (int64_t)cons.h * cons.pages;
+                    merge_segment<D>(p.part_o, p.part_ml, p.out, pl, W, p.B, p.Hq, p.Hkv, cons.b, cons.h, s0,
+                                     cons.pages, lane);
+                    if (lane == 0) p.seg_count[seg] = 0;
+                }
+            }
             fresh = true;
         }
-        if (i + 1 < n) advance(cons, prefix, p.Hkv);
+        if (cons_left > 0) advance(cons, prefix, p.Hkv);
+    }
+    (void)failed;
+    // the last worker to leave puts the two counters back to zero for the next launch
+    if (pooled && lane == 0) {
+        if (atomicAdd(p.ctrl + 1, 1) == (int)W - 1) {
+            p.ctrl[0] = 0;
+            p.ctrl[1] = 0;
+        }
+    }
+    if (p.trace && lane == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        unsigned long long *t = p.trace + 4 * w;
+        t[0] = smid; t[1] = t_entry; t[2] = t_first; t[3] = global_timer_ns();
     }
 }
 
 // ---------------------------------------------------------------------------
-// Merge: out[b,hq,:] = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i over the
-// partials of segment (b, hq / G), M = max_i m_i; one warp per output row.
+// Stand-alone merge kernel: one warp per (sequence, kv head) segment.
 // ---------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(128) merge_kernel(MergeParams p)
 {
-    constexpr int PER = D / 32;          // consecutive output dims per lane
     const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (row >= (int64_t)p.B * p.Hq) return;
-    const int b = (int)(row / p.Hq), hq = (int)(row - (int64_t)b * p.Hq);
-    const int G = p.Hq / p.Hkv, kvh = hq / G, g = hq - kvh * G;
-    uint16_t *dst = p.out + row * D + lane * PER;
+    const int64_t seg = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (seg >= (int64_t)p.B * p.Hkv) return;
+    const int b = (int)(seg / p.Hkv), kvh = (int)(seg - (int64_t)b * p.Hkv);
     const int pages = p.prefix[b + 1] - p.prefix[b];
-    float acc[PER];
-#pragma unroll
-    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
-    float L = 0.f;
-    if (pages > 0) {
-        const int64_t W = p.n_workers;
-        const int64_t T = (int64_t)p.prefix[p.B] * p.Hkv;
-        const int64_t s0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)kvh * pages;
-        const int64_t s1 = s0 + pages, seg = (int64_t)b * p.Hkv + kvh;
-        float M = -INFINITY;
-        // walk the workers whose (non-empty) ranges meet [s0, s1); running-max merge
-        for (int64_t x = s0; x < s1;) {
-            const int w = worker_of(x, T, W);
-            const int64_t at = (w + seg) * G + g;
-            const float2 ml = *reinterpret_cast<const float2 *>(p.part_ml + at * 2);
-            const float M_new = fmaxf(M, ml.x);
-            const float keep = exp2f(M - M_new), wt = exp2f(ml.x - M_new);
-            M = M_new;
-            L = L * keep + wt * ml.y;
-            const float *po = p.part_o + at * D + lane * PER;
-#pragma unroll
-            for (int i = 0; i < PER; ++i) acc[i] = acc[i] * keep + wt * po[i];
-            x = worker_begin((int64_t)w + 1, T, W);
-        }
+    const int G = p.Hq / p.Hkv;
+    if (pages == 0) {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)kvh * G) * D);
+        for (int i = lane; i < G * D / 2; i += 32) dst[i] = 0u;
+        return;
     }
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-#pragma unroll
-    for (int i = 0; i < PER; i += 2)
-        *reinterpret_cast<uint32_t *>(dst + i) = pack_bf16x2(acc[i] * inv, acc[i + 1] * inv);
+    const Plan pl = make_plan((int64_t)p.prefix[p.B] * p.Hkv, p.bal);
+    const int64_t s0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)kvh * pages;
+    merge_segment<D>(p.part_o, p.part_ml, p.out, pl, p.n_workers, p.B, p.Hq, p.Hkv, b, kvh, s0, pages, lane);
 }
 
 template <int D, class State>
@@ -438,8 +625,9 @@ cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, i
 size_t decode_smem_bytes(int D, int B, int warps, int stages)
 {
     if (D != 64 && D != 128) return 0;
-    // 128 bytes of slack for aligning the ring base
-    return 128 + prefix_bytes(B) + (size_t)warps * stages * block_bytes(D) + (size_t)warps * stages * 8;
+    // 128 bytes of slack for aligning the ring base; 8 queue entries per warp
+    return 128 + prefix_bytes(B) + (size_t)warps * stages * block_bytes(D) + (size_t)warps * stages * 8 +
+           (size_t)warps * 8 * 4;
 }
 
 cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid, int warps,
@@ -458,8 +646,8 @@ cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tenso
 
 cudaError_t launch_merge(const MergeParams &p, cudaStream_t s)
 {
-    const int64_t rows = (int64_t)p.B * p.Hq;
-    const unsigned blocks = (unsigned)((rows + 3) / 4);
+    const int64_t segs = (int64_t)p.B * p.Hkv;
+    const unsigned blocks = (unsigned)((segs + 3) / 4);
     if (p.D == 128) merge_kernel<128><<<blocks, 128, 0, s>>>(p);
     else if (p.D == 64) merge_kernel<64><<<blocks, 128, 0, s>>>(p);
     else return cudaErrorInvalidValue;

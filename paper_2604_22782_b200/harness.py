@@ -37,6 +37,20 @@ class DeviceWorkload:
     def owners(self) -> List[int]:
         return [l for l in range(self.w.n_layers) if self.r[l] == l]
 
+    def retune(self, variant=None, tuning=None, merge_mode=None, balance=None) -> None:
+        """Change kernel variant / launch shape / merge mode / balance, then size the workspace again."""
+        if variant is not None:
+            self.cache.skv_set_decode_variant(variant)
+        if tuning is not None:
+            self.cache.skv_set_decode_tuning(*tuning)
+        if merge_mode is not None:
+            self.cache.skv_set_decode_merge_mode(merge_mode)
+        if balance is not None:
+            self.cache.skv_set_decode_balance(*balance)
+        need = self.cache.skv_decode_workspace_bytes(self.batch, self.w.q_heads)
+        if need > self.workspace.numel():
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+
     def kv_bytes_per_call(self) -> int:
         """Algorithmic bytes of one decode-attention call: the owner layer's K,V of
         every attended token, plus Q in and out out."""

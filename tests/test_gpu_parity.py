@@ -50,16 +50,14 @@ def _decode_layer(dw, layer, Q=None, scale=0.0):
     return Q, out
 
 
-def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True):
+def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True,
+                     merge_mode=None, balance=None):
     """One decode step of every layer: prefill n-1 tokens, append the last one, attend; compare all."""
     harness, dw = _make(w, lens=lens, r=r, permute=permute)
     if poison:   # every byte of the page area becomes a bf16 NaN pattern (0x7FC1)
         dw.pool_view = dw.cache.pool[256:].view(torch.int16)
         dw.pool_view.fill_(0x7FC1)
-    if variant:
-        dw.cache.skv_set_decode_variant(variant)
-    if tuning:
-        dw.cache.skv_set_decode_tuning(*tuning)
+    dw.retune(variant=variant or None, tuning=tuning, merge_mode=merge_mode, balance=balance)
     B = dw.batch
     harness.prefill(dw, upto_offset=-1)
     seqs = list(range(B))
@@ -127,6 +125,29 @@ def test_forced_variants_and_launch_shapes(variant, Hq, Hkv):
     w = W.Workload("variants", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=6)
     for tuning in ((4, 3, 2), (1, 2, 1), (8, 2, 1), (2, 6, 2), (3, 4, 3)):
         _full_step_check(w, lens=lens, variant=variant, tuning=tuning, check_cache=False)
+
+
+@pytest.mark.parametrize("merge_mode", [0, 1])
+@pytest.mark.parametrize("balance", [(0, 2, 8), (20, 2, 8), (50, 1, 4), (100, 3, 2), (30, 1, 1)])
+def test_merge_modes_and_balance_settings(merge_mode, balance):
+    """Separate merge kernel vs in-kernel merge; static split, pooled tail, everything pooled, tiny chunk budget."""
+    lens = torch.tensor([5000, 33, 1, 256, 1023, 0, 90, 15, 2048], dtype=torch.int32)
+    for Hq, Hkv in ((8, 2), (2, 2)):
+        w = W.Workload("balance", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=31)
+        _full_step_check(w, lens=lens, check_cache=False, merge_mode=merge_mode, balance=balance)
+
+
+def test_repeated_calls_leave_the_workspace_reusable():
+    """The control words return to zero after every launch: many calls on one workspace give one answer."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([3000, 100, 777, 16, 1], dtype=torch.int32)
+    w = W.Workload("repeat", 1, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0,), seed=37)
+    dw = harness.setup(w, lens=lens)
+    harness.prefill(dw, upto_offset=0)
+    first = _decode_layer(dw, 0)[1].clone()
+    for _ in range(20):
+        again = _decode_layer(dw, 0)[1]
+        assert torch.equal(first.view(torch.int16), again.view(torch.int16))
 
 
 def test_page_permutation_does_not_change_outputs():
