@@ -22,7 +22,7 @@ struct skv_cache {
     size_t page_bytes = 0;           // one page of one owner layer
     int sm_count = 0;
     int max_smem_optin = 0;
-    DecodeTuning tune{0, 4, 3, 2, 1, Balance{20, 2, 0}};
+    DecodeTuning tune{0, 8, 2, 1, 1, Balance{0, 2, 0}};
     int chunks_per_worker = 8;       // pool chunk slots per worker (sizes the workspace)
     // the decode workspace whose control words are known to be zero (see prepare_workspace)
     const void *ws_ready = nullptr;
