@@ -59,7 +59,8 @@ typedef enum skv_status {
     SKV_ERR_LAYER = -5,       /* layer index out of range, or an owner is required */
     SKV_ERR_CUDA = -6,        /* a CUDA runtime call failed (no device, bad stream, ...) */
     SKV_ERR_TIMEOUT = -7,     /* device status: a bounded wait inside a kernel ran out */
-    SKV_ERR_BOUNDS = -8       /* device status: a page id or slot id was out of range */
+    SKV_ERR_BOUNDS = -8,      /* device status: a page id or slot id was out of range */
+    SKV_ERR_TOO_LARGE = -9    /* skv_decode_attn_static: the call needs more than SKV_STATIC_SCRATCH_BYTES */
 } skv_status;
 
 const char *skv_strerror(int status);
@@ -175,6 +176,37 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
 int skv_decode_attn(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
                     const int32_t *seq_lens, void *out, int batch, int q_heads, int pt_stride,
                     float scale, void *workspace, size_t workspace_bytes, void *stream);
+
+/* (No counterpart in the paper; an integration convenience.)
+ * skv_decode_attn for callers that cannot hand the library a workspace because
+ * they cannot allocate device memory at the point of the call: code running
+ * inside a serving engine after it has frozen its memory pool (the engine
+ * pre-allocates every byte it will ever use and treats a later cudaMalloc as a
+ * bug, or has none left to give), plugins loaded into a host process that
+ * forbids allocation on its hot path, and callers without an allocator of
+ * their own (a plain C program handed only the input and output buffers).
+ * Same arguments, result and errors as skv_decode_attn minus the workspace:
+ * the split-K partials and control words live in a fixed area of
+ * SKV_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU
+ * that loads the library gives up that much memory until the process exits.
+ *   - Neither this call nor anything it uses allocates or frees device memory.
+ *   - A call whose skv_decode_workspace_bytes(cache, batch, q_heads) exceeds
+ *     SKV_STATIC_SCRATCH_BYTES is refused with SKV_ERR_TOO_LARGE before
+ *     anything is launched (under the default launch shape the need is about
+ *     (SMs * 8 + 2 * batch * kv_heads) * (q_heads / kv_heads) * (head_dim + 2) * 4
+ *     bytes: 3.5 MB for batch 32 of the Llama-3-8B head shape).
+ *   - The first call on each device looks up the area's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device, from every handle and every stream, share the one
+ *     area, and it keeps the previous call's contents: the library clears the
+ *     control words it needs at zero at the start of each call (stream ordered),
+ *     but two calls that overlap on the GPU (different streams without an
+ *     ordering between them) race on it and give undefined results.  Calls on
+ *     one stream are safe. */
+#define SKV_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
+int skv_decode_attn_static(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
+                           const int32_t *seq_lens, void *out, int batch, int q_heads, int pt_stride,
+                           float scale, void *stream);
 
 /* The two kernels separately (profiling, sequence-sharded use): the split-K
  * pass fills `workspace` with partials; the merge kernel turns the partials in

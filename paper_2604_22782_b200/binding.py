@@ -18,6 +18,8 @@ _HEADER = os.path.join(_HERE, "..", "include", "skv.h")
 SKV_OK = 0
 SKV_ERR_ARG, SKV_ERR_ROUTING, SKV_ERR_UNSUPPORTED, SKV_ERR_NOMEM = -1, -2, -3, -4
 SKV_ERR_LAYER, SKV_ERR_CUDA, SKV_ERR_TIMEOUT, SKV_ERR_BOUNDS = -5, -6, -7, -8
+SKV_ERR_TOO_LARGE = -9
+SKV_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 def lib_path() -> str:
@@ -54,6 +56,7 @@ lib.skv_append.argtypes = [_vp, _int, _vp, _vp, _i64p, _i64, _vp]
 lib.skv_gather.argtypes = [_vp, _int, _i64p, _i64, _vp, _vp, _vp]
 lib.skv_decode_workspace_bytes.argtypes = [_vp, _int, _int, _szp]
 lib.skv_decode_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
+lib.skv_decode_attn_static.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp]
 lib.skv_decode_splitk.argtypes = [_vp, _int, _vp, _i32p, _i32p, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_merge.argtypes = [_vp, _vp, _int, _int, _vp, _sz, _vp]
 lib.skv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
@@ -231,6 +234,16 @@ class SkvCache:
                                  q_heads, page_table.shape[1], scale, _ptr(workspace), workspace.numel(),
                                  _stream_ptr(stream))
         _check(rc, "skv_decode_attn")
+
+    def skv_decode_attn_static(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
+                               out: torch.Tensor, scale: float = 0.0, stream=None) -> None:
+        """skv_decode_attn without a workspace argument, for callers that cannot allocate device memory:
+        the scratch is a fixed SKV_STATIC_SCRATCH_BYTES area inside the library (shared by all calls on
+        the device; calls that overlap on the GPU race on it)."""
+        batch, q_heads = Q.shape[0], Q.shape[1]
+        rc = lib.skv_decode_attn_static(self._h, layer, _ptr(Q), _ptr(page_table), _ptr(seq_lens), _ptr(out),
+                                        batch, q_heads, page_table.shape[1], scale, _stream_ptr(stream))
+        _check(rc, "skv_decode_attn_static")
 
     def skv_decode_splitk(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
                           workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:

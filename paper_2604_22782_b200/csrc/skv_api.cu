@@ -149,6 +149,7 @@ const char *skv_strerror(int status)
     case SKV_ERR_CUDA: return "CUDA runtime error";
     case SKV_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case SKV_ERR_BOUNDS: return "page or slot id out of range";
+    case SKV_ERR_TOO_LARGE: return "batch x heads needs more scratch than the library's built-in scratch area holds";
     default: return "unknown status";
     }
 }
@@ -421,6 +422,30 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
     if (rc) return rc;
     return skv_decode_merge(c, out, batch, q_heads, workspace, workspace_bytes, stream);
 }
+
+}  // extern "C"
+
+// Used by skv_decode_attn_static (skv_static.cu): the same launch as skv_decode_attn on a scratch area the
+// library owns.  The area is shared by every handle and keeps whatever the last call left in it, so its
+// control words are cleared on every call instead of being trusted.
+namespace skv {
+int decode_attn_on_scratch(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
+                           void *out, int batch, int q_heads, int pt_stride, float scale, void *scratch,
+                           size_t scratch_bytes, void *stream)
+{
+    if (!out) return SKV_ERR_ARG;
+    if (c) c->ws_ready = nullptr;
+    if (c && c->tune.fused_merge)
+        return launch_splitk(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, scratch,
+                             scratch_bytes, stream);
+    int rc = launch_splitk(c, layer, Q, page_table, seq_lens, nullptr, batch, q_heads, pt_stride, scale, scratch,
+                           scratch_bytes, stream);
+    if (rc) return rc;
+    return skv_decode_merge(c, out, batch, q_heads, scratch, scratch_bytes, stream);
+}
+}  // namespace skv
+
+extern "C" {
 
 int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, const int64_t *slot_map,
                     const int32_t *page_table, const int32_t *seq_lens, void *out, int batch, int q_heads,

@@ -22,8 +22,8 @@ def test_library_loads_and_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_codes():
-    seen = {skv.skv_strerror(c) for c in range(0, -9, -1)}
-    assert len(seen) == 9 and "unknown status" not in seen
+    seen = {skv.skv_strerror(c) for c in range(0, -10, -1)}
+    assert len(seen) == 10 and "unknown status" not in seen
     assert skv.skv_strerror(-99) == "unknown status"
 
 
