@@ -138,10 +138,9 @@ int skv_gather(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t n, 
 /* ---- Algorithm 2 "Load + Attn": decode attention -------------------------- */
 
 /* Bytes of device workspace skv_decode_attn needs for this batch / head count
- * under the CURRENT launch shape and balance settings (ask again after
- * skv_set_decode_tuning / skv_set_decode_balance).  Independent of sequence
- * lengths.  It holds the split partials, a page-count prefix and a few control
- * words. */
+ * under the CURRENT launch shape (ask again after skv_set_decode_tuning).
+ * Independent of sequence lengths.  It holds, twice (two calls of a chain may
+ * overlap), the split partials and a page-count prefix. */
 int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, size_t *out_bytes);
 
 /* Eq. (3.1) for one layer and one new token per sequence:
@@ -155,20 +154,18 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
  *               appended; 0 gives an all-zero output row
  *   out         device bf16 [batch][q_heads][head_dim]
  *   scale       <= 0 selects 1/sqrt(head_dim)
- *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes.  The
- *               library keeps control words in it that are zero between calls:
- *               it clears them whenever it sees a workspace pointer, batch or
- *               head count it did not use in the previous call, so a workspace
- *               may be shared by calls on one stream, but the caller must not
- *               write to it between two calls that pass the same pointer.
- * Work is split over the sequence (flash-decoding): every warp streams an
- * equal share of the (sequence, kv head, page) blocks plus dynamically claimed
- * chunks of a shared tail, and writes fp32 partial (max, sum, output) triples;
- * the partials of a (sequence, kv head) are combined by a log-sum-exp merge,
- * either by the warp that finishes the segment (default, one kernel) or by a
- * separate merge kernel (skv_set_decode_merge_mode).  Slots past seq_lens[b]
- * in the last page contribute nothing whatever they contain.  No host
- * synchronisation; sequence lengths are read on the device.
+ *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes; needs
+ *               no initialisation and may be shared by calls on one stream.
+ * Two launches.  Split-K (flash-decoding): every warp streams an equal share
+ * of the (sequence, kv head, page) blocks and writes, for each (sequence, kv
+ * head) its share touches, an fp32 partial (max, sum, output).  Merge: one warp
+ * per (sequence, kv head) combines its partials by log-sum-exp and writes the
+ * bf16 rows.  Slots past seq_lens[b] in the last page contribute nothing
+ * whatever they contain.  No host synchronisation; sequence lengths are read
+ * on the device.  The split-K launch waits for the work before it in the
+ * stream before it reads anything; with skv_set_decode_overlap on, the merge
+ * kernel is already resident when the split-K launch ends and the kernel after
+ * the call may be scheduled while the call is still running.
  * Errors: SKV_ERR_ARG, SKV_ERR_LAYER, SKV_ERR_UNSUPPORTED (head ratio),
  * SKV_ERR_NOMEM (workspace), SKV_ERR_CUDA.  Device-side problems (page id out
  * of range, a bounded wait that ran out) are reported by skv_get_status; after
@@ -193,24 +190,24 @@ int skv_decode_attn(skv_cache *cache, int layer, const void *Q, const int32_t *p
  *   - A call whose skv_decode_workspace_bytes(cache, batch, q_heads) exceeds
  *     SKV_STATIC_SCRATCH_BYTES is refused with SKV_ERR_TOO_LARGE before
  *     anything is launched (under the default launch shape the need is about
- *     (SMs * 8 + 2 * batch * kv_heads) * (q_heads / kv_heads) * (head_dim + 2) * 4
- *     bytes: 3.5 MB for batch 32 of the Llama-3-8B head shape).
+ *     2 * (SMs * 8 + batch * kv_heads) * (q_heads / kv_heads) * (head_dim + 2) * 4
+ *     bytes: 6.0 MB for batch 32 of the Llama-3-8B head shape).
  *   - The first call on each device looks up the area's device address (with
  *     that device current); make that first call outside any stream capture.
  *   - All calls on a device, from every handle and every stream, share the one
- *     area, and it keeps the previous call's contents: the library clears the
- *     control words it needs at zero at the start of each call (stream ordered),
- *     but two calls that overlap on the GPU (different streams without an
- *     ordering between them) race on it and give undefined results.  Calls on
- *     one stream are safe. */
+ *     area, and it keeps the previous call's contents.  Nothing in it has to
+ *     start at zero (the merge only reads what the split-K launch of the same
+ *     call wrote), so nothing is cleared; but two calls that overlap on the GPU
+ *     (different streams without an ordering between them) race on it and give
+ *     undefined results.  Calls on one stream are safe. */
 #define SKV_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
 int skv_decode_attn_static(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
                            const int32_t *seq_lens, void *out, int batch, int q_heads, int pt_stride,
                            float scale, void *stream);
 
-/* The two kernels separately (profiling, sequence-sharded use): the split-K
- * pass fills `workspace` with partials; the merge kernel turns the partials in
- * `workspace` into `out`.  Same arguments and errors. */
+/* The two launches of skv_decode_attn separately (profiling, sequence-sharded
+ * use): the split-K pass fills `workspace` with partials; the merge kernel
+ * turns the partials in `workspace` into `out`.  Same arguments and errors. */
 int skv_decode_splitk(skv_cache *cache, int layer, const void *Q, const int32_t *page_table,
                       const int32_t *seq_lens, int batch, int q_heads, int pt_stride, float scale,
                       void *workspace, size_t workspace_bytes, void *stream);
@@ -219,6 +216,12 @@ int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *
 
 /* One whole decode step of Algorithm 2 with inputs already on the device:
  * for l = 0..L-1: append (owners only) then decode attention, on `stream`.
+ * Because every input of the step exists when it starts, and the update of
+ * layer l writes only layer l's pages (which no earlier layer reads), the
+ * library issues all owners' updates first, in one launch, and then the L
+ * attention calls as a chain in which the split-K launch of layer l+1 may begin
+ * while layer l is finishing (skv_set_decode_overlap; results are the same as
+ * layer by layer).
  *   Q        device bf16 [n_layers][batch][q_heads][head_dim]
  *   K, V     device bf16 [n_owners][batch][kv_heads][head_dim], owner layers in
  *            increasing layer order
@@ -268,15 +271,23 @@ int skv_set_decode_variant(skv_cache *cache, int variant);
  * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
 int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
 
-/* 1 (default): skv_decode_attn merges inside the split-K kernel (the warp that
- * completes a segment combines its partials); 0: it launches the merge kernel. */
-int skv_set_decode_merge_mode(skv_cache *cache, int fused);
+/* 1 (default): split-K and merge launches carry the programmatic-dependent-
+ * launch attribute, so the GPU may schedule a launch while the one before it
+ * in the stream is still running (each still waits for the work it depends on
+ * before reading it), and skv_decode_step chains its attention calls; 0: plain
+ * launches, and skv_decode_step goes layer by layer through skv_append /
+ * skv_decode_attn. */
+int skv_set_decode_overlap(skv_cache *cache, int enabled);
 
-/* Load balance of the split-K pass: pool_percent (0..100) of the blocks are
- * not assigned up front but claimed in chunks of at least min_chunk_blocks by
- * warps that finish early; chunks_per_worker (1..64) bounds the number of
- * chunks (and the workspace).  pool_percent 0 = fully static split. */
-int skv_set_decode_balance(skv_cache *cache, int pool_percent, int min_chunk_blocks, int chunks_per_worker);
+/* L2 reuse between consecutive layers that read the same owner (the paper's
+ * depth-wise sharing makes them stream identical pages): with keep_percent > 0
+ * such layers walk every worker's block range in alternating directions, and a
+ * layer whose successor reads the same owner loads the last keep_percent % of
+ * each range with normal L2 priority (everything else is loaded evict-first),
+ * so the successor starts on blocks that are still in L2.  0 (default) = every
+ * layer walks forward, everything evict-first.  Results do not depend on it
+ * beyond floating-point summation order. */
+int skv_set_decode_l2_reuse(skv_cache *cache, int keep_percent);
 
 /* Tracing: while a device buffer of at least 32 * skv_decode_worker_count bytes
  * is set, every split-K launch records four uint64 per worker (warp): SM id,

@@ -66,8 +66,8 @@ lib.skv_decode_step_host.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _v
 lib.skv_get_status.argtypes = [_vp, _vp, ctypes.POINTER(_int)]
 lib.skv_set_decode_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
-lib.skv_set_decode_merge_mode.argtypes = [_vp, _int]
-lib.skv_set_decode_balance.argtypes = [_vp, _int, _int, _int]
+lib.skv_set_decode_overlap.argtypes = [_vp, _int]
+lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
 lib.skv_decode_worker_count.argtypes = [_vp]
 lib.skv_launch_count.argtypes = [_vp, ctypes.POINTER(_i64)]
@@ -295,12 +295,11 @@ class SkvCache:
     def skv_set_decode_tuning(self, warps_per_cta: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
         _check(lib.skv_set_decode_tuning(self._h, warps_per_cta, stages, ctas_per_sm), "skv_set_decode_tuning")
 
-    def skv_set_decode_merge_mode(self, fused: int) -> None:
-        _check(lib.skv_set_decode_merge_mode(self._h, fused), "skv_set_decode_merge_mode")
+    def skv_set_decode_overlap(self, enabled: int) -> None:
+        _check(lib.skv_set_decode_overlap(self._h, enabled), "skv_set_decode_overlap")
 
-    def skv_set_decode_balance(self, pool_percent: int, min_chunk_blocks: int = 2, chunks_per_worker: int = 8) -> None:
-        _check(lib.skv_set_decode_balance(self._h, pool_percent, min_chunk_blocks, chunks_per_worker),
-               "skv_set_decode_balance")
+    def skv_set_decode_l2_reuse(self, keep_percent: int) -> None:
+        _check(lib.skv_set_decode_l2_reuse(self._h, keep_percent), "skv_set_decode_l2_reuse")
 
     def skv_set_trace_buffer(self, buf: Optional[torch.Tensor]) -> None:
         _check(lib.skv_set_trace_buffer(self._h, _ptr(buf), 0 if buf is None else buf.numel() * buf.element_size()),

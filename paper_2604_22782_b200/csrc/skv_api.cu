@@ -22,11 +22,10 @@ struct skv_cache {
     size_t page_bytes = 0;           // one page of one owner layer
     int sm_count = 0;
     int max_smem_optin = 0;
-    DecodeTuning tune{0, 8, 2, 1, 1, Balance{0, 2, 0}};
-    int chunks_per_worker = 8;       // pool chunk slots per worker (sizes the workspace)
-    // the decode workspace whose control words are known to be zero (see prepare_workspace)
-    const void *ws_ready = nullptr;
-    int ws_batch = 0, ws_q_heads = 0, ws_workers = 0, ws_chunks = 0;
+    DecodeTuning tune{0, 2, 2, 4, 1};
+    int l2_keep_pct = 0;             // > 0: consecutive layers that read one owner walk it in opposite directions
+    std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
+    std::vector<uint8_t> walk_keep;      // per layer: the next layer reads the same owner
     int64_t launches = 0;
     unsigned long long *trace = nullptr;   // optional per-worker timestamps (device)
     size_t trace_bytes = 0;
@@ -66,57 +65,41 @@ bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The workspace holds two identical buffers so that two consecutive calls of a chain may overlap on the
+// GPU; each buffer is  page-count prefix | partial (max,sum) | partial outputs.  Nothing in it has to be
+// initialised: every slot the merge kernel reads was written by the split-K launch before it.
 struct WorkspaceLayout {
-    size_t ctrl_off, seg_off, prefix_off, ml_off, o_off, total, zero_bytes;
+    size_t prefix_off, ml_off, o_off, buf_bytes, total;
     int64_t n_slots;
 };
 
-// control words | per-segment block counters | page-count prefix | partial (max,sum) | partial outputs
-WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int n_workers, int max_chunks)
+WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int n_workers)
 {
     WorkspaceLayout w;
     const int G = q_heads / c->kv_heads;
     const int64_t n_seg = (int64_t)batch * c->kv_heads;
-    w.n_slots = (int64_t)n_workers + n_seg + (int64_t)max_chunks + n_seg;
-    w.ctrl_off = 0;
-    w.seg_off = 256;
-    w.prefix_off = w.seg_off + round_up((size_t)n_seg * sizeof(int32_t), 256);
-    w.zero_bytes = w.prefix_off;
+    w.n_slots = (int64_t)n_workers + n_seg;          // a run of worker w in segment s writes slot w + s
+    w.prefix_off = 0;
     w.ml_off = w.prefix_off + round_up((size_t)(batch + 1) * sizeof(int32_t), 256);
     w.o_off = w.ml_off + round_up((size_t)w.n_slots * G * 2 * sizeof(float), 256);
-    w.total = w.o_off + round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
+    w.buf_bytes = w.o_off + round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
+    w.total = 2 * w.buf_bytes;
     return w;
 }
 
 int n_workers_of(const skv_cache *c) { return c->sm_count * c->tune.ctas_per_sm * c->tune.warps; }
 
-int max_chunks_of(const skv_cache *c) { return c->tune.bal.pool_pct > 0 ? c->chunks_per_worker * n_workers_of(c) : 0; }
-
-Balance balance_of(const skv_cache *c)
+// Walk directions for L2 reuse: a layer that reads the same owner as the layer before it walks every
+// block range in the opposite direction, so that it starts on the blocks its predecessor read last.
+void plan_walks(skv_cache *c)
 {
-    Balance b = c->tune.bal;
-    b.max_chunks = max_chunks_of(c);
-    return b;
-}
-
-// The split-K kernel expects its control words and per-segment counters to be zero on entry and leaves
-// them zero on exit, so they are cleared only when the workspace (or the layout in it) changes.
-int prepare_workspace(skv_cache *c, void *workspace, const WorkspaceLayout &wl, int batch, int q_heads, cudaStream_t st)
-{
-    const int W = n_workers_of(c), ch = max_chunks_of(c);
-    if (c->ws_ready == workspace && c->ws_batch == batch && c->ws_q_heads == q_heads && c->ws_workers == W &&
-        c->ws_chunks == ch)
-        return SKV_OK;
-    if (cudaMemsetAsync(workspace, 0, wl.zero_bytes, st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return SKV_ERR_CUDA;
+    const size_t L = (size_t)c->n_layers;
+    c->walk_reverse.assign(L, 0);
+    c->walk_keep.assign(L, 0);
+    for (size_t l = 0; l < L; ++l) {
+        if (l > 0 && c->r[l] == c->r[l - 1]) c->walk_reverse[l] = !c->walk_reverse[l - 1];
+        if (l + 1 < L && c->r[l + 1] == c->r[l]) c->walk_keep[l] = 1;
     }
-    c->ws_ready = workspace;
-    c->ws_batch = batch;
-    c->ws_q_heads = q_heads;
-    c->ws_workers = W;
-    c->ws_chunks = ch;
-    return SKV_OK;
 }
 
 int check_decode_args(const skv_cache *c, int layer, int batch, int q_heads)
@@ -222,6 +205,7 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
         }
     c->n_owners = (int)c->owners.size();
     c->page_bytes = page_bytes_of(kv_heads, head_dim);
+    plan_walks(c);
     c->pool = static_cast<uint8_t *>(device_pool);
     c->pool_bytes = device_pool ? need : 0;
     if (device_pool) {
@@ -282,10 +266,11 @@ int skv_append(skv_cache *c, int layer, const void *K, const void *V, const int6
     p.n_tokens = n_tokens;
     p.n_slots = c->max_pages * PAGE;
     p.page_stride = (int64_t)c->page_bytes;
+    p.layer_stride = 0;
     p.Hkv = c->kv_heads;
     p.D = c->head_dim;
     p.status = c->status_word();
-    if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+    if (launch_append(p, 1, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
     c->launches += 1;
     return SKV_OK;
 }
@@ -319,31 +304,30 @@ int skv_decode_workspace_bytes(const skv_cache *c, int batch, int q_heads, size_
     if (q_heads % c->kv_heads != 0 || q_heads / c->kv_heads > 8) return SKV_ERR_UNSUPPORTED;
     const int sm = c->sm_count > 0 ? c->sm_count : 148;
     const int W = sm * c->tune.ctas_per_sm * c->tune.warps;
-    const int ch = c->tune.bal.pool_pct > 0 ? c->chunks_per_worker * W : 0;
-    *out_bytes = workspace_layout(c, batch, q_heads, W, ch).total;
+    *out_bytes = workspace_layout(c, batch, q_heads, W).total;
     return SKV_OK;
 }
 
 namespace {
-// launches the split-K kernel; `out` non-null selects the fused (in-kernel) merge
+// Launches the split-K kernel on buffer `buf` (0 or 1) of the workspace.  `chained` = the call follows
+// another attention call of the same step whose inputs were all ready before that call was launched, so
+// it need not wait for it before reading.
 int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
-                  void *out, int batch, int q_heads, int pt_stride, float scale, void *workspace,
-                  size_t workspace_bytes, void *stream)
+                  int batch, int q_heads, int pt_stride, float scale, void *workspace, size_t workspace_bytes,
+                  void *stream, int buf = 0, bool chained = false)
 {
     int rc = check_decode_args(c, layer, batch, q_heads);
     if (rc) return rc;
     if (!Q || !page_table || !seq_lens || !workspace || pt_stride <= 0) return SKV_ERR_ARG;
-    if (!aligned(Q, 16) || !aligned(workspace, 256) || (out && !aligned(out, 8))) return SKV_ERR_ARG;
+    if (!aligned(Q, 16) || !aligned(workspace, 256)) return SKV_ERR_ARG;
     const int G = q_heads / c->kv_heads;
     const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W, max_chunks_of(c));
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
     const size_t smem = decode_smem_bytes(c->head_dim, batch, c->tune.warps, c->tune.stages);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = prepare_workspace(c, workspace, wl, batch, q_heads, st);
-    if (rc) return rc;
-    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
     DecodeParams p;
     p.layer_base = c->layer_base(c->slot[(size_t)c->r[(size_t)layer]]);
     p.page_stride = (int64_t)c->page_bytes;
@@ -354,22 +338,29 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.part_o = reinterpret_cast<float *>(ws + wl.o_off);
     p.part_ml = reinterpret_cast<float *>(ws + wl.ml_off);
     p.prefix = reinterpret_cast<int32_t *>(ws + wl.prefix_off);
-    p.ctrl = reinterpret_cast<int32_t *>(ws + wl.ctrl_off);
-    p.seg_count = reinterpret_cast<int32_t *>(ws + wl.seg_off);
-    p.out = static_cast<uint16_t *>(out);
     p.B = batch;
     p.Hq = q_heads;
     p.Hkv = c->kv_heads;
     p.pt_stride = pt_stride;
     const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)c->head_dim);
     p.scale_log2 = sc * 1.4426950408889634f;
-    p.bal = balance_of(c);
+    p.flags = chained ? DECODE_LATE_WAIT : 0;
+    p.keep_pct = 0;
+    if (c->l2_keep_pct > 0) {
+        if (c->walk_reverse[(size_t)layer]) p.flags |= DECODE_REVERSE;
+        if (c->walk_keep[(size_t)layer]) p.keep_pct = c->l2_keep_pct;
+    }
     p.status = c->status_word();
     p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
     const bool tensor_core = c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
     const int grid = c->sm_count * c->tune.ctas_per_sm;
-    if (launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, c->tune.warps, c->tune.stages, st) != cudaSuccess)
-        return SKV_ERR_CUDA;
+    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, c->tune.warps, c->tune.stages,
+                                                c->tune.pdl != 0, st);
+    if (le != cudaSuccess) {
+        (void)cudaGetLastError();
+        // a launch shape with more warps per CTA than the register file holds for this kernel variant
+        return le == cudaErrorLaunchOutOfResources ? SKV_ERR_UNSUPPORTED : SKV_ERR_CUDA;
+    }
     c->launches += 1;
     return SKV_OK;
 }
@@ -379,20 +370,22 @@ int skv_decode_splitk(skv_cache *c, int layer, const void *Q, const int32_t *pag
                       int batch, int q_heads, int pt_stride, float scale, void *workspace,
                       size_t workspace_bytes, void *stream)
 {
-    return launch_splitk(c, layer, Q, page_table, seq_lens, nullptr, batch, q_heads, pt_stride, scale, workspace,
+    return launch_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
                          workspace_bytes, stream);
 }
 
-int skv_decode_merge(skv_cache *c, void *out, int batch, int q_heads, void *workspace, size_t workspace_bytes,
-                     void *stream)
+namespace {
+// the merge kernel on buffer `buf` of the workspace
+int launch_merge_on(skv_cache *c, void *out, int batch, int q_heads, void *workspace, size_t workspace_bytes,
+                    void *stream, int buf)
 {
     int rc = check_decode_args(c, 0, batch, q_heads);
     if (rc) return rc;
     if (!out || !workspace || !aligned(out, 8) || !aligned(workspace, 256)) return SKV_ERR_ARG;
     const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W, max_chunks_of(c));
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
-    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
     MergeParams m;
     m.part_o = reinterpret_cast<const float *>(ws + wl.o_off);
     m.part_ml = reinterpret_cast<const float *>(ws + wl.ml_off);
@@ -403,10 +396,19 @@ int skv_decode_merge(skv_cache *c, void *out, int batch, int q_heads, void *work
     m.Hkv = c->kv_heads;
     m.D = c->head_dim;
     m.n_workers = W;
-    m.bal = balance_of(c);
-    if (launch_merge(m, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+    if (launch_merge(m, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SKV_ERR_CUDA;
+    }
     c->launches += 1;
     return SKV_OK;
+}
+}  // namespace
+
+int skv_decode_merge(skv_cache *c, void *out, int batch, int q_heads, void *workspace, size_t workspace_bytes,
+                     void *stream)
+{
+    return launch_merge_on(c, out, batch, q_heads, workspace, workspace_bytes, stream, 0);
 }
 
 int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
@@ -414,34 +416,24 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
                     size_t workspace_bytes, void *stream)
 {
     if (!out) return SKV_ERR_ARG;
-    if (c && c->tune.fused_merge)
-        return launch_splitk(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, workspace,
-                             workspace_bytes, stream);
-    int rc = skv_decode_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
-                               workspace_bytes, stream);
+    int rc = launch_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
+                           workspace_bytes, stream);
     if (rc) return rc;
-    return skv_decode_merge(c, out, batch, q_heads, workspace, workspace_bytes, stream);
+    return launch_merge_on(c, out, batch, q_heads, workspace, workspace_bytes, stream, 0);
 }
 
 }  // extern "C"
 
-// Used by skv_decode_attn_static (skv_static.cu): the same launch as skv_decode_attn on a scratch area the
-// library owns.  The area is shared by every handle and keeps whatever the last call left in it, so its
-// control words are cleared on every call instead of being trusted.
+// Used by skv_decode_attn_static (skv_static.cu): the same two launches as skv_decode_attn on a scratch
+// area the library owns.  Nothing in the area has to be cleared: the merge kernel only reads slots that
+// the split-K launch of the same call has just written.
 namespace skv {
 int decode_attn_on_scratch(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
                            void *out, int batch, int q_heads, int pt_stride, float scale, void *scratch,
                            size_t scratch_bytes, void *stream)
 {
-    if (!out) return SKV_ERR_ARG;
-    if (c) c->ws_ready = nullptr;
-    if (c && c->tune.fused_merge)
-        return launch_splitk(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, scratch,
-                             scratch_bytes, stream);
-    int rc = launch_splitk(c, layer, Q, page_table, seq_lens, nullptr, batch, q_heads, pt_stride, scale, scratch,
+    return skv_decode_attn(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, scratch,
                            scratch_bytes, stream);
-    if (rc) return rc;
-    return skv_decode_merge(c, out, batch, q_heads, scratch, scratch_bytes, stream);
 }
 }  // namespace skv
 
@@ -459,14 +451,50 @@ int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, c
     const uint8_t *q = static_cast<const uint8_t *>(Q), *k = static_cast<const uint8_t *>(K),
                   *v = static_cast<const uint8_t *>(V);
     uint8_t *o = static_cast<uint8_t *>(out);
-    for (int l = 0; l < c->n_layers; ++l) {
-        const int os = c->slot[(size_t)l];
-        if (os >= 0) {
-            rc = skv_append(c, l, k + (size_t)os * kv_layer, v + (size_t)os * kv_layer, slot_map, batch, stream);
+    if (!c->tune.pdl) {
+        // layer by layer, exactly as a caller of the per-layer entry points would
+        for (int l = 0; l < c->n_layers; ++l) {
+            const int os = c->slot[(size_t)l];
+            if (os >= 0) {
+                rc = skv_append(c, l, k + (size_t)os * kv_layer, v + (size_t)os * kv_layer, slot_map, batch, stream);
+                if (rc) return rc;
+            }
+            rc = skv_decode_attn(c, l, q + (size_t)l * q_layer, page_table, seq_lens, o + (size_t)l * q_layer, batch,
+                                 q_heads, pt_stride, scale, workspace, workspace_bytes, stream);
             if (rc) return rc;
         }
-        rc = skv_decode_attn(c, l, q + (size_t)l * q_layer, page_table, seq_lens, o + (size_t)l * q_layer, batch,
-                             q_heads, pt_stride, scale, workspace, workspace_bytes, stream);
+        return SKV_OK;
+    }
+    // All inputs of the step exist before it starts, and the update of layer l touches only layer l's
+    // pages, which no layer before l reads: so every owner's update goes first, in one launch, and the
+    // attention calls form a chain in which the split-K launch of layer l+1 may start while that of layer l
+    // is finishing and its merge is running (they work on alternate workspace buffers; a split-K launch
+    // waits for everything before it half-way through its own work, which also keeps the launch of layer
+    // l+2 from starting before layer l has been merged).
+    if (!aligned(K, 16) || !aligned(V, 16)) return SKV_ERR_ARG;
+    AppendParams ap;
+    ap.layer_base = c->layer_base(0);
+    ap.K = reinterpret_cast<const uint4 *>(k);
+    ap.V = reinterpret_cast<const uint4 *>(v);
+    ap.slot_map = slot_map;
+    ap.n_tokens = batch;
+    ap.n_slots = c->max_pages * PAGE;
+    ap.page_stride = (int64_t)c->page_bytes;
+    ap.layer_stride = (int64_t)c->max_pages * (int64_t)c->page_bytes;
+    ap.Hkv = c->kv_heads;
+    ap.D = c->head_dim;
+    ap.status = c->status_word();
+    if (launch_append(ap, c->n_owners, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SKV_ERR_CUDA;
+    }
+    c->launches += 1;
+    for (int l = 0; l < c->n_layers; ++l) {
+        rc = launch_splitk(c, l, q + (size_t)l * q_layer, page_table, seq_lens, batch, q_heads, pt_stride, scale,
+                           workspace, workspace_bytes, stream, l & 1, l > 0);
+        if (rc) return rc;
+        // the merge kernel waits for that launch and lets the next split-K launch be scheduled at once
+        rc = launch_merge_on(c, o + (size_t)l * q_layer, batch, q_heads, workspace, workspace_bytes, stream, l & 1);
         if (rc) return rc;
     }
     return SKV_OK;
@@ -559,7 +587,6 @@ int skv_get_status(skv_cache *c, void *stream, int *device_status)
         return SKV_ERR_CUDA;
     }
     *device_status = (word & STATUS_TIMEOUT) ? SKV_ERR_TIMEOUT : (word & STATUS_BOUNDS) ? SKV_ERR_BOUNDS : SKV_OK;
-    if (word & STATUS_TIMEOUT) c->ws_ready = nullptr;     // a worker gave up: counters may be left non-zero
     return SKV_OK;
 }
 
@@ -577,7 +604,7 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     if (warps_per_cta) t.warps = warps_per_cta;
     if (stages) t.stages = stages;
     if (ctas_per_sm) t.ctas_per_sm = ctas_per_sm;
-    if (t.warps < 1 || t.warps > 16 || t.stages < 2 || t.stages > 8 || t.ctas_per_sm < 1 || t.ctas_per_sm > 8)
+    if (t.warps < 1 || t.warps > 16 || t.stages < 1 || t.stages > 8 || t.ctas_per_sm < 1 || t.ctas_per_sm > 16)
         return SKV_ERR_ARG;
     if (c->pool) {
         const size_t smem = decode_smem_bytes(c->head_dim, 1, t.warps, t.stages);
@@ -587,21 +614,17 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     return SKV_OK;
 }
 
-int skv_set_decode_merge_mode(skv_cache *c, int fused)
+int skv_set_decode_overlap(skv_cache *c, int enabled)
 {
-    if (!c || fused < 0 || fused > 1) return SKV_ERR_ARG;
-    c->tune.fused_merge = fused;
+    if (!c || enabled < 0 || enabled > 1) return SKV_ERR_ARG;
+    c->tune.pdl = enabled;
     return SKV_OK;
 }
 
-int skv_set_decode_balance(skv_cache *c, int pool_percent, int min_chunk_blocks, int chunks_per_worker)
+int skv_set_decode_l2_reuse(skv_cache *c, int keep_percent)
 {
-    if (!c || pool_percent < 0 || pool_percent > 100 || min_chunk_blocks < 1 || chunks_per_worker < 1 ||
-        chunks_per_worker > 64)
-        return SKV_ERR_ARG;
-    c->tune.bal.pool_pct = pool_percent;
-    c->tune.bal.min_chunk = min_chunk_blocks;
-    c->chunks_per_worker = chunks_per_worker;
+    if (!c || keep_percent < 0 || keep_percent > 100) return SKV_ERR_ARG;
+    c->l2_keep_pct = keep_percent;
     return SKV_OK;
 }
 

@@ -8,7 +8,8 @@ namespace {
 
 constexpr int COPY_THREADS = 256;
 
-// One thread moves one 16-byte chunk (8 bf16 of one head of one token).
+// One thread moves one 16-byte chunk (8 bf16 of one head of one token); grid.y picks K or V,
+// grid.z the owner layer when one launch serves several.
 // Reads are fully coalesced along the token row; writes land 16 bytes apart at
 // a stride of PAGE*16 bytes (the chunk-major page layout).
 __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
@@ -29,8 +30,9 @@ __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
     const int64_t page = slot / PAGE;
     const int off = (int)(slot - page * PAGE);
     const int which = blockIdx.y;                       // 0 = K, 1 = V
-    const uint4 *src = which ? p.V : p.K;
-    uint8_t *dst = p.layer_base + page * p.page_stride + (int64_t)h * block_bytes(p.D) +
+    const int64_t layer = blockIdx.z;                   // owner layers of one launch, consecutive in the pool
+    const uint4 *src = (which ? p.V : p.K) + layer * p.n_tokens * row_chunks;
+    uint8_t *dst = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * block_bytes(p.D) +
                    (int64_t)which * half_bytes(p.D) + ((int64_t)c * PAGE + off) * 16;
     *reinterpret_cast<uint4 *>(dst) = __ldg(src + idx);
 }
@@ -61,13 +63,15 @@ __global__ void __launch_bounds__(COPY_THREADS) gather_kernel(GatherParams p)
 
 }  // namespace
 
-cudaError_t launch_append(const AppendParams &p, cudaStream_t s)
+// n_layers consecutive owner layers (grid.z) take rows from K/V [n_layers][n_tokens][Hkv][D] with one slot map
+cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s)
 {
     const int64_t chunks = p.n_tokens * p.Hkv * (p.D / CHUNK_ELEMS);
     const int64_t blocks = (chunks + COPY_THREADS - 1) / COPY_THREADS;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
-    append_kernel<<<dim3((unsigned)blocks, 2), COPY_THREADS, 0, s>>>(p);
+    if (n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
+    append_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), COPY_THREADS, 0, s>>>(p);
     return cudaGetLastError();
 }
 

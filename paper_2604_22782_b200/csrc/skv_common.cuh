@@ -27,13 +27,14 @@ constexpr int STATUS_TIMEOUT = 1;
 constexpr int STATUS_BOUNDS = 2;
 
 struct AppendParams {
-    uint8_t *layer_base;        // first page of this owner layer
-    const uint4 *K;             // [n_tokens][Hkv][D] bf16 viewed as 16-byte chunks
+    uint8_t *layer_base;        // first page of the (first) owner layer written
+    const uint4 *K;             // [n_layers_here][n_tokens][Hkv][D] bf16 viewed as 16-byte chunks
     const uint4 *V;
-    const int64_t *slot_map;
+    const int64_t *slot_map;    // [n_tokens], shared by all layers of the launch
     int64_t n_tokens;
     int64_t n_slots;            // max_pages * PAGE
     int64_t page_stride;        // bytes between pages of one layer
+    int64_t layer_stride;       // bytes between consecutive owner layers in the pool (grid.z walks them)
     int Hkv, D;
     int *status;
 };
@@ -50,34 +51,10 @@ struct GatherParams {
     int *status;
 };
 
-// How one decode call's blocks are handed to the W workers (warps).  The
-// flattened block list [0, T) is cut in two: [0, Ts) is split statically into
-// W equal contiguous ranges; the tail [Ts, T) (the "pool") is cut into chunks
-// of `chunk` blocks that workers claim one at a time from an atomic counter
-// once their static range is done, so that faster SMs take more of the work.
-struct Plan {
-    int64_t T, Ts;
-    int chunk, n_chunks;
-};
-
-struct Balance {
-    int pool_pct;       // share of the blocks that goes to the pool (0 = fully static)
-    int min_chunk;      // smallest pool chunk, in blocks
-    int max_chunks;     // upper bound on the number of pool chunks (sizes the workspace)
-};
-
-__host__ __device__ inline Plan make_plan(int64_t T, const Balance &b)
-{
-    Plan pl;
-    pl.T = T;
-    int64_t pool = b.max_chunks > 0 ? (T * b.pool_pct) / 100 : 0;
-    int64_t c = b.min_chunk > 0 ? b.min_chunk : 1;
-    if (pool > c * b.max_chunks) c = (pool + b.max_chunks - 1) / b.max_chunks;
-    pl.chunk = (int)c;
-    pl.n_chunks = (int)((pool + c - 1) / c);
-    pl.Ts = T - pool;
-    return pl;
-}
+// DecodeParams::flags
+constexpr int DECODE_REVERSE = 1;     // every worker walks its block range from the last block to the first
+constexpr int DECODE_LATE_WAIT = 2;   // inputs are known to be ready: the wait on the previous kernel in the
+                                      // stream is taken half-way through the range instead of before the first read
 
 struct DecodeParams {
     const uint8_t *layer_base;  // first page of the owner layer that is read
@@ -88,13 +65,12 @@ struct DecodeParams {
     const int32_t *seq_lens;    // [B]
     float *part_o;              // [n_slots][G][D]
     float *part_ml;             // [n_slots][G][2]  (running max in log2 units, sum)
-    int32_t *prefix;            // [B+1] cumulative page counts (written by CTA 0)
-    int32_t *ctrl;              // [0] pool claim counter, [1] exited-worker counter (both 0 between launches)
-    int32_t *seg_count;         // [B*Hkv] blocks finished per segment (0 between launches); fused merge only
-    uint16_t *out;              // [B][Hq][D] bf16 bits: non-null = merge inside this kernel (last arriver)
+    int32_t *prefix;            // [B+1] cumulative page counts (written by CTA 0 for the merge kernel)
     int B, Hq, Hkv, pt_stride;
     float scale_log2;           // scale * log2(e)
-    Balance bal;
+    int flags;
+    int keep_pct;               // share of each worker's range, at the END of its walk, that is loaded with
+                                // normal L2 priority; the rest is loaded evict-first
     int *status;
     unsigned long long *trace;  // optional [n_workers][4]: sm id, entry ns, first-page ns, exit ns
 };
@@ -106,7 +82,6 @@ struct MergeParams {
     uint16_t *out;              // [B][Hq][D] bf16 bits
     int B, Hq, Hkv, D;
     int n_workers;
-    Balance bal;
 };
 
 struct DecodeTuning {
@@ -114,18 +89,17 @@ struct DecodeTuning {
     int warps;                  // per CTA
     int stages;                 // per warp
     int ctas_per_sm;
-    int fused_merge;            // 1: the split-K kernel's last arriver per segment merges
-    Balance bal;
+    int pdl;                    // 1: launches carry the programmatic-dependent-launch attribute
 };
 
 // host launchers (each returns a cudaError_t from the launch)
-cudaError_t launch_append(const AppendParams &p, cudaStream_t s);
+cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s);
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
 // smem bytes the split-K kernel needs for this shape, or 0 if unsupported
 size_t decode_smem_bytes(int D, int B, int warps, int stages);
 cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid,
-                                 int warps, int stages, cudaStream_t s);
-cudaError_t launch_merge(const MergeParams &p, cudaStream_t s);
+                                 int warps, int stages, bool pdl, cudaStream_t s);
+cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 
 // ---- worker <-> work-range arithmetic (shared by split-K and merge) --------
 // The flattened work space orders (sequence b, kv head h, page pg) b-major:
@@ -199,6 +173,35 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
         : "memory");
 }
+
+// same, with an L2 eviction-priority policy (from make_policy_*)
+__device__ __forceinline__ void bulk_copy_g2s_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                                   uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ uint64_t make_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ uint64_t make_policy_evict_normal()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// Programmatic dependent launch: wait for the kernel before this one in the stream (a no-op when the
+// launch carried no such attribute); let the kernel after this one start being scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void fence_barrier_init()
 {

@@ -7,10 +7,12 @@
 // per WARP (W = grid * warps per CTA).  A warp streams its blocks through a
 // private shared-memory ring filled by linear bulk copies (one 2*PAGE*D*2-byte
 // copy per block, completion on an mbarrier), keeps a running (max, sum, out)
-// per query head of the kv head's group, and writes one fp32 partial per
-// (sequence, kv head) segment its range touches, to slot  worker + segment.
-// Every warp does the same number of blocks (+-1) whatever the length mix, so
-// there is no tail; warps never synchronise with each other after the prologue.
+// per query head of the kv head's group, and at the end of every run inside a
+// (sequence, kv head) segment writes one fp32 partial to slot  worker + segment.
+// Every warp does the same number of blocks (+-1) whatever the length mix;
+// warps never synchronise with each other after the prologue.  The merge
+// kernel (one warp per segment) combines a segment's partials; it is launched
+// so that it is already resident, waiting, when the split-K kernel ends.
 #include "skv_common.cuh"
 
 #include <math.h>
@@ -20,6 +22,7 @@ namespace skv {
 namespace {
 
 constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr int WIN = 128;   // page ids a warp keeps in registers (4 per lane)
 
 struct Cursor {        // a position in the flattened (b, h, page) list
     int b, h, pg, pages;
@@ -41,21 +44,34 @@ __device__ __forceinline__ Cursor locate(const int32_t *prefix, int B, int Hkv, 
     return c;
 }
 
-// Only called while another position remains, so b never runs past B-1.
-__device__ __forceinline__ void advance(Cursor &c, const int32_t *prefix, int Hkv)
+// One position forward (or backward).  Only called while another position remains in that
+// direction, so b stays inside [0, B).
+__device__ __forceinline__ void step(Cursor &c, const int32_t *prefix, int Hkv, bool reverse)
 {
-    if (++c.pg < c.pages) return;
-    c.pg = 0;
-    if (++c.h < Hkv) return;
-    c.h = 0;
-    do {
-        ++c.b;
-        c.pages = prefix[c.b + 1] - prefix[c.b];
-    } while (c.pages == 0);
+    if (!reverse) {
+        if (++c.pg < c.pages) return;
+        c.pg = 0;
+        if (++c.h < Hkv) return;
+        c.h = 0;
+        do {
+            ++c.b;
+            c.pages = prefix[c.b + 1] - prefix[c.b];
+        } while (c.pages == 0);
+    } else {
+        if (--c.pg >= 0) return;
+        if (--c.h < 0) {
+            c.h = Hkv - 1;
+            do {
+                --c.b;
+                c.pages = prefix[c.b + 1] - prefix[c.b];
+            } while (c.pages == 0);
+        }
+        c.pg = c.pages - 1;
+    }
 }
 
-// Shared-memory carve-up (dynamic): prefix[B+1] | rings | barriers
-__host__ __device__ inline size_t prefix_bytes(int B) { return (((size_t)(B + 1) * 4) + 127) & ~(size_t)127; }
+// Shared-memory carve-up (dynamic): prefix[B+1] | lens[B] | rings | barriers | CTA arrival word
+__host__ __device__ inline size_t table_bytes(int B) { return (((size_t)(2 * B + 1) * 4) + 127) & ~(size_t)127; }
 
 // ---------------------------------------------------------------------------
 // Per-warp compute state, tensor-core variant: the G query heads of one kv head
@@ -142,6 +158,7 @@ struct TensorCoreState {
         }
     }
 
+    // the run's partial (max, sum, unnormalised out) of every query head of the group -> slot
     __device__ __forceinline__ void finish(const DecodeParams &p, int64_t slot, int G, int lane)
     {
         const int g = lane >> 2, tig = lane & 3;
@@ -154,13 +171,14 @@ struct TensorCoreState {
             if (tig == 0) *reinterpret_cast<float2 *>(p.part_ml + (slot * G + g) * 2) = make_float2(m, l);
         }
     }
+
 };
 
 // ---------------------------------------------------------------------------
 // CUDA-core variant for one query head per kv head (MHA): a GEMV per page, so
 // no tensor cores.  Lane = (token slot t = lane&15, dim half = lane>>4); every
 // lane runs its own online softmax over the tokens that fall in its slot and
-// the 16 slots are combined once per segment.
+// the 16 slots are combined once per run.
 // ---------------------------------------------------------------------------
 template <int D>
 struct CudaCoreState {
@@ -231,14 +249,14 @@ struct CudaCoreState {
         }
     }
 
-    __device__ __forceinline__ void finish(const DecodeParams &p, int64_t slot, int /*G*/, int lane)
+    // combine the 16 token slots: afterwards lanes with t == 0 hold the run's sum in o[], and (M, lt) everywhere
+    __device__ __forceinline__ void reduce(float &M, float &lt, int lane)
     {
-        const int t = lane & 15, hf = lane >> 4;
-        float M = m;
+        M = m;
 #pragma unroll
         for (int d = 1; d < 16; d <<= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, d));
         const float wgt = (m == -INFINITY) ? 0.f : fast_exp2(m - M);
-        float lt = l * wgt;
+        lt = l * wgt;
 #pragma unroll
         for (int d = 1; d < 16; d <<= 1) lt += __shfl_xor_sync(FULL, lt, d);
 #pragma unroll
@@ -248,6 +266,13 @@ struct CudaCoreState {
             for (int d = 1; d < 16; d <<= 1) x += __shfl_xor_sync(FULL, x, d);
             o[i] = x;
         }
+    }
+
+    __device__ __forceinline__ void finish(const DecodeParams &p, int64_t slot, int /*G*/, int lane)
+    {
+        const int t = lane & 15, hf = lane >> 4;
+        float M, lt;
+        reduce(M, lt, lane);
         if (t == 0) {
             float *po = p.part_o + slot * D + hf * (D / 2);
 #pragma unroll
@@ -256,110 +281,111 @@ struct CudaCoreState {
             if (hf == 0) *reinterpret_cast<float2 *>(p.part_ml + slot * 2) = make_float2(M, lt);
         }
     }
+
 };
 
 // ---------------------------------------------------------------------------
-// Where the partials of one segment (sequence b, kv head kvh) live.  A static
-// range that meets the segment wrote slot  worker + seg;  a pool chunk that
-// meets it wrote slot  W + n_seg + chunk + seg.  Lane k of the calling warp
-// gets the k-th partial's slot (or -1); returns how many there are.  A segment
-// with more than 32 partials is walked in rounds of 32 (`round`).
+// Where the partials of a segment live.  The segment's blocks are [s0, s0 + pages) of the flattened
+// list.  Normally worker w writes the partial of its run inside segment seg to slot  w + seg, so a
+// segment's partials sit in consecutive slots.  When there are fewer blocks than workers every
+// non-empty range is a single block x, and its partial goes to slot  x + seg  (consecutive again).
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ int partial_slots(const Plan &pl, int64_t W, int64_t n_seg, int64_t s0, int pages,
-                                             int64_t seg, int lane, int round, int64_t &slot)
+__device__ __forceinline__ int partial_slot(int64_t T, int64_t W, int64_t w, int64_t x_any, int64_t seg)
 {
-    const int64_t s1 = s0 + pages;
-    int n_static = 0;
-    int64_t w_first = 0;
-    const bool sparse = pl.Ts < W;            // then every non-empty static range is a single block
-    if (s0 < pl.Ts) {
-        const int64_t e = s1 < pl.Ts ? s1 : pl.Ts;
-        if (sparse) {
-            n_static = (int)(e - s0);
-        } else {
-            w_first = worker_of(s0, pl.Ts, W);
-            n_static = worker_of(e - 1, pl.Ts, W) - (int)w_first + 1;
-        }
-    }
-    int n_pool = 0;
-    int64_t j_first = 0;
-    if (s1 > pl.Ts && pl.n_chunks > 0) {
-        const int64_t a = s0 > pl.Ts ? s0 : pl.Ts;
-        j_first = (a - pl.Ts) / pl.chunk;
-        n_pool = (int)((s1 - 1 - pl.Ts) / pl.chunk - j_first) + 1;
-    }
-    const int k = round * 32 + lane;
-    slot = -1;
-    if (k < n_static) slot = (sparse ? (int64_t)worker_of(s0 + k, pl.Ts, W) : w_first + k) + seg;
-    else if (k < n_static + n_pool) slot = W + n_seg + j_first + (k - n_static) + seg;
-    return n_static + n_pool;
+    return (int)((T < W ? x_any : w) + seg);
 }
 
-// Log-sum-exp merge of one segment's partials for its G query heads, by one warp:
-// out[b, kvh*G+g, :] = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i,  M = max_i m_i.
-template <int D>
-__device__ __noinline__ void merge_segment(const float *part_o, const float *part_ml, uint16_t *out,
-                                              const Plan &pl, int64_t W, int B, int Hq, int Hkv, int b, int kvh,
-                                              int64_t s0, int pages, int lane)
+__device__ __forceinline__ void segment_partials(int64_t T, int64_t W, int64_t seg, int64_t s0, int pages, int &slot0,
+                                                 int &n)
 {
-    constexpr int PER = D / 32;               // consecutive output dims per lane
-    const int G = Hq / Hkv;
-    const int64_t seg = (int64_t)b * Hkv + kvh, n_seg = (int64_t)B * Hkv;
-    int64_t slot;
-    const int n = partial_slots(pl, W, n_seg, s0, pages, seg, lane, 0, slot);
-    for (int g = 0; g < G; ++g) {
-        float acc[PER];
+    if (T < W) {
+        slot0 = (int)(s0 + seg);
+        n = pages;
+    } else {
+        const int w_first = worker_of(s0, T, W);
+        slot0 = (int)(w_first + seg);
+        n = worker_of(s0 + pages - 1, T, W) - w_first + 1;
+    }
+}
+
+// Log-sum-exp merge of the n partials at slots slot0 .. slot0+n-1 for the G query heads of a
+// segment, by one warp:
+//   out[g, :] = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i,  M = max_i m_i.
+// With G rounded up to a power of two G', the G'*D outputs are dealt to the 32 lanes in contiguous
+// pieces of E2 = G'*D/64 float2 (a piece lies inside one head's row); NB partials are fetched
+// together so that a typical segment costs one round trip to L2.
+template <int D, int E2MAX, int NB>
+__device__ __forceinline__ void merge_rows(const float *part_o, const float *part_ml, uint16_t *out_seg, int G,
+                                           int slot0, int n, int lane)
+{
+    const int Gp = G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8;   // rows dealt out (lanes of rows >= G idle)
+    const int E2 = Gp * D / 64;               // float2 per lane (<= E2MAX)
+    const int e0 = lane * 2 * E2, g = e0 / D, d0 = e0 - g * D;
+    if (g >= G) return;                       // no warp-wide operation below
+    float2 acc[E2MAX];
 #pragma unroll
-        for (int i = 0; i < PER; ++i) acc[i] = 0.f;
-        float M = -INFINITY, L = 0.f;
-        for (int r = 0; r * 32 < n; ++r) {
-            int64_t my = slot;
-            if (r > 0) partial_slots(pl, W, n_seg, s0, pages, seg, lane, r, my);
-            // this round's (max, sum) pairs, one partial per lane
-            float2 ml = make_float2(-INFINITY, 0.f);
-            if (my >= 0) ml = __ldcg(reinterpret_cast<const float2 *>(part_ml + (my * G + g) * 2));
-            float Mr = ml.x;
+    for (int e = 0; e < E2MAX; ++e) acc[e] = make_float2(0.f, 0.f);
+    float M = -INFINITY, L = 0.f;
+    const unsigned row = (unsigned)G * D;     // floats per partial
+    const float2 *po = reinterpret_cast<const float2 *>(part_o + (size_t)slot0 * row + g * D + d0);
+    const float2 *pm = reinterpret_cast<const float2 *>(part_ml + ((size_t)slot0 * G + g) * 2);
+    for (int j0 = 0; j0 < n; j0 += NB) {
+        float2 ml[NB];
+        float2 v[NB][E2MAX];
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) Mr = fmaxf(Mr, __shfl_xor_sync(FULL, Mr, d));
-            const float M_new = fmaxf(M, Mr);
-            const float keep = exp2f(M - M_new);          // 0 on the first round
-            const float wt = (my >= 0) ? exp2f(ml.x - M_new) : 0.f;
-            float Lr = wt * ml.y;
+        for (int u = 0; u < NB; ++u) {
+            ml[u] = make_float2(-INFINITY, 0.f);
+            if (j0 + u < n) {
+                ml[u] = __ldcg(pm + (j0 + u) * G);
+                const float2 *src = po + (size_t)(j0 + u) * (row / 2);
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) Lr += __shfl_xor_sync(FULL, Lr, d);
-            L = L * keep + Lr;
-            M = M_new;
-#pragma unroll
-            for (int i = 0; i < PER; ++i) acc[i] *= keep;
-            const int cnt = (n - r * 32) < 32 ? (n - r * 32) : 32;
-            for (int i0 = 0; i0 < cnt; i0 += 4) {
-                float v[4][PER], wv[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = (i0 + u) < cnt ? (i0 + u) : i0;       // clamp: weight 0 below
-                    const int64_t sl = __shfl_sync(FULL, my, i);
-                    wv[u] = (i0 + u) < cnt ? __shfl_sync(FULL, wt, i) : 0.f;
-                    const float *po = part_o + (sl * G + g) * D + lane * PER;
-                    if constexpr (PER == 4) {
-                        const float4 t = __ldcg(reinterpret_cast<const float4 *>(po));
-                        v[u][0] = t.x; v[u][1] = t.y; v[u][2] = t.z; v[u][3] = t.w;
-                    } else {
-                        const float2 t = __ldcg(reinterpret_cast<const float2 *>(po));
-                        v[u][0] = t.x; v[u][1] = t.y;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-#pragma unroll
-                    for (int i = 0; i < PER; ++i) acc[i] = fmaf(wv[u], v[u][i], acc[i]);
+                for (int e = 0; e < E2MAX; ++e)
+                    if (e < E2) v[u][e] = __ldcg(src + e);
             }
         }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        uint16_t *dst = out + ((int64_t)b * Hq + (int64_t)kvh * G + g) * D + lane * PER;
+        float Mb = ml[0].x;
 #pragma unroll
-        for (int i = 0; i < PER; i += 2)
-            *reinterpret_cast<uint32_t *>(dst + i) = pack_bf16x2(acc[i] * inv, acc[i + 1] * inv);
+        for (int u = 1; u < NB; ++u) Mb = fmaxf(Mb, ml[u].x);
+        const float M_new = fmaxf(M, Mb);            // finite: a partial holds at least one token
+        const float keep = fast_exp2(M - M_new);     // 0 for the first batch
+        L *= keep;
+#pragma unroll
+        for (int e = 0; e < E2MAX; ++e) { acc[e].x *= keep; acc[e].y *= keep; }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            if (j0 + u < n) {
+                const float wt = fast_exp2(ml[u].x - M_new);
+                L = fmaf(wt, ml[u].y, L);
+#pragma unroll
+                for (int e = 0; e < E2MAX; ++e)
+                    if (e < E2) {
+                        acc[e].x = fmaf(wt, v[u][e].x, acc[e].x);
+                        acc[e].y = fmaf(wt, v[u][e].y, acc[e].y);
+                    }
+            }
+        }
+        M = M_new;
     }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    uint32_t *dst = reinterpret_cast<uint32_t *>(out_seg + g * D + d0);
+#pragma unroll
+    for (int e = 0; e < E2MAX; ++e)
+        if (e < E2) dst[e] = pack_bf16x2(acc[e].x * inv, acc[e].y * inv);
+}
+
+template <int D>
+__device__ __forceinline__ void merge_segment(const float *part_o, const float *part_ml, uint16_t *out_seg, int G,
+                                              int slot0, int n, int lane)
+{
+    const int E2 = (G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8) * D / 64;
+#ifndef SKV_MERGE_PAYLOAD
+#define SKV_MERGE_PAYLOAD 64                  // float2 in flight per lane while merging
+#endif
+    constexpr int P = SKV_MERGE_PAYLOAD;
+    if (E2 <= 2) merge_rows<D, 2, (P / 2 > 16 ? 16 : P / 2)>(part_o, part_ml, out_seg, G, slot0, n, lane);
+    else if (E2 <= 4) merge_rows<D, 4, (P / 4 > 16 ? 16 : P / 4)>(part_o, part_ml, out_seg, G, slot0, n, lane);
+    else if (E2 <= 8) merge_rows<D, 8, P / 8>(part_o, part_ml, out_seg, G, slot0, n, lane);
+    else merge_rows<D, 16, P / 16>(part_o, part_ml, out_seg, G, slot0, n, lane);
 }
 
 // ---------------------------------------------------------------------------
@@ -368,35 +394,41 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = block_bytes(D);
-    constexpr int QLEN = 8;                   // per-warp queue of range ids between producer and consumer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint64_t t_entry = p.trace ? global_timer_ns() : 0;
     uint64_t t_first = 0;
 
-    // carve shared memory: prefix | rings | barriers | range queues  (ring base rounded up to 128 bytes)
+    // carve shared memory: tables | rings | barriers | arrival word  (ring base rounded up to 128 bytes)
     const uint32_t base = smem_u32(smem_raw);
     const uint32_t pad = (128u - (base & 127u)) & 127u;
     int32_t *prefix = reinterpret_cast<int32_t *>(smem_raw + pad);
-    const size_t rings_off = pad + prefix_bytes(p.B);
-    const uint32_t rings = base + (uint32_t)rings_off;
-    const uint32_t ring = rings + (uint32_t)(warp * stages * BLOCK);
+    int32_t *lens = prefix + p.B + 1;
+    const size_t rings_off = pad + table_bytes(p.B);
+    const uint32_t ring = base + (uint32_t)rings_off + (uint32_t)(warp * stages * BLOCK);
     const size_t bars_off = rings_off + (size_t)nwarps * stages * BLOCK;
     const uint32_t bars = base + (uint32_t)bars_off + (uint32_t)(warp * stages * 8);
-    int32_t *queue = reinterpret_cast<int32_t *>(smem_raw + bars_off + (size_t)nwarps * stages * 8) + warp * QLEN;
+    int *arrivals = reinterpret_cast<int *>(smem_raw + bars_off + (size_t)nwarps * stages * 8);
 
     if (lane == 0) {
         for (int s = 0; s < stages; ++s) mbar_init(bars + 8 * s, 1);
         fence_barrier_init();
     }
-    // cumulative page counts of the batch (warp 0), visible to every warp after the barrier
+    if (threadIdx.x == 0) *arrivals = 0;
+    const bool late_wait = (p.flags & DECODE_LATE_WAIT) != 0;
+    const bool reverse = (p.flags & DECODE_REVERSE) != 0;
+    if (!late_wait) pdl_wait();            // anything read below may come from the kernel before this one
+
+    // sequence lengths and cumulative page counts of the batch (warp 0), visible to all after the barrier
     if (warp == 0) {
         int carry = 0;
         for (int i0 = 0; i0 < p.B; i0 += 32) {
             const int i = i0 + lane;
-            int v = 0;
+            int n = 0, v = 0;
             if (i < p.B) {
-                const int n = __ldg(p.seq_lens + i);
-                v = n > 0 ? (n + PAGE - 1) / PAGE : 0;
+                n = __ldg(p.seq_lens + i);
+                n = n > 0 ? n : 0;
+                v = (n + PAGE - 1) / PAGE;
+                lens[i] = n;
             }
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -409,71 +441,53 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
         if (lane == 0) prefix[0] = 0;
     }
     __syncthreads();
-    if (blockIdx.x == 0) {
+    if (blockIdx.x == 0)       // the merge kernel reads the page counts from global memory
         for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.prefix[i] = prefix[i];
-        if (p.out) {     // fused merge: rows of empty sequences are zero and belong to nobody else
-            const int row_words = p.Hq * D / 2;
-            for (int b = 0; b < p.B; ++b)
-                if (prefix[b + 1] == prefix[b])
-                    for (int i = threadIdx.x; i < row_words; i += blockDim.x)
-                        reinterpret_cast<uint32_t *>(p.out)[(int64_t)b * row_words + i] = 0u;
-        }
-    }
 
     const int64_t W = (int64_t)gridDim.x * nwarps, w = (int64_t)blockIdx.x * nwarps + warp;
-    const int64_t n_seg = (int64_t)p.B * p.Hkv;
-    const Plan pl = make_plan((int64_t)prefix[p.B] * p.Hkv, p.bal);
-    if (pl.T == 0) return;
-    const bool pooled = pl.n_chunks > 0;
+    const int64_t T = (int64_t)prefix[p.B] * p.Hkv;
+    int64_t x0 = 0;
+    int n = 0;
+    if (T > 0) {
+        x0 = worker_begin(w, T, W);
+        n = (int)(worker_begin(w + 1, T, W) - x0);
+    }
+    const int64_t x_first = reverse ? x0 + n - 1 : x0;
 
-    // static range of this worker
-    const int64_t x0 = worker_begin(w, pl.Ts, W);
-    const int n_static = (int)(worker_begin(w + 1, pl.Ts, W) - x0);
-    // first pool claim, requested now and looked at only when the static range has been issued
-    int next_j = 0;
-    if (pooled && lane == 0) next_j = atomicAdd(p.ctrl, 1);
+    // Half-way point of this worker: (in a chain of calls) wait for the kernel before this one, then let the
+    // one after it be scheduled once every warp of the CTA has got here.
+    bool synced = false;
+    auto pdl_sync = [&]() {
+        synced = true;
+        if (late_wait) pdl_wait();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = (atomicAdd(arrivals, 1) == nwarps - 1);
+        if (__shfl_sync(FULL, last, 0)) pdl_trigger();
+    };
 
-    // ---- producer: walks ranges (static, then claimed chunks) and keeps the ring full ----
-    Cursor prod = {0, 0, 0, 0};
-    int prod_left = 0, q_tail = 0, in_flight = 0, p_stage = 0;
-    bool static_given = false, prod_done = false;
-    int win_b = -1, win_base = 0, win_ids = 0;   // page ids of the current sequence, 32 at a time, one per lane
+    // ---- producer: keeps the ring full ----
+    const uint64_t pol_stream = make_policy_evict_first(), pol_keep = make_policy_evict_normal();
+    const int keep_from = n - (int)(((int64_t)n * p.keep_pct) / 100);
+    Cursor prod = {0, 0, 0, 1};
+    if (n > 0) prod = locate(prefix, p.B, p.Hkv, x_first);
+    int prod_left = n, issued = 0, in_flight = 0, p_stage = 0;
+    int win_b = -1, win_base = 0, ids0 = 0, ids1 = 0, ids2 = 0, ids3 = 0;   // page ids: 4 per lane
     auto issue = [&]() -> bool {
-        if (prod_done) return false;
-        if (prod_left == 0) {
-            int id = -1, cnt = 0;
-            int64_t begin = 0;
-            if (!static_given) {
-                static_given = true;
-                begin = x0;
-                cnt = n_static;
-            }
-            if (cnt == 0 && pooled) {
-                const int j = __shfl_sync(FULL, next_j, 0);
-                if (j < pl.n_chunks) {
-                    if (lane == 0) next_j = atomicAdd(p.ctrl, 1);
-                    id = j;
-                    begin = pl.Ts + (int64_t)j * pl.chunk;
-                    const int64_t rest = pl.T - begin;
-                    cnt = rest < pl.chunk ? (int)rest : pl.chunk;
-                }
-            }
-            if (cnt == 0) {
-                prod_done = true;
-                return false;
-            }
-            if (lane == 0) queue[q_tail & (QLEN - 1)] = id;
-            ++q_tail;
-            prod = locate(prefix, p.B, p.Hkv, begin);
-            prod_left = cnt;
-        }
-        if (prod.b != win_b || prod.pg < win_base || prod.pg >= win_base + 32) {
+        if (prod_left == 0) return false;
+        if (prod.b != win_b || prod.pg < win_base || prod.pg >= win_base + WIN) {
             win_b = prod.b;
-            win_base = prod.pg;
-            const int i = prod.pg + lane;
-            win_ids = (i < prod.pages) ? __ldg(p.page_table + (int64_t)prod.b * p.pt_stride + i) : 0;
+            win_base = reverse ? (prod.pg >= WIN ? prod.pg - (WIN - 1) : 0) : prod.pg;
+            const int32_t *row = p.page_table + (int64_t)prod.b * p.pt_stride + win_base + lane;
+            const int left = prod.pages - win_base - lane;
+            ids0 = left > 0 ? __ldg(row) : 0;
+            ids1 = left > 32 ? __ldg(row + 32) : 0;
+            ids2 = left > 64 ? __ldg(row + 64) : 0;
+            ids3 = left > 96 ? __ldg(row + 96) : 0;
         }
-        int id = __shfl_sync(FULL, win_ids, prod.pg - win_base);
+        const int rel = prod.pg - win_base, sel = rel >> 5;
+        const int mine = sel == 0 ? ids0 : sel == 1 ? ids1 : sel == 2 ? ids2 : ids3;
+        int id = __shfl_sync(FULL, mine, rel & 31);
         if (lane == 0) {
             if (id < 0 || (int64_t)id >= p.max_pages) {
                 atomicOr(p.status, STATUS_BOUNDS);
@@ -482,103 +496,62 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
             const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)prod.h * BLOCK;
             const uint32_t bar = bars + 8 * p_stage;
             mbar_expect_tx(bar, BLOCK);
-            bulk_copy_g2s(ring + (uint32_t)(p_stage * BLOCK), src, BLOCK, bar);
+            bulk_copy_g2s_hint(ring + (uint32_t)(p_stage * BLOCK), src, BLOCK, bar,
+                               issued >= keep_from ? pol_keep : pol_stream);
         }
         if (++p_stage == stages) p_stage = 0;
         ++in_flight;
-        if (--prod_left > 0) advance(prod, prefix, p.Hkv);
+        ++issued;
+        if (--prod_left > 0) step(prod, prefix, p.Hkv, reverse);
         return true;
     };
-    // the queue holds at most `stages`+1 ranges: a range is queued only when one of its blocks is issued
     while (in_flight < stages && issue()) {}
 
-    // ---- consumer ----
-    State st;
-    Cursor cons = {0, 0, 0, 0};
-    int cons_left = 0, q_head = 0, c_stage = 0, run_pages = 0, n_b = 0;
-    int64_t slot_base = 0;
+    // ---- consumer: one iteration of the outer loop per run inside a (sequence, kv head) segment ----
+    Cursor cons = {0, 0, 0, 1};
+    if (n > 0) cons = locate(prefix, p.B, p.Hkv, x_first);
+    int consumed = 0, c_stage = 0;
+    const int half = n / 2;
     uint32_t parity = 0;
-    bool fresh = true, first = true, failed = false;
-    while (in_flight > 0) {
-        if (cons_left == 0) {
-            __syncwarp();
-            const int id = queue[q_head & (QLEN - 1)];
-            ++q_head;
-            int64_t begin;
-            if (id < 0) {
-                begin = x0;
-                cons_left = n_static;
-                slot_base = w;
-            } else {
-                begin = pl.Ts + (int64_t)id * pl.chunk;
-                const int64_t rest = pl.T - begin;
-                cons_left = rest < pl.chunk ? (int)rest : pl.chunk;
-                slot_base = W + n_seg + id;
-            }
-            cons = locate(prefix, p.B, p.Hkv, begin);
-            fresh = true;
-        }
-        if (fresh) {
-            st.begin(p, cons.b, cons.h, G, lane);
-            n_b = __ldg(p.seq_lens + cons.b);
-            run_pages = 0;
-            fresh = false;
-        }
-        const bool ok = mbar_wait_bounded(bars + 8 * c_stage, parity);
-        if (!__all_sync(FULL, ok)) {
-            // give up: flag it, let the copies still in flight land (bounded), leave
-            if (lane == 0) atomicOr(p.status, STATUS_TIMEOUT);
-            int s = c_stage;
-            uint32_t par = parity;
-            for (int k = 1; k < in_flight; ++k) {
-                if (++s == stages) { s = 0; par ^= 1u; }
-                mbar_wait_bounded(bars + 8 * s, par);
-            }
-            failed = true;
-            break;
-        }
-        if (p.trace && first) t_first = global_timer_ns();
-        first = false;
-        const uint32_t sK = ring + (uint32_t)(c_stage * BLOCK);
-        const int left = n_b - cons.pg * PAGE;
-        st.page(sK, sK + half_bytes(D), left < PAGE ? left : PAGE, p.scale_log2, lane);
-        __syncwarp();                       // every lane is done reading this stage
-        --in_flight;
-        issue();                            // refill it
-        if (++c_stage == stages) { c_stage = 0; parity ^= 1u; }
-        ++run_pages;
-        --cons_left;
-        if (cons.pg + 1 == cons.pages || cons_left == 0) {
-            // this worker's run inside segment (b, h) ends: publish the partial
-            const int64_t seg = (int64_t)cons.b * p.Hkv + cons.h;
-            st.finish(p, slot_base + seg, G, lane);
-            if (p.out) {
-                // the worker that completes the segment's block count merges it
-                __threadfence();
-                __syncwarp();
-                int done = 0;
-                if (lane == 0) done = atomicAdd(p.seg_count + seg, run_pages) + run_pages;
-                done = __shfl_sync(FULL, done, 0);
-                if (done == cons.pages) {
-                    __threadfence();
-                    const int64_t s0 = (int64_t)prefix[cons.b] * p.Hkv + (int64_t)cons.h * cons.pages;
-                    merge_segment<D>(p.part_o, p.part_ml, p.out, pl, W, p.B, p.Hq, p.Hkv, cons.b, cons.h, s0,
-                                     cons.pages, lane);
-                    if (lane == 0) p.seg_count[seg] = 0;
+    bool failed = false;
+    while (consumed < n && !failed) {
+        const int b = cons.b, h = cons.h, pages = cons.pages, n_b = lens[cons.b];
+        const int64_t seg = (int64_t)b * p.Hkv + h;
+        {
+            State st;                          // lives for this run only
+            st.begin(p, b, h, G, lane);
+            for (;;) {
+                if (!synced && consumed >= half) pdl_sync();
+                const bool ok = mbar_wait_bounded(bars + 8 * c_stage, parity);
+                if (!__all_sync(FULL, ok)) {
+                    // give up: flag it, let the copies still in flight land (bounded), leave
+                    if (lane == 0) atomicOr(p.status, STATUS_TIMEOUT);
+                    int s = c_stage;
+                    uint32_t par = parity;
+                    for (int k = 1; k < in_flight; ++k) {
+                        if (++s == stages) { s = 0; par ^= 1u; }
+                        mbar_wait_bounded(bars + 8 * s, par);
+                    }
+                    failed = true;
+                    break;
                 }
+                if (p.trace && consumed == 0) t_first = global_timer_ns();
+                const uint32_t sK = ring + (uint32_t)(c_stage * BLOCK);
+                const int left = n_b - cons.pg * PAGE;
+                st.page(sK, sK + half_bytes(D), left < PAGE ? left : PAGE, p.scale_log2, lane);
+                __syncwarp();                       // every lane is done reading this stage
+                --in_flight;
+                issue();                            // refill it
+                if (++c_stage == stages) { c_stage = 0; parity ^= 1u; }
+                ++consumed;
+                const bool run_ends = (reverse ? (cons.pg == 0) : (cons.pg + 1 == pages)) || consumed == n;
+                if (consumed < n) step(cons, prefix, p.Hkv, reverse);
+                if (run_ends) break;
             }
-            fresh = true;
-        }
-        if (cons_left > 0) advance(cons, prefix, p.Hkv);
-    }
-    (void)failed;
-    // the last worker to leave puts the two counters back to zero for the next launch
-    if (pooled && lane == 0) {
-        if (atomicAdd(p.ctrl + 1, 1) == (int)W - 1) {
-            p.ctrl[0] = 0;
-            p.ctrl[1] = 0;
+            if (!failed) st.finish(p, partial_slot(T, W, w, x0, seg), G, lane);
         }
     }
+    if (!synced) pdl_sync();
     if (p.trace && lane == 0) {
         unsigned smid;
         asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
@@ -590,11 +563,15 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
 // ---------------------------------------------------------------------------
 // Stand-alone merge kernel: one warp per (sequence, kv head) segment.
 // ---------------------------------------------------------------------------
+constexpr int MERGE_WARPS = 2;
+
 template <int D>
-__global__ void __launch_bounds__(128) merge_kernel(MergeParams p)
+__global__ void __launch_bounds__(MERGE_WARPS * 32) merge_kernel(MergeParams p)
 {
+    pdl_trigger();        // nothing after this kernel in the stream needs to wait for its start
+    pdl_wait();           // the partials come from the kernel before this one
     const int lane = threadIdx.x & 31;
-    const int64_t seg = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int64_t seg = (int64_t)blockIdx.x * MERGE_WARPS + (threadIdx.x >> 5);
     if (seg >= (int64_t)p.B * p.Hkv) return;
     const int b = (int)(seg / p.Hkv), kvh = (int)(seg - (int64_t)b * p.Hkv);
     const int pages = p.prefix[b + 1] - p.prefix[b];
@@ -604,20 +581,31 @@ __global__ void __launch_bounds__(128) merge_kernel(MergeParams p)
         for (int i = lane; i < G * D / 2; i += 32) dst[i] = 0u;
         return;
     }
-    const Plan pl = make_plan((int64_t)p.prefix[p.B] * p.Hkv, p.bal);
+    const int64_t T = (int64_t)p.prefix[p.B] * p.Hkv;
     const int64_t s0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)kvh * pages;
-    merge_segment<D>(p.part_o, p.part_ml, p.out, pl, p.n_workers, p.B, p.Hq, p.Hkv, b, kvh, s0, pages, lane);
+    int slot0, n_part;
+    segment_partials(T, p.n_workers, seg, s0, pages, slot0, n_part);
+    merge_segment<D>(p.part_o, p.part_ml, p.out + ((int64_t)b * p.Hq + (int64_t)kvh * G) * D, G, slot0, n_part, lane);
 }
 
 template <int D, class State>
-cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, int stages, cudaStream_t s)
+cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, int stages, bool pdl, cudaStream_t s)
 {
     const size_t smem = decode_smem_bytes(D, p.B, warps, stages);
     auto kern = decode_splitk_kernel<D, State>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, warps * 32, smem, s>>>(p, G, stages);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)(warps * 32));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, p, G, stages);
 }
 
 }  // namespace
@@ -625,33 +613,39 @@ cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, i
 size_t decode_smem_bytes(int D, int B, int warps, int stages)
 {
     if (D != 64 && D != 128) return 0;
-    // 128 bytes of slack for aligning the ring base; 8 queue entries per warp
-    return 128 + prefix_bytes(B) + (size_t)warps * stages * block_bytes(D) + (size_t)warps * stages * 8 +
-           (size_t)warps * 8 * 4;
+    // 128 bytes of slack for aligning the ring base; 16 bytes for the arrival word
+    return 128 + table_bytes(B) + (size_t)warps * stages * block_bytes(D) + (size_t)warps * stages * 8 + 16;
 }
 
 cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid, int warps,
-                                 int stages, cudaStream_t s)
+                                 int stages, bool pdl, cudaStream_t s)
 {
     if (D == 128) {
-        if (tensor_core) return launch_splitk_t<128, TensorCoreState<128>>(p, G, grid, warps, stages, s);
-        return launch_splitk_t<128, CudaCoreState<128>>(p, G, grid, warps, stages, s);
+        if (tensor_core) return launch_splitk_t<128, TensorCoreState<128>>(p, G, grid, warps, stages, pdl, s);
+        return launch_splitk_t<128, CudaCoreState<128>>(p, G, grid, warps, stages, pdl, s);
     }
     if (D == 64) {
-        if (tensor_core) return launch_splitk_t<64, TensorCoreState<64>>(p, G, grid, warps, stages, s);
-        return launch_splitk_t<64, CudaCoreState<64>>(p, G, grid, warps, stages, s);
+        if (tensor_core) return launch_splitk_t<64, TensorCoreState<64>>(p, G, grid, warps, stages, pdl, s);
+        return launch_splitk_t<64, CudaCoreState<64>>(p, G, grid, warps, stages, pdl, s);
     }
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_merge(const MergeParams &p, cudaStream_t s)
+cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s)
 {
     const int64_t segs = (int64_t)p.B * p.Hkv;
-    const unsigned blocks = (unsigned)((segs + 3) / 4);
-    if (p.D == 128) merge_kernel<128><<<blocks, 128, 0, s>>>(p);
-    else if (p.D == 64) merge_kernel<64><<<blocks, 128, 0, s>>>(p);
-    else return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((segs + MERGE_WARPS - 1) / MERGE_WARPS));
+    cfg.blockDim = dim3(MERGE_WARPS * 32);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    if (p.D == 128) return cudaLaunchKernelEx(&cfg, merge_kernel<128>, p);
+    if (p.D == 64) return cudaLaunchKernelEx(&cfg, merge_kernel<64>, p);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace skv

@@ -37,16 +37,16 @@ class DeviceWorkload:
     def owners(self) -> List[int]:
         return [l for l in range(self.w.n_layers) if self.r[l] == l]
 
-    def retune(self, variant=None, tuning=None, merge_mode=None, balance=None) -> None:
-        """Change kernel variant / launch shape / merge mode / balance, then size the workspace again."""
+    def retune(self, variant=None, tuning=None, overlap=None, l2_keep=None) -> None:
+        """Change kernel variant / launch shape / overlap / L2 reuse, then size the workspace again."""
         if variant is not None:
             self.cache.skv_set_decode_variant(variant)
         if tuning is not None:
             self.cache.skv_set_decode_tuning(*tuning)
-        if merge_mode is not None:
-            self.cache.skv_set_decode_merge_mode(merge_mode)
-        if balance is not None:
-            self.cache.skv_set_decode_balance(*balance)
+        if overlap is not None:
+            self.cache.skv_set_decode_overlap(overlap)
+        if l2_keep is not None:
+            self.cache.skv_set_decode_l2_reuse(l2_keep)
         need = self.cache.skv_decode_workspace_bytes(self.batch, self.w.q_heads)
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)

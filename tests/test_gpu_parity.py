@@ -51,13 +51,13 @@ def _decode_layer(dw, layer, Q=None, scale=0.0):
 
 
 def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True,
-                     merge_mode=None, balance=None):
+                     overlap=None, l2_keep=None):
     """One decode step of every layer: prefill n-1 tokens, append the last one, attend; compare all."""
     harness, dw = _make(w, lens=lens, r=r, permute=permute)
     if poison:   # every byte of the page area becomes a bf16 NaN pattern (0x7FC1)
         dw.pool_view = dw.cache.pool[256:].view(torch.int16)
         dw.pool_view.fill_(0x7FC1)
-    dw.retune(variant=variant or None, tuning=tuning, merge_mode=merge_mode, balance=balance)
+    dw.retune(variant=variant or None, tuning=tuning, overlap=overlap, l2_keep=l2_keep)
     B = dw.batch
     harness.prefill(dw, upto_offset=-1)
     seqs = list(range(B))
@@ -123,18 +123,61 @@ def test_forced_variants_and_launch_shapes(variant, Hq, Hkv):
     """Tensor-core kernel on MHA, CUDA-core kernel, and other warps/stages/CTAs-per-SM settings."""
     lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15], dtype=torch.int32)
     w = W.Workload("variants", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=6)
-    for tuning in ((4, 3, 2), (1, 2, 1), (8, 2, 1), (2, 6, 2), (3, 4, 3)):
+    for tuning in ((4, 3, 2), (1, 2, 1), (8, 2, 1), (2, 6, 2), (3, 4, 3), (2, 2, 4), (1, 1, 8), (8, 1, 1)):
         _full_step_check(w, lens=lens, variant=variant, tuning=tuning, check_cache=False)
 
 
-@pytest.mark.parametrize("merge_mode", [0, 1])
-@pytest.mark.parametrize("balance", [(0, 2, 8), (20, 2, 8), (50, 1, 4), (100, 3, 2), (30, 1, 1)])
-def test_merge_modes_and_balance_settings(merge_mode, balance):
-    """Separate merge kernel vs in-kernel merge; static split, pooled tail, everything pooled, tiny chunk budget."""
+@pytest.mark.parametrize("overlap,l2_keep", [(1, 0), (0, 0), (1, 30), (0, 100), (1, 1)])
+def test_overlap_and_walk_directions(overlap, l2_keep):
+    """Plain vs overlappable launches; forward-only walks vs alternating directions with part of each
+    range kept in L2 (layers 0,1,2 read owner 0, layer 3 owns)."""
     lens = torch.tensor([5000, 33, 1, 256, 1023, 0, 90, 15, 2048], dtype=torch.int32)
     for Hq, Hkv in ((8, 2), (2, 2)):
-        w = W.Workload("balance", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=31)
-        _full_step_check(w, lens=lens, check_cache=False, merge_mode=merge_mode, balance=balance)
+        w = W.Workload("walks", 4, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 0, 3), seed=31)
+        _full_step_check(w, lens=lens, check_cache=False, overlap=overlap, l2_keep=l2_keep)
+
+
+@pytest.mark.parametrize("overlap,l2_keep", [(1, 0), (1, 40), (0, 0)])
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (4, 2, 64)])
+def test_whole_step_entry_points_match_the_oracle(overlap, l2_keep, Hq, Hkv, D):
+    """skv_decode_step (all updates first, then the chained attention launches) and skv_decode_step_host
+    against the oracle for every layer, and against each other bit for bit, repeated to reuse both
+    workspace buffers."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 0, 15, 3000, 16, 17], dtype=torch.int32)
+    w = W.Workload("step", 5, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2, 2, 2), seed=43)
+    dw = harness.setup(w, lens=lens)
+    dw.retune(overlap=overlap, l2_keep=l2_keep)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    o = _oracle_for(dw, list(range(dw.batch)), range(w.n_layers))
+    refs = [o.decode_attn(l, t["Q"][l].cpu(), dw.lens_cpu) for l in range(w.n_layers)]
+    for rep in range(3):
+        t["out"].fill_(float("nan"))
+        dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"],
+                                 dw.workspace)
+        torch.cuda.synchronize()
+        assert dw.cache.skv_get_status() == 0
+        for l in range(w.n_layers):
+            ok, err = _within_tol(t["out"][l], refs[l])
+            assert ok, f"rep {rep} layer {l}: max abs err {err}"
+    hb = harness.step_tensors(dw, device="cpu", pin=True)
+    staging = torch.empty(dw.cache.skv_decode_step_staging_bytes(dw.batch, w.q_heads, dw.page_table_cpu.shape[1]),
+                          dtype=torch.uint8, device=dw.device)
+    dw.cache.skv_decode_step_host(hb["Q"], hb["K"], hb["V"], dw.slot_new.cpu().pin_memory(),
+                                  dw.page_table_cpu.contiguous().pin_memory(), dw.lens_cpu.contiguous().pin_memory(),
+                                  hb["out"], staging)
+    torch.cuda.synchronize()
+    assert torch.equal(hb["out"].view(torch.int16), t["out"].cpu().view(torch.int16))
+    # the updates really happened: the newest token of every owner layer reads back bit-exactly
+    has = dw.slot_new >= 0
+    for i, l in enumerate(dw.owners):
+        Kg = torch.zeros_like(t["K"][i])
+        Vg = torch.zeros_like(Kg)
+        dw.cache.skv_gather(l, dw.slot_new, Kg, Vg)
+        torch.cuda.synchronize()
+        assert torch.equal(Kg[has].view(torch.int16), t["K"][i][has].view(torch.int16))
+        assert torch.equal(Vg[has].view(torch.int16), t["V"][i][has].view(torch.int16))
 
 
 def test_repeated_calls_leave_the_workspace_reusable():
