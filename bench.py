@@ -37,7 +37,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel,
 # from the ncu capture summarised under profiles/ (None until captured)
-NCU_TRAFFIC_BYTES = {"llama3_8b": None}
+NCU_TRAFFIC_BYTES = {"llama3_8b": 343290000}
+DEFAULT_L2_KEEP = 35     # the library's default share of each block range kept in L2 for the next layer
 
 
 def _peaks():
@@ -149,6 +150,29 @@ def run_reference(args, w):
     }))
 
 
+def rank_workload(w, rank: int, world: int):
+    """Weak scaling: every rank holds its own batch of the same shape (rank-specific seed), no exchange."""
+    if world <= 1:
+        return w
+    import dataclasses
+    return dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of a list of floats over all ranks (identity for one rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_rate(units_per_rank_per_step: float, steps: int, ms_max_over_ranks: float, world: int) -> float:
+    """Units all ranks processed divided by the slowest rank's time (units per second)."""
+    return world * units_per_rank_per_step * steps / (ms_max_over_ranks * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -178,10 +202,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     from paper_2604_22782_b200 import harness
-    # weak scaling: every rank holds its own batch of the same shape (rank-specific seed), no exchange
-    if world > 1:
-        import dataclasses
-        w = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+    w = rank_workload(w, rank, world)
     dw = harness.setup(w, device=dev)
     dw.retune(variant=args.variant or None,
               tuning=[int(x) for x in args.tuning.split(",")] if args.tuning else None,
@@ -190,7 +211,8 @@ def main():
     harness.prefill(dw, upto_offset=-1)
     t = harness.step_tensors(dw)
     L, n_own = w.n_layers, len(dw.owners)
-    step_bytes = L * dw.kv_bytes_per_call() + n_own * dw.append_bytes_per_call()
+    attn_bytes = dw.kv_bytes_per_call()
+    step_bytes = L * attn_bytes + n_own * dw.append_bytes_per_call()
     cache = dw.cache
 
     def step():
@@ -202,25 +224,40 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = cache.skv_launch_count()
-    with ClockSampler(local) as clocks:
+    def timed_steps(fn):
+        """args.warmup untimed calls, then args.steps calls between two events (barrier + synchronize on
+        both sides); returns milliseconds for the args.steps calls."""
+        for _ in range(args.warmup):
+            fn()
         barrier()
-        ev0.record()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         for _ in range(args.steps):
-            step()
-        ev1.record()
+            fn()
+        e1.record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        launches = cache.skv_launch_count() - launches0
+        return e0.elapsed_time(e1)
 
-        # the dominant kernel alone: the same layers through the per-layer entry points, an event pair
-        # around every attention launch (events between launches also keep them from overlapping)
+    with ClockSampler(local) as clocks:
+        # (1) the headline: whole decode steps, inputs resident in HBM, library defaults
+        launches0 = cache.skv_launch_count()
+        ms = timed_steps(step)
+        launches = (cache.skv_launch_count() - launches0) * args.steps // (args.steps + args.warmup)
+        out_default = t["out"].clone()
+
+        # (2) the roofline leg: the same steps with L2 reuse between layers switched off, so that every
+        # attention launch streams all of its pages from HBM.  The split-K kernel's average launch
+        # duration is taken as (time of the timed region) / (split-K launches in it): its launches
+        # overlap each other and the small merge and update kernels, so they cannot be bracketed one
+        # by one without changing what is measured; the quotient charges those kernels to it.
+        dw.retune(l2_keep=0)
+        ms_hbm = timed_steps(step)
+        dw.retune(l2_keep=args.l2_keep if args.l2_keep >= 0 else DEFAULT_L2_KEEP)
+
+        # (3) one attention call at a time (no overlap between calls): per-layer entry points with an
+        # event pair around every skv_decode_attn (split-K + merge)
         pairs = []
-        for _ in range(args.steps):
+        for _ in range(max(2, args.steps // 4)):
             for l in range(L):
                 if dw.r[l] == l:
                     cache.skv_append(l, t["K"][dw.owners.index(l)], t["V"][dw.owners.index(l)], dw.slot_new)
@@ -230,14 +267,13 @@ def main():
                 b.record()
                 pairs.append((l, a, b))
         torch.cuda.synchronize(dev)
-        per = [(l, a.elapsed_time(b)) for l, a, b in pairs]
-        kern_ms = sum(x for _, x in per) / len(per)
+        per = [(l, a.elapsed_time(b)) for l, a, b in pairs[L:]]
         own = [x for l, x in per if dw.r[l] == l]
         non = [x for l, x in per if dw.r[l] != l]
-        kern_ms_owner = sum(own) / len(own)
-        kern_ms_reader = sum(non) / len(non) if non else None
+        call_ms_owner = sum(own) / len(own)
+        call_ms_reader = sum(non) / len(non) if non else None
 
-        # end to end: host buffers in, host buffer out, copies inside the timed region
+        # (4) end to end: host buffers in, host buffer out, copies inside the timed region
         hb = harness.step_tensors(dw, device="cpu", pin=True)
         h_slot = dw.slot_new.cpu().pin_memory()
         h_pt = dw.page_table_cpu.contiguous().pin_memory()
@@ -248,36 +284,22 @@ def main():
         def step_host():
             cache.skv_decode_step_host(hb["Q"], hb["K"], hb["V"], h_slot, h_pt, h_len, hb["out"], staging)
 
-        for _ in range(args.warmup):
-            step_host()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            step_host()
-        e1.record()
-        barrier()
-        ms_e2e = e0.elapsed_time(e1)
+        ms_e2e = timed_steps(step_host)
     status = cache.skv_get_status()
     if status != 0:
         raise SystemExit(f"device status {status}")
-    if not torch.equal(hb["out"].view(torch.int16), t["out"].cpu().view(torch.int16)):
+    if not torch.equal(hb["out"].view(torch.int16), out_default.cpu().view(torch.int16)):
         raise SystemExit("host-buffer step and device-resident step disagree")
 
-    times = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(times[0]), float(times[1])
+    ms, ms_hbm, ms_e2e = max_over_ranks([ms, ms_hbm, ms_e2e], world, dev)
     if rank != 0:
         return
 
     peak, peak_kind = _peaks()
-    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
-    e2e_value = world * step_bytes * args.steps / (ms_e2e * 1e-3) / 1e9
-    # the roofline figure is taken on the owner layers' launches: their pages were last touched a whole
-    # model pass ago, so nothing of them is in L2 (a layer that re-reads its predecessor's owner can be faster)
-    achieved = dw.kv_bytes_per_call() / (kern_ms_owner * 1e-3) / 1e9
+    value = whole_job_rate(step_bytes, args.steps, ms, world) / 1e9
+    e2e_value = whole_job_rate(step_bytes, args.steps, ms_e2e, world) / 1e9
+    us_per_launch = ms_hbm * 1e3 / (args.steps * L)
+    achieved = attn_bytes / (us_per_launch * 1e-6) / 1e9
     h2d = sum(hb[k].numel() * 2 for k in ("Q", "K", "V")) + h_slot.numel() * 8 + h_pt.numel() * 4 + h_len.numel() * 4
     d2h = hb["out"].numel() * 2
     line = {
@@ -287,8 +309,8 @@ def main():
         "config": {"workload": w.name, "family": w.family, "n_layers": L, "owners": n_own, "batch": dw.batch,
                    "tokens": int(dw.lens_cpu.sum()), "q_heads": w.q_heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size,
-                   "l2": "inputs larger than L2: every attention call streams %.0f MB of pages" % (dw.kv_bytes_per_call() / 1e6),
-                   "step": "append (owners) + decode attention for every layer"},
+                   "l2": "inputs larger than L2: every attention call streams %.0f MB of pages" % (attn_bytes / 1e6),
+                   "step": "update of every owner layer + decode attention (split-K + merge) for every layer"},
         "steps_per_s": world * args.steps / (ms * 1e-3),
         "attn_calls_per_s": world * L * args.steps / (ms * 1e-3),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
@@ -298,11 +320,14 @@ def main():
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_splitk_kernel", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "us_per_launch": kern_ms_owner * 1e3,
-                     "us_per_launch_all_layers": kern_ms * 1e3,
-                     "us_per_launch_reader_layers": None if kern_ms_reader is None else kern_ms_reader * 1e3,
-                     "bytes_per_launch": dw.kv_bytes_per_call(),
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "us_per_launch": us_per_launch,
+                     "bytes_per_launch": attn_bytes,
+                     "how": "whole steps with L2 reuse between layers off; timed region / split-K launches in it",
                      "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "single_call": {"us_owner_layers": call_ms_owner * 1e3,
+                        "us_reader_layers": None if call_ms_reader is None else call_ms_reader * 1e3,
+                        "gbs_owner_layers": attn_bytes / (call_ms_owner * 1e-3) / 1e9,
+                        "how": "skv_decode_attn (split-K + merge) alone between two events, nothing overlapping it"},
     }
     if not args.no_cpu_baseline and world == 1:
         n_seqs = min(w.batch, args.ref_seqs)

@@ -266,7 +266,9 @@ int skv_get_status(skv_cache *cache, void *stream, int *device_status);
  * kernel (only q_heads == kv_heads), 2 = tensor-core kernel. */
 int skv_set_decode_variant(skv_cache *cache, int variant);
 
-/* Launch shape of the split-K kernel: warps per CTA (1..16), pipeline stages
+/* Launch shape of the split-K kernel (default: 8 warps per SM with two 8 KB
+ * stages each, as 2 warps x 4 CTAs per SM for the tensor-core kernel and
+ * 1 warp x 8 CTAs per SM for the CUDA-core kernel): warps per CTA (1..16), pipeline stages
  * per warp (2..8) and CTAs per SM (1..8); 0 keeps the current value.
  * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
 int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
@@ -284,9 +286,9 @@ int skv_set_decode_overlap(skv_cache *cache, int enabled);
  * such layers walk every worker's block range in alternating directions, and a
  * layer whose successor reads the same owner loads the last keep_percent % of
  * each range with normal L2 priority (everything else is loaded evict-first),
- * so the successor starts on blocks that are still in L2.  0 (default) = every
- * layer walks forward, everything evict-first.  Results do not depend on it
- * beyond floating-point summation order. */
+ * so the successor starts on blocks that are still in L2.  Default 35;
+ * 0 = every layer walks forward, everything evict-first.  Results do not depend
+ * on it beyond floating-point summation order. */
 int skv_set_decode_l2_reuse(skv_cache *cache, int keep_percent);
 
 /* Tracing: while a device buffer of at least 32 * skv_decode_worker_count bytes

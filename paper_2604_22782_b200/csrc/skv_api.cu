@@ -23,7 +23,8 @@ struct skv_cache {
     int sm_count = 0;
     int max_smem_optin = 0;
     DecodeTuning tune{0, 2, 2, 4, 1};
-    int l2_keep_pct = 0;             // > 0: consecutive layers that read one owner walk it in opposite directions
+    bool shape_is_default = true;    // until skv_set_decode_tuning is called: the CUDA-core kernel runs as 1 x 2 x 8
+    int l2_keep_pct = 35;            // > 0: consecutive layers that read one owner walk it in opposite directions
     std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
     std::vector<uint8_t> walk_keep;      // per layer: the next layer reads the same owner
     int64_t launches = 0;
@@ -324,7 +325,16 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     const int W = n_workers_of(c);
     const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
-    const size_t smem = decode_smem_bytes(c->head_dim, batch, c->tune.warps, c->tune.stages);
+    const bool tensor_core = c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
+    // Default launch shapes (8 warps per SM, two 8 KB stages each, many small CTAs so that the CTAs of the
+    // next launch can move in one by one): 2 warps x 4 CTAs per SM for the tensor-core kernel, 1 warp x 8
+    // CTAs per SM for the CUDA-core kernel (measured best for each on B200).  Same worker count either way.
+    int warps = c->tune.warps, ctas = c->tune.ctas_per_sm;
+    if (c->shape_is_default && !tensor_core) {
+        warps = 1;
+        ctas = 8;
+    }
+    const size_t smem = decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
@@ -352,9 +362,8 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     }
     p.status = c->status_word();
     p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
-    const bool tensor_core = c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
-    const int grid = c->sm_count * c->tune.ctas_per_sm;
-    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, c->tune.warps, c->tune.stages,
+    const int grid = c->sm_count * ctas;
+    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, warps, c->tune.stages,
                                                 c->tune.pdl != 0, st);
     if (le != cudaSuccess) {
         (void)cudaGetLastError();
@@ -611,6 +620,7 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
         if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     }
     c->tune = t;
+    c->shape_is_default = false;
     return SKV_OK;
 }
 
