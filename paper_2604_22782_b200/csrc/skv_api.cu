@@ -405,6 +405,8 @@ int launch_merge_on(skv_cache *c, void *out, int batch, int q_heads, void *works
     m.Hkv = c->kv_heads;
     m.D = c->head_dim;
     m.n_workers = W;
+    // with overlappable launches the merge grid must be resident in one wave (see merge_kernel)
+    m.max_ctas = c->tune.pdl ? (c->sm_count > 0 ? c->sm_count : 1) : 0x7FFFFFFF;
     if (launch_merge(m, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;

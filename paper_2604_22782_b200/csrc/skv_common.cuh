@@ -82,6 +82,7 @@ struct MergeParams {
     uint16_t *out;              // [B][Hq][D] bf16 bits
     int B, Hq, Hkv, D;
     int n_workers;
+    int max_ctas;               // grid limit (one CTA per SM)
 };
 
 struct DecodeTuning {

@@ -373,21 +373,6 @@ __device__ __forceinline__ void merge_rows(const float *part_o, const float *par
         if (e < E2) dst[e] = pack_bf16x2(acc[e].x * inv, acc[e].y * inv);
 }
 
-template <int D>
-__device__ __forceinline__ void merge_segment(const float *part_o, const float *part_ml, uint16_t *out_seg, int G,
-                                              int slot0, int n, int lane)
-{
-    const int E2 = (G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8) * D / 64;
-#ifndef SKV_MERGE_PAYLOAD
-#define SKV_MERGE_PAYLOAD 64                  // float2 in flight per lane while merging
-#endif
-    constexpr int P = SKV_MERGE_PAYLOAD;
-    if (E2 <= 2) merge_rows<D, 2, (P / 2 > 16 ? 16 : P / 2)>(part_o, part_ml, out_seg, G, slot0, n, lane);
-    else if (E2 <= 4) merge_rows<D, 4, (P / 4 > 16 ? 16 : P / 4)>(part_o, part_ml, out_seg, G, slot0, n, lane);
-    else if (E2 <= 8) merge_rows<D, 8, P / 8>(part_o, part_ml, out_seg, G, slot0, n, lane);
-    else merge_rows<D, 16, P / 16>(part_o, part_ml, out_seg, G, slot0, n, lane);
-}
-
 // ---------------------------------------------------------------------------
 template <int D, class State>
 __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
@@ -564,28 +549,51 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
 // Stand-alone merge kernel: one warp per (sequence, kv head) segment.
 // ---------------------------------------------------------------------------
 constexpr int MERGE_WARPS = 2;
+#ifndef SKV_MERGE_PAYLOAD
+#define SKV_MERGE_PAYLOAD 64                  // float2 in flight per lane while merging
+#endif
 
+// this warp's share of the segments: seg0, seg0 + stride, ...
+template <int D, int E2MAX, int NB>
+__device__ __forceinline__ void merge_loop(const MergeParams &p, int64_t seg0, int64_t stride, int lane)
+{
+    const int64_t n_seg = (int64_t)p.B * p.Hkv;
+    const int G = p.Hq / p.Hkv;
+    const int64_t T = (int64_t)p.prefix[p.B] * p.Hkv;
+    for (int64_t seg = seg0; seg < n_seg; seg += stride) {
+        const int b = (int)(seg / p.Hkv), kvh = (int)(seg - (int64_t)b * p.Hkv);
+        const int pages = p.prefix[b + 1] - p.prefix[b];
+        uint16_t *out_seg = p.out + ((int64_t)b * p.Hq + (int64_t)kvh * G) * D;
+        if (pages == 0) {
+            uint32_t *dst = reinterpret_cast<uint32_t *>(out_seg);
+            for (int i = lane; i < G * D / 2; i += 32) dst[i] = 0u;
+            continue;
+        }
+        const int64_t s0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)kvh * pages;
+        int slot0, n_part;
+        segment_partials(T, p.n_workers, seg, s0, pages, slot0, n_part);
+        merge_rows<D, E2MAX, NB>(p.part_o, p.part_ml, out_seg, G, slot0, n_part, lane);
+    }
+}
+
+// One warp per (sequence, kv head) segment, a grid of at most one CTA per SM walking the segments:
+// every CTA must be resident (waiting for the split-K launch to end) before the launch after this
+// one may be scheduled, so the grid has to fit beside the split-K CTAs in one wave.
 template <int D>
 __global__ void __launch_bounds__(MERGE_WARPS * 32) merge_kernel(MergeParams p)
 {
     pdl_trigger();        // nothing after this kernel in the stream needs to wait for its start
     pdl_wait();           // the partials come from the kernel before this one
     const int lane = threadIdx.x & 31;
-    const int64_t seg = (int64_t)blockIdx.x * MERGE_WARPS + (threadIdx.x >> 5);
-    if (seg >= (int64_t)p.B * p.Hkv) return;
-    const int b = (int)(seg / p.Hkv), kvh = (int)(seg - (int64_t)b * p.Hkv);
-    const int pages = p.prefix[b + 1] - p.prefix[b];
+    const int64_t seg0 = (int64_t)blockIdx.x * MERGE_WARPS + (threadIdx.x >> 5);
+    const int64_t stride = (int64_t)gridDim.x * MERGE_WARPS;
     const int G = p.Hq / p.Hkv;
-    if (pages == 0) {
-        uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)kvh * G) * D);
-        for (int i = lane; i < G * D / 2; i += 32) dst[i] = 0u;
-        return;
-    }
-    const int64_t T = (int64_t)p.prefix[p.B] * p.Hkv;
-    const int64_t s0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)kvh * pages;
-    int slot0, n_part;
-    segment_partials(T, p.n_workers, seg, s0, pages, slot0, n_part);
-    merge_segment<D>(p.part_o, p.part_ml, p.out + ((int64_t)b * p.Hq + (int64_t)kvh * G) * D, G, slot0, n_part, lane);
+    const int E2 = (G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8) * D / 64;   // float2 per lane, see merge_rows
+    constexpr int P = SKV_MERGE_PAYLOAD;
+    if (E2 <= 2) merge_loop<D, 2, (P / 2 > 16 ? 16 : P / 2)>(p, seg0, stride, lane);
+    else if (E2 <= 4) merge_loop<D, 4, (P / 4 > 16 ? 16 : P / 4)>(p, seg0, stride, lane);
+    else if (E2 <= 8) merge_loop<D, 8, P / 8>(p, seg0, stride, lane);
+    else merge_loop<D, 16, P / 16>(p, seg0, stride, lane);
 }
 
 template <int D, class State>
@@ -635,7 +643,8 @@ cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s)
 {
     const int64_t segs = (int64_t)p.B * p.Hkv;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((segs + MERGE_WARPS - 1) / MERGE_WARPS));
+    const int64_t want = (segs + MERGE_WARPS - 1) / MERGE_WARPS;
+    cfg.gridDim = dim3((unsigned)(want < p.max_ctas ? want : p.max_ctas));
     cfg.blockDim = dim3(MERGE_WARPS * 32);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
