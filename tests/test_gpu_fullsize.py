@@ -1,0 +1,132 @@
+"""The five full-size workloads, in the launch configuration the benchmark times (library defaults,
+whole step through skv_decode_step).  The oracle cannot hold these whole, so:
+  - cache contents are compared bit for bit for EVERY token of EVERY owner layer, on the device,
+    against the rows the generator draws (the update is a pure copy);
+  - attention outputs are compared with the oracle, element by element within
+    |out - ref| <= 1e-2 + 1e-2 |ref|, for a sample of sequences (shortest, longest, seeded picks;
+    full length, all heads) on a sample of layers (first owner, its first reader, last owner, last layer);
+  - every other output row must be finite and lie inside the convex-combination bound
+    |out| <= max |V| of the generator's value table."""
+import pytest
+import torch
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 1e-2, 1e-2
+
+
+def _sample_sequences(lens, k, seed):
+    order = torch.argsort(lens.to(torch.int64), stable=True)
+    picks = [int(order[0]), int(order[-1])]
+    g = torch.Generator().manual_seed(seed)
+    for i in torch.randperm(lens.numel(), generator=g).tolist():
+        if len(picks) >= k:
+            break
+        if i not in picks:
+            picks.append(i)
+    return picks[:k]
+
+
+def _sample_layers(r):
+    L = len(r)
+    owners = [l for l in range(L) if r[l] == l]
+    first_reader = next((l for l in range(L) if r[l] != l), 0)
+    return sorted({0, first_reader, owners[-1], L - 1})
+
+
+def _check_workload(w, n_seqs):
+    from oracle import Oracle
+    from paper_2604_22782_b200 import harness
+    dw = harness.setup(w)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    t["out"].fill_(float("nan"))
+    dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+
+    # byte accounting scales exactly with the owner count
+    stats = dw.cache.skv_cache_stats()
+    assert stats["n_owners"] == len(dw.owners)
+    assert stats["bytes_per_token"] == 2 * len(dw.owners) * w.kv_heads * w.head_dim * 2
+    assert stats["kv_bytes"] == len(dw.owners) * dw.total_pages * (2 * w.page_size * w.kv_heads * w.head_dim * 2)
+
+    # cache: every token of every owner layer, bit for bit, against what the generator draws
+    seq_idx, pos = W.token_index(dw.lens_cpu)
+    slots = W.slot_map_for(dw.page_table_cpu, seq_idx, pos, w.page_size)
+    chunk = 1 << 16
+    for l in dw.owners:
+        for s in range(0, seq_idx.numel(), chunk):
+            e = min(seq_idx.numel(), s + chunk)
+            Kd, Vd = W.draw_kv(w, l, seq_idx[s:e], pos[s:e], device=dw.device)
+            Kg, Vg = torch.empty_like(Kd), torch.empty_like(Vd)
+            dw.cache.skv_gather(l, slots[s:e].to(dw.device), Kg, Vg)
+            assert torch.equal(Kg.view(torch.int16), Kd.view(torch.int16)), f"K of layer {l}, tokens {s}..{e}"
+            assert torch.equal(Vg.view(torch.int16), Vd.view(torch.int16)), f"V of layer {l}, tokens {s}..{e}"
+
+    # attention outputs of the sampled sequences on the sampled layers against the oracle
+    seqs = _sample_sequences(dw.lens_cpu, n_seqs, w.seed + 7)
+    layers = _sample_layers(dw.r)
+    sub_lens = dw.lens_cpu[seqs]
+    o = Oracle(w.n_layers, dw.r, w.q_heads, w.kv_heads, w.head_dim, len(seqs), int(sub_lens.max()))
+    local, lpos = W.token_index(sub_lens)
+    glob = torch.as_tensor(seqs, dtype=torch.int64)[local]
+    for src in sorted({dw.r[l] for l in layers}):
+        for s in range(0, local.numel(), chunk):     # drawn on the device (same bits as on the CPU), used on the CPU
+            e = min(local.numel(), s + chunk)
+            K, V = W.draw_kv(w, src, glob[s:e], lpos[s:e], device=dw.device)
+            o.append(src, K.cpu(), V.cpu(), local[s:e], lpos[s:e])
+    worst = 0.0
+    for l in layers:
+        Q = t["Q"][l].cpu()[seqs]
+        ref = o.decode_attn(l, Q, sub_lens)
+        got = t["out"][l].cpu()[seqs].double()
+        err = (got - ref).abs()
+        assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {l}: max abs err {err.max().item()}"
+        worst = max(worst, err.max().item())
+    o.close()
+
+    # every row: finite and inside the convex-combination bound
+    vmax = 5.0 * w.kv_std            # the generator's table ends below 4.5 standard deviations
+    out = t["out"].float()
+    assert torch.isfinite(out).all()
+    assert out.abs().max().item() <= vmax
+    return worst
+
+
+def test_llama3_8b_full_size():
+    """Config 2: 32 layers, 32q/8kv, D=128, 16 owners, batch 32, lengths U[1024,4096]."""
+    _check_workload(W.get_workload("llama3_8b"), n_seqs=6)
+
+
+def test_qwen3_8b_full_size():
+    """Config 3: 36 layers in groups of 4 (9 owners), batch 64, lengths U[2048,8192], Q std 0.5."""
+    _check_workload(W.get_workload("qwen3_8b"), n_seqs=4)
+
+
+def test_llama2_7b_32k_full_size():
+    """Config 4: MHA 32/32, stochastic routing map, batch 8 x 32768 tokens (the CUDA-core kernel)."""
+    w = W.get_workload("llama2_7b_32k")
+    free, _ = torch.cuda.mem_get_info()
+    from paper_2604_22782_b200.binding import skv_cache_pool_bytes
+    need = skv_cache_pool_bytes(W.routing_map(w), w.kv_heads, w.head_dim, w.page_size, 8 * 2048)
+    if free < need + (8 << 30):
+        pytest.skip(f"needs {need / 1e9:.0f} GB of device memory for the pool")
+    _check_workload(w, n_seqs=2)
+
+
+@pytest.mark.parametrize("group", [1, 2, 4, 8])
+def test_sharing_sweep_full_size(group):
+    """Config 5: Llama-3-8B shape, batch 128, lengths U[512,2048], owner fraction 1/group."""
+    _check_workload(W.sweep_workload(group), n_seqs=4)
+
+
+def test_sharing_sweep_cache_bytes_scale_exactly():
+    """Pool bytes of the four sweep points are in the ratio 32:16:8:4 (same pages, fewer owner layers)."""
+    from paper_2604_22782_b200.binding import skv_cache_pool_bytes
+    lens = W.seq_lens(W.sweep_workload(1))
+    pages = int(((lens.to(torch.int64) + 15) // 16).sum())
+    sizes = [skv_cache_pool_bytes(W.routing_map(W.sweep_workload(g)), 8, 128, 16, pages) - 256 for g in (1, 2, 4, 8)]
+    assert [s * g for s, g in zip(sizes, (1, 2, 4, 8))] == [sizes[0]] * 4
