@@ -62,7 +62,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "25"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -72,6 +72,12 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
+
+    def wait_first(self, timeout_s: float = 5.0):
+        """nvidia-smi needs a moment to start: wait for its first sample before the timed work begins."""
+        t0 = time.time()
+        while self.proc and not self.rows and time.time() - t0 < timeout_s:
+            time.sleep(0.05)
 
     def __exit__(self, *a):
         if self.proc:
@@ -186,6 +192,7 @@ def main():
     ap.add_argument("--tuning", default="", help="warps,stages,ctas_per_sm of the split-K kernel")
     ap.add_argument("--overlap", type=int, default=-1, help="1 = overlappable (chained) launches, 0 = plain launches")
     ap.add_argument("--l2-keep", type=int, default=-1, help="percent of each block range kept in L2 for the next layer")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sharing-ratio sweep (owner fractions 1, 1/2, 1/4, 1/8)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = W.get_workload(args.workload)
@@ -239,6 +246,7 @@ def main():
         return e0.elapsed_time(e1)
 
     with ClockSampler(local) as clocks:
+        clocks.wait_first()
         # (1) the headline: whole decode steps, inputs resident in HBM, library defaults
         launches0 = cache.skv_launch_count()
         ms = timed_steps(step)
@@ -341,10 +349,63 @@ def main():
             "value": nbytes / best / 1e9, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
             "sample": f"1 decode-attention call (layer {layer} reading layer {dw.r[layer]}) over the first {n_seqs} "
                       f"sequences ({int(sl.sum())} tokens), best of 3, {best * 1e3:.1f} ms"}
+    if not args.no_sweep and world == 1:
+        del dw, cache, t, hb, staging
+        torch.cuda.empty_cache()
+        line["sharing_sweep"] = sharing_sweep(args, dev)
     print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def sharing_sweep(args, dev):
+    """Llama-3-8B shape, batch 128, lengths U[512,2048]: owner fractions 1, 1/2, 1/4, 1/8 (evenly spaced
+    owners).  Per ratio: cache bytes, the largest batch a 120e9-byte KV budget holds, whole decode steps per
+    second (update of the owners + attention of all 32 layers) and the time per attention call."""
+    from paper_2604_22782_b200 import harness
+    rows = []
+    budget = 120e9
+    for g in (1, 2, 4, 8):
+        w = W.sweep_workload(g)
+        dw = harness.setup(w, device=dev)
+        harness.prefill(dw, upto_offset=-1)
+        t = harness.step_tensors(dw)
+        cache = dw.cache
+
+        def step():
+            cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"],
+                                  dw.workspace)
+
+        for _ in range(args.warmup):
+            step()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = max(3, args.steps // 2)
+        e0.record()
+        for _ in range(n):
+            step()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / n
+        st = cache.skv_cache_stats()
+        pages = (dw.lens_cpu.to(torch.int64) + w.page_size - 1) // w.page_size
+        per_seq_mean = st["n_owners"] * float(pages.double().mean()) * st["page_bytes"]
+        per_seq_worst = st["n_owners"] * ((w.len_hi + w.page_size - 1) // w.page_size) * st["page_bytes"]
+        tokens = int(dw.lens_cpu.sum())
+        rows.append({
+            "owner_fraction": 1.0 / g, "owners": st["n_owners"], "kv_bytes_per_token": st["bytes_per_token"],
+            "kv_bytes_tokens": st["bytes_per_token"] * tokens, "kv_bytes_pages": st["kv_bytes"],
+            "max_batch_120e9_mean_len": int(budget // per_seq_mean),
+            "max_batch_120e9_max_len": int(budget // per_seq_worst),
+            "ms_per_step": ms, "steps_per_s": 1e3 / ms, "us_per_attn_call": ms * 1e3 / w.n_layers,
+            "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
+        })
+        if cache.skv_get_status() != 0:
+            raise SystemExit("device status after the sweep")
+        del dw, cache, t
+        torch.cuda.empty_cache()
+    return rows
 
 
 if __name__ == "__main__":
