@@ -269,3 +269,23 @@ def test_explicit_scale_is_used():
     assert ok, err
     ok_default, _ = _within_tol(out, o.decode_attn(0, Q.cpu(), dw.lens_cpu))
     assert not ok_default
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,hi", [(300, 4, 1, 40), (3000, 4, 2, 48), (700, 8, 8, 33)])
+def test_many_short_sequences(B, Hq, Hkv, hi):
+    """Large batches of very short sequences (some empty): fewer blocks than workers in the first case
+    (every worker holds at most one block), several whole segments per worker in the others."""
+    g = torch.Generator().manual_seed(B)
+    lens = torch.randint(0, hi + 1, (B,), generator=g, dtype=torch.int32)
+    w = W.Workload("short_many", 2, Hq, Hkv, 128, 16, B, 0, hi, "explicit", explicit_r=(0, 0), seed=51)
+    _full_step_check(w, lens=lens, check_cache=False)
+
+
+def test_all_sequences_empty():
+    """Nothing cached anywhere: every output row is zero and nothing is read."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.zeros(5, dtype=torch.int32)
+    w = W.Workload("empty", 1, 8, 2, 128, 16, 5, 0, 0, "explicit", explicit_r=(0,), seed=53)
+    dw = harness.setup(w, lens=lens)
+    _, out = _decode_layer(dw, 0)
+    assert torch.count_nonzero(out.view(torch.int16)) == 0

@@ -297,3 +297,60 @@ def test_oracle_on_the_tiny_workload_matches_library_attention():
         Q = W.draw_q(w, l)
         want = _sdpa64(Q, dense[r[l]][0], dense[r[l]][1], lens, w.head_dim ** -0.5)
         assert torch.allclose(o.decode_attn(l, Q, lens), want, rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ do the pins bite?
+class _Mutant(Oracle):
+    """The oracle with one plausible mistake planted on the CPU side of its interface."""
+
+    def __init__(self, mistake, *a, **k):
+        super().__init__(*a, **k)
+        self.mistake = mistake
+
+    def append(self, layer, K, V, seq_idx, pos):
+        if self.mistake == "swap_kv":
+            K, V = V, K
+        super().append(layer, K, V, seq_idx, pos)
+
+    def decode_attn(self, layer, Q, seq_lens, scale=None):
+        scale = self.D ** -0.5 if scale is None else scale
+        if self.mistake == "no_scale":
+            scale = 1.0
+        if self.mistake == "short_by_one":
+            seq_lens = (seq_lens - 1).clamp(min=0)
+        if self.mistake == "own_layer":          # ignores the routing map: reads the layer's own store
+            return self._identity_twin.decode_attn(layer, Q, seq_lens, scale)
+        if self.mistake == "head_mod":           # query head h reads kv head h % Hkv instead of h // G
+            G = self.Hq // self.Hkv
+            perm = torch.tensor([(h % self.Hkv) * G + h // self.Hkv for h in range(self.Hq)])
+            inv = torch.empty_like(perm)
+            inv[perm] = torch.arange(self.Hq)
+            return super().decode_attn(layer, Q[:, inv].contiguous(), seq_lens, scale)[:, perm]
+        return super().decode_attn(layer, Q, seq_lens, scale)
+
+
+def _pins_hold(make):
+    """A small set of the pins above, as one predicate over an oracle constructor."""
+    L, B, n, Hq, Hkv, D = 4, 2, 12, 4, 2, 16
+    r = [0, 0, 2, 2]
+    o = make(L, r, Hq, Hkv, D, B, n)
+    twin = Oracle(L, list(range(L)), Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=11)
+    _fill(twin, L, B, n, Hkv, D, seed=11)
+    o._identity_twin = twin
+    lens = torch.tensor([12, 5], dtype=torch.int32)
+    ok = True
+    for l in range(L):
+        Q = _rand_bf16((B, Hq, D), 70 + l)
+        want = _sdpa64(Q, store[r[l]][0], store[r[l]][1], lens, D ** -0.5)     # library attention on the source layer
+        ok &= torch.allclose(o.decode_attn(l, Q, lens), want, rtol=1e-12, atol=1e-13)
+    one = torch.tensor([1, 1], dtype=torch.int32)                               # a single cached token returns its V
+    got = o.decode_attn(0, _rand_bf16((B, Hq, D), 5), one)
+    ok &= torch.equal(got, store[0][1][:, 0].double().repeat_interleave(Hq // Hkv, 1))
+    return bool(ok)
+
+
+def test_planted_mistakes_fail_the_pins():
+    assert _pins_hold(Oracle)
+    for mistake in ("swap_kv", "no_scale", "short_by_one", "own_layer", "head_mod"):
+        assert not _pins_hold(lambda *a, m=mistake: _Mutant(m, *a)), f"the pins accept an oracle with '{mistake}'"
