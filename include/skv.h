@@ -99,7 +99,8 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
                      int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes,
                      void *stream);
 
-/* Frees host state only; never touches device_pool. */
+/* Frees host state (and the handle's copy stream and events, if
+ * skv_decode_step_host created them); never touches device_pool. */
 void skv_cache_destroy(skv_cache *cache);
 
 /* r[layer] (>= 0) or SKV_ERR_LAYER. */
@@ -235,9 +236,13 @@ int skv_decode_step(skv_cache *cache, const void *Q, const void *K, const void *
 
 /* One whole decode step of Algorithm 2 from HOST buffers: copies the step's
  * inputs to the device, runs append + decode attention for layers 0..L-1 in
- * order, and copies the outputs back, all on `stream` (the caller
- * synchronises).  Host buffers should be pinned for the copies to be
- * asynchronous.
+ * order, and copies the outputs back.  Everything is ordered after the work
+ * already on `stream`, and `stream` is complete only when the outputs are in
+ * h_out (the caller synchronises `stream`); inside, the layers are cut into up
+ * to four groups and a copy stream owned by the handle (created on the first
+ * call, destroyed by skv_cache_destroy) moves one group's queries in and
+ * another group's outputs out while a third group's kernels run.  Host buffers
+ * should be pinned for the copies to be asynchronous.
  *   hQ          host bf16 [n_layers][batch][q_heads][head_dim]
  *   hK, hV      host bf16 [n_owners][batch][kv_heads][head_dim], owner layers
  *               in increasing layer order

@@ -30,6 +30,11 @@ struct skv_cache {
     int64_t launches = 0;
     unsigned long long *trace = nullptr;   // optional per-worker timestamps (device)
     size_t trace_bytes = 0;
+    // skv_decode_step_host: a copy stream and events that let host<->device copies of one part of the
+    // step run beside the kernels of another (created on first use, destroyed with the handle)
+    static constexpr int HOST_GROUPS = 4;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_entry = nullptr, ev_exit = nullptr, ev_in[HOST_GROUPS] = {}, ev_done[HOST_GROUPS] = {};
 
     int *status_word() const { return reinterpret_cast<int *>(pool); }
     uint8_t *layer_base(int owner_slot) const
@@ -224,7 +229,22 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
     return SKV_OK;
 }
 
-void skv_cache_destroy(skv_cache *cache) { delete cache; }
+void skv_cache_destroy(skv_cache *cache)
+{
+    if (!cache) return;
+    if (cache->copy_stream) {
+        (void)cudaStreamSynchronize(cache->copy_stream);
+        (void)cudaStreamDestroy(cache->copy_stream);
+        (void)cudaEventDestroy(cache->ev_entry);
+        (void)cudaEventDestroy(cache->ev_exit);
+        for (int g = 0; g < skv_cache::HOST_GROUPS; ++g) {
+            (void)cudaEventDestroy(cache->ev_in[g]);
+            (void)cudaEventDestroy(cache->ev_done[g]);
+        }
+        (void)cudaGetLastError();
+    }
+    delete cache;
+}
 
 int skv_layer_owner(const skv_cache *c, int layer)
 {
@@ -450,43 +470,17 @@ int decode_attn_on_scratch(skv_cache *c, int layer, const void *Q, const int32_t
 
 extern "C" {
 
-int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, const int64_t *slot_map,
-                    const int32_t *page_table, const int32_t *seq_lens, void *out, int batch, int q_heads,
-                    int pt_stride, float scale, void *workspace, size_t workspace_bytes, void *stream)
+}  // extern "C"
+
+namespace {
+// The updates of every owner layer of one step in one launch.  K, V: [n_owners][batch][kv_heads][head_dim].
+int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot_map, int batch, void *stream)
 {
-    int rc = check_decode_args(c, 0, batch, q_heads);
-    if (rc) return rc;
-    if (!Q || !K || !V || !slot_map || !out) return SKV_ERR_ARG;
-    const size_t q_layer = (size_t)batch * q_heads * c->head_dim * 2;
-    const size_t kv_layer = (size_t)batch * c->kv_heads * c->head_dim * 2;
-    const uint8_t *q = static_cast<const uint8_t *>(Q), *k = static_cast<const uint8_t *>(K),
-                  *v = static_cast<const uint8_t *>(V);
-    uint8_t *o = static_cast<uint8_t *>(out);
-    if (!c->tune.pdl) {
-        // layer by layer, exactly as a caller of the per-layer entry points would
-        for (int l = 0; l < c->n_layers; ++l) {
-            const int os = c->slot[(size_t)l];
-            if (os >= 0) {
-                rc = skv_append(c, l, k + (size_t)os * kv_layer, v + (size_t)os * kv_layer, slot_map, batch, stream);
-                if (rc) return rc;
-            }
-            rc = skv_decode_attn(c, l, q + (size_t)l * q_layer, page_table, seq_lens, o + (size_t)l * q_layer, batch,
-                                 q_heads, pt_stride, scale, workspace, workspace_bytes, stream);
-            if (rc) return rc;
-        }
-        return SKV_OK;
-    }
-    // All inputs of the step exist before it starts, and the update of layer l touches only layer l's
-    // pages, which no layer before l reads: so every owner's update goes first, in one launch, and the
-    // attention calls form a chain in which the split-K launch of layer l+1 may start while that of layer l
-    // is finishing and its merge is running (they work on alternate workspace buffers; a split-K launch
-    // waits for everything before it half-way through its own work, which also keeps the launch of layer
-    // l+2 from starting before layer l has been merged).
     if (!aligned(K, 16) || !aligned(V, 16)) return SKV_ERR_ARG;
     AppendParams ap;
     ap.layer_base = c->layer_base(0);
-    ap.K = reinterpret_cast<const uint4 *>(k);
-    ap.V = reinterpret_cast<const uint4 *>(v);
+    ap.K = static_cast<const uint4 *>(K);
+    ap.V = static_cast<const uint4 *>(V);
     ap.slot_map = slot_map;
     ap.n_tokens = batch;
     ap.n_slots = c->max_pages * PAGE;
@@ -500,15 +494,62 @@ int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, c
         return SKV_ERR_CUDA;
     }
     c->launches += 1;
-    for (int l = 0; l < c->n_layers; ++l) {
+    return SKV_OK;
+}
+
+// Attention of layers [l0, l1) of one step.  With overlappable launches: a chain in which the split-K launch
+// of layer l+1 may start while that of layer l is finishing and its merge is running (they work on alternate
+// workspace buffers; a split-K launch waits for everything before it half-way through its own work, which
+// also keeps the launch of layer l+2 from starting before layer l has been merged); the first launch of
+// the chain waits before it reads anything.  `updates_done` = the owners' updates of the step have been
+// issued already (else each owner layer is updated just before its attention).
+int step_layers(skv_cache *c, int l0, int l1, const uint8_t *q, const uint8_t *k, const uint8_t *v,
+                const int64_t *slot_map, const int32_t *page_table, const int32_t *seq_lens, uint8_t *o, int batch,
+                int q_heads, int pt_stride, float scale, void *workspace, size_t workspace_bytes, void *stream,
+                bool updates_done)
+{
+    const size_t q_layer = (size_t)batch * q_heads * c->head_dim * 2;
+    const size_t kv_layer = (size_t)batch * c->kv_heads * c->head_dim * 2;
+    for (int l = l0; l < l1; ++l) {
+        const int os = c->slot[(size_t)l];
+        int rc;
+        if (os >= 0 && !updates_done) {
+            rc = skv_append(c, l, k + (size_t)os * kv_layer, v + (size_t)os * kv_layer, slot_map, batch, stream);
+            if (rc) return rc;
+        }
+        const bool chained = c->tune.pdl && updates_done && l > l0;
         rc = launch_splitk(c, l, q + (size_t)l * q_layer, page_table, seq_lens, batch, q_heads, pt_stride, scale,
-                           workspace, workspace_bytes, stream, l & 1, l > 0);
+                           workspace, workspace_bytes, stream, l & 1, chained);
         if (rc) return rc;
         // the merge kernel waits for that launch and lets the next split-K launch be scheduled at once
         rc = launch_merge_on(c, o + (size_t)l * q_layer, batch, q_heads, workspace, workspace_bytes, stream, l & 1);
         if (rc) return rc;
     }
     return SKV_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, const int64_t *slot_map,
+                    const int32_t *page_table, const int32_t *seq_lens, void *out, int batch, int q_heads,
+                    int pt_stride, float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_decode_args(c, 0, batch, q_heads);
+    if (rc) return rc;
+    if (!Q || !K || !V || !slot_map || !out) return SKV_ERR_ARG;
+    // All inputs of the step exist before it starts, and the update of layer l touches only layer l's
+    // pages, which no layer before l reads: so (with overlappable launches) every owner's update goes
+    // first, in one launch, and the attention calls form one chain.  Without them: layer by layer,
+    // exactly as a caller of the per-layer entry points would.
+    const bool batched = c->tune.pdl != 0;
+    if (batched) {
+        rc = step_updates(c, K, V, slot_map, batch, stream);
+        if (rc) return rc;
+    }
+    return step_layers(c, 0, c->n_layers, static_cast<const uint8_t *>(Q), static_cast<const uint8_t *>(K),
+                       static_cast<const uint8_t *>(V), slot_map, page_table, seq_lens, static_cast<uint8_t *>(out),
+                       batch, q_heads, pt_stride, scale, workspace, workspace_bytes, stream, batched);
 }
 
 // ---- whole decode step from host buffers -------------------------------------
@@ -549,6 +590,22 @@ int skv_decode_step_staging_bytes(const skv_cache *c, int batch, int q_heads, in
     return SKV_OK;
 }
 
+namespace {
+bool host_step_resources(skv_cache *c)
+{
+    if (c->copy_stream) return true;
+    bool ok = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_entry, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_exit, cudaEventDisableTiming) == cudaSuccess;
+    for (int g = 0; ok && g < skv_cache::HOST_GROUPS; ++g) {
+        ok = ok && cudaEventCreateWithFlags(&c->ev_in[g], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->ev_done[g], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) (void)cudaGetLastError();
+    return ok;
+}
+}  // namespace
+
 int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const void *hV, const int64_t *h_slot_map,
                          const int32_t *h_page_table, const int32_t *h_seq_lens, void *h_out, int batch,
                          int q_heads, int pt_stride, float scale, void *staging, size_t staging_bytes, void *stream)
@@ -561,27 +618,57 @@ int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const voi
     rc = staging_layout(c, batch, q_heads, pt_stride, &s);
     if (rc) return rc;
     if (staging_bytes < s.total) return SKV_ERR_NOMEM;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!host_step_resources(c)) return SKV_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream), cs = c->copy_stream;
     uint8_t *d = static_cast<uint8_t *>(staging);
+    const uint8_t *hq = static_cast<const uint8_t *>(hQ);
+    uint8_t *ho = static_cast<uint8_t *>(h_out);
     const size_t q_layer = (size_t)batch * q_heads * c->head_dim * 2;
     const size_t kv_layer = (size_t)batch * c->kv_heads * c->head_dim * 2;
-    bool ok = true;
-    ok &= cudaMemcpyAsync(d + s.q, hQ, q_layer * c->n_layers, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + s.k, hK, kv_layer * c->n_owners, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + s.v, hV, kv_layer * c->n_owners, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + s.slot_map, h_slot_map, (size_t)batch * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + s.page_table, h_page_table, (size_t)batch * pt_stride * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + s.seq_lens, h_seq_lens, (size_t)batch * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
-    rc = skv_decode_step(c, d + s.q, d + s.k, d + s.v, reinterpret_cast<const int64_t *>(d + s.slot_map),
-                         reinterpret_cast<const int32_t *>(d + s.page_table),
-                         reinterpret_cast<const int32_t *>(d + s.seq_lens), d + s.out, batch, q_heads, pt_stride,
-                         scale, d + s.ws, s.ws_bytes, stream);
-    if (rc) return rc;
-    if (cudaMemcpyAsync(h_out, d + s.out, q_layer * c->n_layers, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return SKV_ERR_CUDA;
+    const int L = c->n_layers, NG = L < skv_cache::HOST_GROUPS ? L : skv_cache::HOST_GROUPS;
+    auto first_layer = [&](int g) { return (int)(((int64_t)g * L) / NG); };
+    // The layers are cut into NG groups.  Copy stream: small inputs, then the queries group by group;
+    // caller's stream: the kernels of a group as soon as its queries have arrived; copy stream again: a
+    // group's output rows as soon as its kernels are done.  So only the first group's inputs and the
+    // last group's outputs are not hidden behind kernels.
+    bool ok = cudaEventRecord(c->ev_entry, st) == cudaSuccess;             // staging may still be in use by
+    ok = ok && cudaStreamWaitEvent(cs, c->ev_entry, 0) == cudaSuccess;     // earlier work on the caller's stream
+    ok = ok && cudaMemcpyAsync(d + s.slot_map, h_slot_map, (size_t)batch * 8, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + s.page_table, h_page_table, (size_t)batch * pt_stride * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + s.seq_lens, h_seq_lens, (size_t)batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + s.k, hK, kv_layer * c->n_owners, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + s.v, hV, kv_layer * c->n_owners, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    for (int g = 0; ok && g < NG; ++g) {
+        const int l0 = first_layer(g), l1 = first_layer(g + 1);
+        ok = ok && cudaMemcpyAsync(d + s.q + l0 * q_layer, hq + l0 * q_layer, (size_t)(l1 - l0) * q_layer,
+                                   cudaMemcpyHostToDevice, cs) == cudaSuccess;
+        ok = ok && cudaEventRecord(c->ev_in[g], cs) == cudaSuccess;
     }
+    if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
+    const int64_t *slot_map = reinterpret_cast<const int64_t *>(d + s.slot_map);
+    const int32_t *page_table = reinterpret_cast<const int32_t *>(d + s.page_table);
+    const int32_t *seq_lens = reinterpret_cast<const int32_t *>(d + s.seq_lens);
+    const bool batched = c->tune.pdl != 0;
+    for (int g = 0; g < NG; ++g) {
+        const int l0 = first_layer(g), l1 = first_layer(g + 1);
+        if (cudaStreamWaitEvent(st, c->ev_in[g], 0) != cudaSuccess) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
+        if (g == 0 && batched) {
+            rc = step_updates(c, d + s.k, d + s.v, slot_map, batch, stream);
+            if (rc) return rc;
+        }
+        rc = step_layers(c, l0, l1, d + s.q, d + s.k, d + s.v, slot_map, page_table, seq_lens, d + s.out, batch,
+                         q_heads, pt_stride, scale, d + s.ws, s.ws_bytes, stream, batched);
+        if (rc) return rc;
+        ok = cudaEventRecord(c->ev_done[g], st) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(cs, c->ev_done[g], 0) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(ho + l0 * q_layer, d + s.out + l0 * q_layer, (size_t)(l1 - l0) * q_layer,
+                                   cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+        if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
+    }
+    // the caller's stream is complete only when the last rows are on the host
+    ok = cudaEventRecord(c->ev_exit, cs) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(st, c->ev_exit, 0) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
     return SKV_OK;
 }
 
