@@ -18,6 +18,12 @@
  *                       stores (Eq. (3.2) / Algorithm 2 say which l' to use).
  *                       Attn is scaled dot-product softmax attention; query
  *                       head h reads KV head floor(h / (Hq/Hkv)).
+ *   oracle_attn_rows    Pre-fill (Section 3.1.1 "processing the initial prompt of T
+ *                       tokens in parallel"): Eq. (3.1) for many query tokens at
+ *                       once, each a row (sequence b, position pos) that attends
+ *                       the source layer's tokens 0..pos of its sequence (a
+ *                       decoder is causal).  One decode step is the special case
+ *                       of one row per sequence at pos = seq_len - 1.
  *   oracle_mu           Eq. (3.2): owner set S -> map mu (0-based layers).
  *   oracle_group_map    Section 4.3: groups of g consecutive layers share the
  *                       first layer's cache.
@@ -181,6 +187,57 @@ int oracle_decode_attn(const oracle_t *o, int layer, const uint16_t *Q, const in
                 for (int d = 0; d < D; ++d) y[d] += w[t] * bf16_to_f64(v[d]);
             }
             free(w);
+        }
+    }
+    return fail ? -2 : 0;
+}
+
+/* Eq. (3.1) with l' = r[layer] for n_q query tokens processed in parallel (pre-fill):
+ * row i is a token of sequence q_seq[i] at position q_pos[i]; a decoder is causal, so it
+ * attends the source layer's tokens t = 0 .. q_pos[i] of that sequence:
+ *   s_t = scale * <Q[i,h,:], K_src[q_seq[i], t, kv(h), :]>,  w = softmax(s),
+ *   out[i,h,:] = sum_t w_t * V_src[q_seq[i], t, kv(h), :].
+ * Q: [n_q][Hq][D] bf16 bits; out: [n_q][Hq][D] fp64 (not rounded). */
+int oracle_attn_rows(const oracle_t *o, int layer, const uint16_t *Q, const int64_t *q_seq, const int64_t *q_pos,
+                     int64_t n_q, double scale, double *out)
+{
+    if (!o || layer < 0 || layer >= o->L) return -1;
+    int src = o->r[layer];
+    if (!o->K[src] || !o->V[src]) return -1;
+    int G = o->Hq / o->Hkv, D = o->D;
+    for (int64_t i = 0; i < n_q; ++i)
+        if (q_seq[i] < 0 || q_seq[i] >= o->B || q_pos[i] < 0 || q_pos[i] >= o->n_max) return -3;
+    int fail = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int64_t i = 0; i < n_q; ++i) {
+        for (int h = 0; h < o->Hq; ++h) {
+            int64_t b = q_seq[i], n = q_pos[i] + 1;
+            int kv = h / G;
+            const uint16_t *q = Q + ((size_t)i * (size_t)o->Hq + (size_t)h) * (size_t)D;
+            double *y = out + ((size_t)i * (size_t)o->Hq + (size_t)h) * (size_t)D;
+            double *s = (double *)malloc(sizeof(double) * (size_t)n);
+            if (!s) {
+#pragma omp atomic write
+                fail = 1;
+                continue;
+            }
+            double smax = -INFINITY;
+            for (int64_t t = 0; t < n; ++t) {
+                const uint16_t *k = o->K[src] + row_index(o, b, t) + (size_t)kv * (size_t)D;
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+                s[t] = scale * acc;
+                if (s[t] > smax) smax = s[t];
+            }
+            double denom = 0.0;
+            for (int64_t t = 0; t < n; ++t) { s[t] = exp(s[t] - smax); denom += s[t]; }
+            for (int d = 0; d < D; ++d) y[d] = 0.0;
+            for (int64_t t = 0; t < n; ++t) {
+                const uint16_t *v = o->V[src] + row_index(o, b, t) + (size_t)kv * (size_t)D;
+                double w = s[t] / denom;
+                for (int d = 0; d < D; ++d) y[d] += w * bf16_to_f64(v[d]);
+            }
+            free(s);
         }
     }
     return fail ? -2 : 0;

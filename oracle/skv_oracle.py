@@ -44,6 +44,7 @@ def _load():
         lib.oracle_attn_weights.argtypes = [vp, ctypes.c_int, u16p, ctypes.c_int, ctypes.c_int,
                                             ctypes.c_int64, ctypes.c_double, f64p]
         lib.oracle_decode_attn.argtypes = [vp, ctypes.c_int, u16p, i32p, ctypes.c_double, f64p]
+        lib.oracle_attn_rows.argtypes = [vp, ctypes.c_int, u16p, i64p, i64p, ctypes.c_int64, ctypes.c_double, f64p]
         lib.oracle_mu.argtypes = [ctypes.c_int, i32p, ctypes.c_int, i32p]
         lib.oracle_group_map.argtypes = [ctypes.c_int, ctypes.c_int, i32p]
         lib.oracle_count_owners.argtypes = [ctypes.c_int, i32p]
@@ -150,4 +151,22 @@ class Oracle:
         rc = self.lib.oracle_decode_attn(self.h, layer, qb.data_ptr(), lens.data_ptr(), scale, out.data_ptr())
         if rc != 0:
             raise RuntimeError(f"oracle_decode_attn failed: {rc}")
+        return out
+
+    def attn_rows(self, layer: int, Q: torch.Tensor, q_seq: torch.Tensor, q_pos: torch.Tensor,
+                  scale: Optional[float] = None) -> torch.Tensor:
+        """Pre-fill: row i of Q [n_q, Hq, D] is a token of sequence q_seq[i] at position q_pos[i] and
+        attends tokens 0..q_pos[i] of the source layer's store of that sequence."""
+        qb = _bf16_bits(Q)
+        n_q = qb.shape[0]
+        assert qb.shape == (n_q, self.Hq, self.D)
+        s = q_seq.to(torch.int64).contiguous()
+        p = q_pos.to(torch.int64).contiguous()
+        assert s.numel() == n_q and p.numel() == n_q
+        scale = self.D ** -0.5 if scale is None else scale
+        out = torch.empty((n_q, self.Hq, self.D), dtype=torch.float64)
+        rc = self.lib.oracle_attn_rows(self.h, layer, qb.data_ptr(), s.data_ptr(), p.data_ptr(), n_q, scale,
+                                       out.data_ptr())
+        if rc != 0:
+            raise RuntimeError(f"oracle_attn_rows failed: {rc}")
         return out

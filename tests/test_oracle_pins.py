@@ -354,3 +354,79 @@ def test_planted_mistakes_fail_the_pins():
     assert _pins_hold(Oracle)
     for mistake in ("swap_kv", "no_scale", "short_by_one", "own_layer", "head_mod"):
         assert not _pins_hold(lambda *a, m=mistake: _Mutant(m, *a)), f"the pins accept an oracle with '{mistake}'"
+
+
+# ------------------------------------------------------------------ pre-fill rows (many query tokens at once)
+def _causal_sdpa64(Q, K, V, pos, scale):
+    """torch's library attention in fp64 with an explicit boolean mask: query row i sees keys t <= pos[i].
+    Q [nq,Hq,D]; K,V [n,Hkv,D] of one sequence."""
+    nq, Hq, D = Q.shape
+    n, Hkv = K.shape[0], K.shape[1]
+    G = Hq // Hkv
+    q = Q.double().permute(1, 0, 2)[None]                                   # [1,Hq,nq,D]
+    k = K.double().permute(1, 0, 2).repeat_interleave(G, 0)[None]           # [1,Hq,n,D]
+    v = V.double().permute(1, 0, 2).repeat_interleave(G, 0)[None]
+    mask = torch.arange(n)[None, :] <= pos.to(torch.int64)[:, None]         # [nq,n]
+    out = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=mask[None, None], scale=scale)
+    return out[0].permute(1, 0, 2)                                          # [nq,Hq,D]
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 32), (6, 2, 16), (4, 4, 64)])
+def test_prefill_rows_equal_library_causal_attention(Hq, Hkv, D):
+    """Whole prompt at once and a later chunk of it: library attention with a causal mask, on the source layer."""
+    L, B, n = 3, 2, 29
+    r = [0, 0, 2]
+    o = Oracle(L, r, Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=17)
+    for l in range(L):
+        for b, (p0, p1) in enumerate([(0, 29), (11, 23)]):       # sequence 0: full prompt; sequence 1: a chunk
+            pos = torch.arange(p0, p1)
+            Q = _rand_bf16((pos.numel(), Hq, D), 300 + 10 * l + b)
+            got = o.attn_rows(l, Q, torch.full_like(pos, b), pos, 0.21)
+            want = _causal_sdpa64(Q, store[r[l]][0][b], store[r[l]][1][b], pos, 0.21)
+            assert torch.allclose(got, want, rtol=1e-12, atol=1e-13)
+
+
+def test_prefill_row_at_the_last_position_is_the_decode_step():
+    """One row per sequence at pos = len-1 is Algorithm 2's decode attention."""
+    L, B, n, Hq, Hkv, D = 2, 3, 17, 4, 2, 16
+    o = Oracle(L, [0, 0], Hq, Hkv, D, B, n)
+    _fill(o, L, B, n, Hkv, D, seed=19)
+    lens = torch.tensor([17, 1, 9], dtype=torch.int32)
+    Q = _rand_bf16((B, Hq, D), 77)
+    a = o.attn_rows(1, Q, torch.arange(B), lens.to(torch.int64) - 1)
+    assert torch.equal(a, o.decode_attn(1, Q, lens))
+
+
+def test_prefill_first_token_sees_only_itself_and_rows_do_not_see_the_future():
+    L, B, n, Hq, Hkv, D = 1, 1, 12, 4, 2, 16
+    o = Oracle(L, [0], Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=23)
+    pos = torch.arange(n)
+    Q = _rand_bf16((n, Hq, D), 5)
+    out = o.attn_rows(0, Q, torch.zeros(n, dtype=torch.int64), pos)
+    assert torch.equal(out[0], store[0][1][0, 0].double().repeat_interleave(Hq // Hkv, 0))
+    # overwrite the tokens after position 5: rows 0..5 must not move, rows 6.. must
+    K2, V2 = _rand_bf16((n - 6, Hkv, D), 91), _rand_bf16((n - 6, Hkv, D), 92)
+    o.append(0, K2, V2, torch.zeros(n - 6, dtype=torch.int64), torch.arange(6, n))
+    out2 = o.attn_rows(0, Q, torch.zeros(n, dtype=torch.int64), pos)
+    assert torch.equal(out2[:6], out[:6]) and not torch.equal(out2[6:], out[6:])
+
+
+def test_prefill_brute_force_tiny():
+    """Explicit weights without max-subtraction, a handful of rows."""
+    L, B, n, Hq, Hkv, D = 2, 2, 5, 2, 1, 4
+    o = Oracle(L, [0, 0], Hq, Hkv, D, B, n)
+    store = _fill(o, L, B, n, Hkv, D, seed=29)
+    q_seq = torch.tensor([0, 1, 1, 0])
+    q_pos = torch.tensor([4, 0, 3, 2])
+    Q = _rand_bf16((4, Hq, D), 31)
+    got = o.attn_rows(1, Q, q_seq, q_pos, 0.5)
+    for i in range(4):
+        b, p = int(q_seq[i]), int(q_pos[i])
+        for h in range(Hq):
+            ws = [math.exp(0.5 * sum(float(Q[i, h, d]) * float(store[0][0][b, t, 0, d]) for d in range(D)))
+                  for t in range(p + 1)]
+            for d in range(D):
+                want = sum(w * float(store[0][1][b, t, 0, d]) for t, w in enumerate(ws)) / sum(ws)
+                assert abs(float(got[i, h, d]) - want) < 1e-12
