@@ -215,6 +215,32 @@ int skv_decode_splitk(skv_cache *cache, int layer, const void *Q, const int32_t 
 int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *workspace,
                      size_t workspace_bytes, void *stream);
 
+/* ---- pre-fill attention (Section 3.1.1 "Pre-fill") ------------------------ */
+
+/* Eq. (3.1) for the tokens of a prompt (or of a chunk of it) processed in
+ * parallel: query row i of sequence b is the token at position
+ *   pos = seq_lens[b] - q_len_b + i,   q_len_b = cu_q_lens[b+1] - cu_q_lens[b],
+ * i.e. the rows of a sequence are its LAST q_len_b cached tokens, and it attends
+ * the tokens 0..pos of the cache of layer r[layer] (a decoder is causal):
+ *   out[row,h,:] = sum_{t <= pos} softmax_t(scale * <Q[row,h,:], K[b,t,kv(h),:]>) * V[b,t,kv(h),:]
+ * The rows' own K,V must have been appended before (skv_append takes any number
+ * of tokens), so q_len_b <= seq_lens[b].  One row per sequence gives the decode
+ * step of skv_decode_attn.
+ *   Q          device bf16 [n_q][q_heads][head_dim], sequences concatenated,
+ *              n_q = cu_q_lens[batch]; 4-byte aligned
+ *   cu_q_lens  device int32 [batch+1], non-decreasing, cu_q_lens[0] = first row
+ *   page_table, seq_lens   as in skv_decode_attn
+ *   out        device bf16 [n_q][q_heads][head_dim]
+ *   max_q_len  host bound on q_len_b (sizes the grid; no host synchronisation)
+ * One launch, no workspace: a CTA owns 64 query rows (64 / (q_heads/kv_heads)
+ * tokens x the query heads of one kv head) and streams the pages they see.
+ * Errors as skv_decode_attn; a sequence with q_len_b > seq_lens[b] or
+ * q_len_b > max_q_len raises SKV_ERR_BOUNDS in the device status and its rows
+ * are left untouched. */
+int skv_prefill_attn(skv_cache *cache, int layer, const void *Q, const int32_t *cu_q_lens,
+                     const int32_t *page_table, const int32_t *seq_lens, void *out, int batch,
+                     int max_q_len, int q_heads, int pt_stride, float scale, void *stream);
+
 /* One whole decode step of Algorithm 2 with inputs already on the device:
  * for l = 0..L-1: append (owners only) then decode attention, on `stream`.
  * Because every input of the step exists when it starts, and the update of

@@ -57,6 +57,7 @@ lib.skv_gather.argtypes = [_vp, _int, _i64p, _i64, _vp, _vp, _vp]
 lib.skv_decode_workspace_bytes.argtypes = [_vp, _int, _int, _szp]
 lib.skv_decode_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_attn_static.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp]
+lib.skv_prefill_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _i32p, _vp, _int, _int, _int, _int, _f32, _vp]
 lib.skv_decode_splitk.argtypes = [_vp, _int, _vp, _i32p, _i32p, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_merge.argtypes = [_vp, _vp, _int, _int, _vp, _sz, _vp]
 lib.skv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
@@ -244,6 +245,15 @@ class SkvCache:
         rc = lib.skv_decode_attn_static(self._h, layer, _ptr(Q), _ptr(page_table), _ptr(seq_lens), _ptr(out),
                                         batch, q_heads, page_table.shape[1], scale, _stream_ptr(stream))
         _check(rc, "skv_decode_attn_static")
+
+    def skv_prefill_attn(self, layer: int, Q: torch.Tensor, cu_q_lens: torch.Tensor, page_table: torch.Tensor,
+                         seq_lens: torch.Tensor, out: torch.Tensor, max_q_len: int, scale: float = 0.0,
+                         stream=None) -> None:
+        batch, q_heads = seq_lens.shape[0], Q.shape[1]
+        rc = lib.skv_prefill_attn(self._h, layer, _ptr(Q), _ptr(cu_q_lens), _ptr(page_table), _ptr(seq_lens),
+                                  _ptr(out), batch, max_q_len, q_heads, page_table.shape[1], scale,
+                                  _stream_ptr(stream))
+        _check(rc, "skv_prefill_attn")
 
     def skv_decode_splitk(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
                           workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:

@@ -552,6 +552,44 @@ int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, c
                        batch, q_heads, pt_stride, scale, workspace, workspace_bytes, stream, batched);
 }
 
+// ---- pre-fill attention -------------------------------------------------------
+int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q_lens, const int32_t *page_table,
+                     const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
+                     float scale, void *stream)
+{
+    int rc = check_decode_args(c, layer, batch, q_heads);
+    if (rc) return rc;
+    if (!Q || !cu_q_lens || !page_table || !seq_lens || !out || pt_stride <= 0 || max_q_len <= 0) return SKV_ERR_ARG;
+    if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
+    if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
+    const int G = q_heads / c->kv_heads;
+    if (prefill_smem_bytes(c->head_dim) > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
+    PrefillParams p;
+    p.layer_base = c->layer_base(c->slot[(size_t)c->r[(size_t)layer]]);
+    p.page_stride = (int64_t)c->page_bytes;
+    p.max_pages = c->max_pages;
+    p.Q = static_cast<const uint16_t *>(Q);
+    p.out = static_cast<uint16_t *>(out);
+    p.cu_q = cu_q_lens;
+    p.page_table = page_table;
+    p.seq_lens = seq_lens;
+    p.B = batch;
+    p.Hq = q_heads;
+    p.Hkv = c->kv_heads;
+    p.pt_stride = pt_stride;
+    const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)c->head_dim);
+    p.scale_log2 = sc * 1.4426950408889634f;
+    p.status = c->status_word();
+    const int tq = prefill_tile_tokens(G);
+    const int q_tiles = (max_q_len + tq - 1) / tq;
+    if (launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SKV_ERR_CUDA;
+    }
+    c->launches += 1;
+    return SKV_OK;
+}
+
 // ---- whole decode step from host buffers -------------------------------------
 namespace {
 struct StagingLayout {

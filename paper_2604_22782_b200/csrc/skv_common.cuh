@@ -85,6 +85,20 @@ struct MergeParams {
     int max_ctas;               // grid limit (one CTA per SM)
 };
 
+struct PrefillParams {
+    const uint8_t *layer_base;  // first page of the owner layer that is read
+    int64_t page_stride;
+    int64_t max_pages;
+    const uint16_t *Q;          // [n_q][Hq][D] bf16 bits, sequences concatenated
+    uint16_t *out;              // [n_q][Hq][D] bf16 bits
+    const int32_t *cu_q;        // [B+1] first query row of every sequence
+    const int32_t *page_table;  // [B][pt_stride]
+    const int32_t *seq_lens;    // [B] cached tokens including the new ones
+    int B, Hq, Hkv, pt_stride;
+    float scale_log2;
+    int *status;
+};
+
 struct DecodeTuning {
     int variant;                // 0 auto, 1 CUDA-core (G=1), 2 tensor-core
     int warps;                  // per CTA
@@ -101,6 +115,9 @@ size_t decode_smem_bytes(int D, int B, int warps, int stages);
 cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid,
                                  int warps, int stages, bool pdl, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
+size_t prefill_smem_bytes(int D);
+int prefill_tile_tokens(int G);                 // query tokens per CTA tile
+cudaError_t launch_prefill(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
 
 // ---- worker <-> work-range arithmetic (shared by split-K and merge) --------
 // The flattened work space orders (sequence b, kv head h, page pg) b-major:

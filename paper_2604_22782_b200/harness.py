@@ -130,3 +130,18 @@ def step_tensors(dw: DeviceWorkload, device=None, pin: bool = False) -> Dict[str
     if pin and device.type == "cpu":
         t = {k: v.pin_memory() for k, v in t.items()}
     return t
+
+
+def prefill_inputs(dw: DeviceWorkload, layer: int, q_lens: torch.Tensor, device=None) -> Dict[str, torch.Tensor]:
+    """Query rows of a pre-fill call: sequence b contributes its LAST q_lens[b] tokens (positions
+    lens[b]-q_lens[b] .. lens[b]-1).  Returns Q [n_q,Hq,D] (drawn), cu_q_lens [B+1] (int32), and the rows'
+    (sequence, position) as int64 CPU tensors."""
+    w = dw.w
+    device = dw.device if device is None else device
+    q64 = q_lens.to(torch.int64)
+    q_seq, i = W.token_index(q64)
+    q_pos = (dw.lens_cpu.to(torch.int64) - q64)[q_seq] + i
+    Q = W.draw_rows(w.seed, W.KIND_Q, layer, q_seq, q_pos, w.q_heads, w.head_dim, w.q_std, device)
+    cu = torch.zeros(q64.numel() + 1, dtype=torch.int32)
+    cu[1:] = torch.cumsum(q64, 0).to(torch.int32)
+    return {"Q": Q, "cu_q_lens": cu.to(device), "q_seq": q_seq, "q_pos": q_pos}
