@@ -232,8 +232,9 @@ int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *
  *   page_table, seq_lens   as in skv_decode_attn
  *   out        device bf16 [n_q][q_heads][head_dim]
  *   max_q_len  host bound on q_len_b (sizes the grid; no host synchronisation)
- * One launch, no workspace: a CTA owns 64 query rows (64 / (q_heads/kv_heads)
- * tokens x the query heads of one kv head) and streams the pages they see.
+ * One launch, no workspace: a CTA owns 64 or 128 query rows (that many /
+ * (q_heads/kv_heads) tokens x the query heads of one kv head) and streams the
+ * pages they see (skv_set_prefill_variant).
  * Errors as skv_decode_attn; a sequence with q_len_b > seq_lens[b] or
  * q_len_b > max_q_len raises SKV_ERR_BOUNDS in the device status and its rows
  * are left untouched. */
@@ -303,6 +304,13 @@ int skv_set_decode_variant(skv_cache *cache, int variant);
  * per warp (2..8) and CTAs per SM (1..8); 0 keeps the current value.
  * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
 int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
+
+/* Pre-fill kernel variant: 0 = automatic (the tcgen05 kernel when head_dim is
+ * 128, q_heads / kv_heads divides 128 and Q, out are 16-byte aligned; else the
+ * mma.sync kernel), 1 = mma.sync kernel (64 query rows per CTA), 2 = tcgen05
+ * kernel (128 query rows per CTA, accumulators in tensor memory;
+ * SKV_ERR_UNSUPPORTED from skv_prefill_attn where it does not apply). */
+int skv_set_prefill_variant(skv_cache *cache, int variant);
 
 /* 1 (default): split-K and merge launches carry the programmatic-dependent-
  * launch attribute, so the GPU may schedule a launch while the one before it

@@ -67,6 +67,7 @@ lib.skv_decode_step_host.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _v
 lib.skv_get_status.argtypes = [_vp, _vp, ctypes.POINTER(_int)]
 lib.skv_set_decode_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
+lib.skv_set_prefill_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
@@ -304,6 +305,9 @@ class SkvCache:
 
     def skv_set_decode_tuning(self, warps_per_cta: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
         _check(lib.skv_set_decode_tuning(self._h, warps_per_cta, stages, ctas_per_sm), "skv_set_decode_tuning")
+
+    def skv_set_prefill_variant(self, variant: int) -> None:
+        _check(lib.skv_set_prefill_variant(self._h, variant), "skv_set_prefill_variant")
 
     def skv_set_decode_overlap(self, enabled: int) -> None:
         _check(lib.skv_set_decode_overlap(self._h, enabled), "skv_set_decode_overlap")

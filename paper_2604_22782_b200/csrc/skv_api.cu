@@ -23,6 +23,7 @@ struct skv_cache {
     int sm_count = 0;
     int max_smem_optin = 0;
     DecodeTuning tune{0, 2, 2, 4, 1};
+    int prefill_variant = 0;         // 0 auto (tcgen05 where supported), 1 mma.sync kernel, 2 tcgen05 kernel
     bool shape_is_default = true;    // until skv_set_decode_tuning is called: the CUDA-core kernel runs as 1 x 2 x 8
     int l2_keep_pct = 35;            // > 0: consecutive layers that read one owner walk it in opposite directions
     std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
@@ -563,7 +564,11 @@ int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q
     if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
     if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
     const int G = q_heads / c->kv_heads;
-    if (prefill_smem_bytes(c->head_dim) > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
+    const bool can_umma = prefill_umma_supported(c->head_dim, G) && aligned(Q, 16) && aligned(out, 16) &&
+                          prefill_umma_smem_bytes(c->head_dim) <= (size_t)c->max_smem_optin;
+    if (c->prefill_variant == 2 && !can_umma) return SKV_ERR_UNSUPPORTED;
+    const bool umma = c->prefill_variant == 2 || (c->prefill_variant == 0 && can_umma);
+    if (!umma && prefill_smem_bytes(c->head_dim) > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     PrefillParams p;
     p.layer_base = c->layer_base(c->slot[(size_t)c->r[(size_t)layer]]);
     p.page_stride = (int64_t)c->page_bytes;
@@ -580,9 +585,11 @@ int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q
     const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)c->head_dim);
     p.scale_log2 = sc * 1.4426950408889634f;
     p.status = c->status_word();
-    const int tq = prefill_tile_tokens(G);
+    const int tq = umma ? prefill_umma_tile_tokens(G) : prefill_tile_tokens(G);
     const int q_tiles = (max_q_len + tq - 1) / tq;
-    if (launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    const cudaError_t le = umma ? launch_prefill_umma(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream))
+                                : launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream));
+    if (le != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;
     }
@@ -748,6 +755,13 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     }
     c->tune = t;
     c->shape_is_default = false;
+    return SKV_OK;
+}
+
+int skv_set_prefill_variant(skv_cache *c, int variant)
+{
+    if (!c || variant < 0 || variant > 2) return SKV_ERR_ARG;
+    c->prefill_variant = variant;
     return SKV_OK;
 }
 

@@ -118,6 +118,11 @@ cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 size_t prefill_smem_bytes(int D);
 int prefill_tile_tokens(int G);                 // query tokens per CTA tile
 cudaError_t launch_prefill(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
+// the tcgen05 (UMMA / tensor-memory) variant
+size_t prefill_umma_smem_bytes(int D);
+bool prefill_umma_supported(int D, int G);
+int prefill_umma_tile_tokens(int G);
+cudaError_t launch_prefill_umma(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
 
 // ---- worker <-> work-range arithmetic (shared by split-K and merge) --------
 // The flattened work space orders (sequence b, kv head h, page pg) b-major:

@@ -1,0 +1,400 @@
+// Pre-fill attention on the 5th-generation tensor cores (tcgen05): the same computation as
+// skv_prefill.cu with both contractions issued as UMMA instructions and their accumulators in
+// tensor memory.
+//
+// One CTA (128 threads, 2 CTAs per SM) owns 128 query rows: 128/G tokens x the G query heads of
+// one kv head, row r = token r/G, head r%G, and thread r owns row r (= TMEM lane r).
+//   Q tile   shared memory, K-major core-matrix layout [D/8 chunks][128 rows][16 B]
+//   K, V     pages of the owner layer, 64 keys (4 pages) per stage, 2 stages, linear bulk copies;
+//            the pool's page layout IS the UMMA no-swizzle core-matrix layout: a K half is
+//            K-major [chunk][key][16 B], a V half read as the B operand of P V is MN-major
+//   S = Q K^T  TMEM columns [0,64):   per page one M128 N16 K16 instruction per 16 dims
+//   P          TMEM columns [64,96):  bf16 pairs, written by the softmax threads, A operand of P V
+//   O += P V   TMEM columns [128,128+D): per page one M128 N=D K16 instruction
+// Softmax state (running max, sum) lives in the row's thread.  O is rescaled lazily: the running
+// max used for the exponentials only moves when the true max has grown by more than 8 (in log2
+// units), so most key blocks cost no pass over O; the final division uses the same max, so the
+// result is the exact softmax.
+// Every wait is bounded; on a timeout the CTA flags the status word, lets its copies land,
+// frees its tensor memory and returns.
+#include "skv_common.cuh"
+
+#include <math.h>
+
+namespace skv {
+
+namespace {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr int ROWS = 128;
+constexpr int KB = 4;                 // pages per key block
+constexpr int NSTAGE = 2;
+constexpr int COL_S = 0, COL_P = 64, COL_O = 128;
+constexpr int TMEM_COLS = 256;
+constexpr float RESCALE_STEP = 8.f;
+
+// ---- tcgen05 wrappers ---------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, no swizzle: 8-row x 16-byte core matrices.
+//   K-major operand:  lbo = bytes between the two 16-byte halves of a K=16 step, sbo = bytes between
+//                     8-row groups along M/N
+//   MN-major operand: sbo = bytes between 8-element groups along M/N, lbo = bytes between 8-row groups along K
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
+{
+    return (1u << 4) /* D fp32 */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
+           ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128, 2) prefill_umma_kernel(PrefillParams p, int G)
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    constexpr int BLOCK = block_bytes(D), HALF = half_bytes(D), CH = D / 8;
+    constexpr int Q_BYTES = ROWS * D * 2;
+    constexpr uint32_t IDESC_QK = instr_desc(ROWS, PAGE, false), IDESC_PV = instr_desc(ROWS, D, true);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const int TQ = ROWS / G;
+
+    const uint32_t base = smem_u32(smem_raw);
+    const uint32_t pad = (128u - (base & 127u)) & 127u;
+    const uint32_t q_smem = base + pad;
+    const uint32_t ring = q_smem + Q_BYTES;
+    const uint32_t bars = ring + NSTAGE * KB * BLOCK;          // full[NSTAGE], mma_done
+    const uint32_t bar_mma = bars + 8 * NSTAGE;
+    const uint32_t slot = bar_mma + 8;
+    volatile uint32_t *slot_ptr = reinterpret_cast<volatile uint32_t *>(smem_raw + pad + Q_BYTES + NSTAGE * KB * BLOCK + 8 * NSTAGE + 8);
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) mbar_init(bars + 8 * s, 1);
+        mbar_init(bar_mma, 1);
+        fence_barrier_init();
+    }
+    pdl_wait();
+    const int q_begin = __ldg(p.cu_q + b), q_len = __ldg(p.cu_q + b + 1) - q_begin;
+    const int n_b = __ldg(p.seq_lens + b);
+    const int n_tiles = (q_len + TQ - 1) / TQ;
+    const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
+    if (blockIdx.x == 0 && tid == 0 && (q_len < 0 || q_len > n_b || n_tiles > (int)gridDim.x))
+        atomicOr(p.status, STATUS_BOUNDS);
+    if (q_len <= 0 || q_len > n_b || qt >= n_tiles) return;    // uniform over the CTA, before any allocation
+    const int q0 = qt * TQ;
+    const int q_end = (q0 + TQ < q_len) ? q0 + TQ : q_len;
+    const int pos0 = n_b - q_len;
+    const int n_keys = pos0 + q_end;
+    const int n_pages = (n_keys + PAGE - 1) / PAGE;
+    const int n_kb = (n_pages + KB - 1) / KB;
+
+    if (warp == 0) {
+        tmem_alloc(slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+
+    // copies: key block kb -> stage kb % NSTAGE (thread 0)
+    auto issue_copy = [&](int kb) {
+        const int s = kb % NSTAGE, pg0 = kb * KB;
+        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+        int ids[KB];
+#pragma unroll
+        for (int j = 0; j < KB; ++j) ids[j] = j < np ? __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + j) : 0;
+        const uint32_t bar = bars + 8 * s;
+        mbar_expect_tx(bar, (uint32_t)(np * BLOCK));
+#pragma unroll
+        for (int j = 0; j < KB; ++j) {
+            if (j < np) {
+                int id = ids[j];
+                if (id < 0 || (int64_t)id >= p.max_pages) {
+                    atomicOr(p.status, STATUS_BOUNDS);
+                    id = 0;
+                }
+                bulk_copy_g2s(ring + (uint32_t)((s * KB + j) * BLOCK),
+                              p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK, BLOCK, bar);
+            }
+        }
+    };
+    int copies = 0;
+    if (tid == 0)
+        for (; copies < NSTAGE && copies < n_kb; ++copies) issue_copy(copies);
+
+    // this thread's row: Q into shared memory in core-matrix layout (rows outside the tile are zero)
+    const int qi = tid / G, g = tid - qi * G;
+    const bool row_ok = q0 + qi < q_end;
+    const int pos = row_ok ? pos0 + q0 + qi : 0x7FFFFFFF;
+    const int64_t row_off = ((int64_t)(q_begin + q0 + qi) * p.Hq + (int64_t)h * G + g) * D;
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + row_off);
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const uint4 v = row_ok ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(q_smem + (uint32_t)(c * ROWS * 16 + tid * 16)),
+                         "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+    }
+    fence_proxy_async();               // the tensor core reads Q through the async proxy
+    tc_fence_before();
+    __syncthreads();                   // Q tile complete, TMEM address published
+    tc_fence_after();
+    const uint32_t tmem = *slot_ptr;
+    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's 32 lanes
+
+    // S(kb) = Q K^T: per present page, D/16 instructions of K=16 (thread 0)
+    auto issue_qk = [&](int kb) {
+        const int s = kb % NSTAGE, pg0 = kb * KB;
+        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+        for (int j = 0; j < np; ++j) {
+            const uint32_t k_page = ring + (uint32_t)((s * KB + j) * BLOCK);
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint64_t a = smem_desc(q_smem + (uint32_t)(ks * 2 * ROWS * 16), ROWS * 16, 128);
+                const uint64_t bd = smem_desc(k_page + (uint32_t)(ks * 2 * PAGE * 16), PAGE * 16, 128);
+                umma_ss(tmem + COL_S + PAGE * j, a, bd, IDESC_QK, ks > 0);
+            }
+        }
+        tc_commit(bar_mma);
+    };
+    // O += P V: per present page one instruction of K=16 keys (thread 0)
+    auto issue_pv = [&](int kb) {
+        const int s = kb % NSTAGE, pg0 = kb * KB;
+        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+        for (int j = 0; j < np; ++j) {
+            const uint32_t v_page = ring + (uint32_t)((s * KB + j) * BLOCK) + HALF;
+            const uint64_t bd = smem_desc(v_page, 128, PAGE * 16);
+            umma_ts(tmem + COL_O, tmem + COL_P + 8 * j, bd, IDESC_PV, (kb > 0 || j > 0) ? 1u : 0u);
+        }
+    };
+
+    bool failed = false;
+    // first key block's scores
+    if (tid == 0) {
+        const bool ok = mbar_wait_bounded(bars, 0);
+        if (ok) { tc_fence_after(); issue_qk(0); }
+        else atomicOr(p.status, STATUS_TIMEOUT);
+    }
+
+    float m_used = -INFINITY, l_sum = 0.f;
+    for (int kb = 0; kb < n_kb; ++kb) {
+        const int s = kb % NSTAGE, pg0 = kb * KB;
+        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+        // S(kb) is complete, and with it every instruction issued before it: P V of block kb-1
+        const bool ok = mbar_wait_bounded(bar_mma, (uint32_t)(kb & 1));
+        if (__syncthreads_or(!ok)) {
+            if (tid == 0) atomicOr(p.status, STATUS_TIMEOUT);
+            failed = true;
+            break;
+        }
+        tc_fence_after();
+        // the stage of block kb-1 is free again
+        if (tid == 0 && kb >= 1 && copies < n_kb) issue_copy(copies++);
+        // slots of the sequence's last page that were never written may hold anything: zero their V rows
+        const int last_valid = n_b - (pg0 + np - 1) * PAGE;
+        if (last_valid < PAGE) {
+            const uint32_t sV = ring + (uint32_t)((s * KB + np - 1) * BLOCK) + HALF;
+            for (int i = tid; i < CH * PAGE; i += ROWS)
+                if ((i & (PAGE - 1)) >= last_valid)
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(sV + (uint32_t)(i * 16)), "r"(0u) : "memory");
+            fence_proxy_async();
+        }
+        // this row's 64 scores
+        uint32_t raw[2][32];
+        tmem_ld32(lane_base + COL_S, raw[0]);
+        tmem_ld32(lane_base + COL_S + 32, raw[1]);
+        tmem_wait_ld();
+        const int t_base = pg0 * PAGE;
+        const int n_there = np * PAGE;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const int col = hh * 32 + c;
+                const float v = (col < n_there && t_base + col <= pos) ? __uint_as_float(raw[hh][c]) * p.scale_log2 : -INFINITY;
+                raw[hh][c] = __float_as_uint(v);
+                mx = fmaxf(mx, v);
+            }
+        // lazy rescaling: move the reference max only when the true max has run away from it
+        float alpha = 1.f;
+        const bool move = mx > m_used + RESCALE_STEP;          // also true for the first block with a visible key
+        if (move) {
+            alpha = fast_exp2(m_used - mx);                    // 0 when m_used = -inf
+            m_used = mx;
+        }
+        if (kb > 0 && __any_sync(FULL, move)) {                // O of blocks 0..kb-1 is complete (see the wait above)
+#pragma unroll
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+                uint32_t ov[32];
+                tmem_ld32(lane_base + COL_O + 32 * q4, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                tmem_st32(lane_base + COL_O + 32 * q4, ov);
+            }
+        }
+        l_sum *= alpha;
+        uint32_t pk[32];
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const int hh = c >> 4, cc = (2 * c) & 31;
+            const float p0 = fast_exp2(__uint_as_float(raw[hh][cc]) - m_used);
+            const float p1 = fast_exp2(__uint_as_float(raw[hh][cc + 1]) - m_used);
+            sum += p0 + p1;
+            pk[c] = pack_bf16x2(p0, p1);
+        }
+        l_sum += sum;
+        tmem_st32(lane_base + COL_P, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncthreads();               // every row's P (and rescaled O) is in tensor memory; V rows zeroed
+        if (tid == 0) {
+            tc_fence_after();
+            issue_pv(kb);
+            if (kb + 1 < n_kb) {
+                const int s1 = (kb + 1) % NSTAGE;
+                const bool ok1 = mbar_wait_bounded(bars + 8 * s1, (uint32_t)(((kb + 1) / NSTAGE) & 1));
+                if (ok1) issue_qk(kb + 1);                      // its commit also covers P V of block kb
+                else { atomicOr(p.status, STATUS_TIMEOUT); tc_commit(bar_mma); }
+            } else {
+                tc_commit(bar_mma);
+            }
+        }
+    }
+    if (!failed) {
+        const bool ok = mbar_wait_bounded(bar_mma, (uint32_t)(n_kb & 1));   // the last P V
+        if (__syncthreads_or(!ok)) {
+            if (tid == 0) atomicOr(p.status, STATUS_TIMEOUT);
+            failed = true;
+        }
+    }
+    if (!failed) {
+        tc_fence_after();
+        pdl_trigger();
+        const float inv = 1.f / l_sum;
+        uint16_t *dst = p.out + row_off;
+#pragma unroll
+        for (int q4 = 0; q4 < D / 32; ++q4) {
+            uint32_t ov[32];
+            tmem_ld32(lane_base + COL_O + 32 * q4, ov);
+            tmem_wait_ld();
+            if (row_ok) {
+#pragma unroll
+                for (int c = 0; c < 32; c += 8) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                    w.y = pack_bf16x2(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                    w.z = pack_bf16x2(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                    w.w = pack_bf16x2(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(dst + 32 * q4 + c) = w;
+                }
+            }
+        }
+    } else if (tid == 0) {
+        // let copies that are still in flight land before the shared memory goes away (bounded)
+        for (int kb = 0; kb < copies; ++kb) mbar_wait_bounded(bars + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+}  // namespace
+
+size_t prefill_umma_smem_bytes(int D)
+{
+    if (D != 128) return 0;
+    return 128 + (size_t)ROWS * D * 2 + (size_t)NSTAGE * KB * block_bytes(D) + 8 * NSTAGE + 8 + 16;
+}
+
+bool prefill_umma_supported(int D, int G) { return D == 128 && G >= 1 && G <= 8 && ROWS % G == 0; }
+
+int prefill_umma_tile_tokens(int G) { return ROWS / G; }
+
+cudaError_t launch_prefill_umma(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s)
+{
+    const size_t smem = prefill_umma_smem_bytes(D);
+    if (smem == 0 || q_tiles <= 0 || !prefill_umma_supported(D, G)) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)q_tiles, (unsigned)p.Hkv, (unsigned)p.B);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaError_t e = cudaFuncSetAttribute(prefill_umma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, prefill_umma_kernel<128>, p, G);
+}
+
+}  // namespace skv

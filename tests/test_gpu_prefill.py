@@ -10,9 +10,10 @@ pytestmark = pytest.mark.gpu
 ATOL, RTOL = 1e-2, 1e-2
 
 
-def _setup(w, lens, poison=False):
+def _setup(w, lens, poison=False, variant=0):
     from paper_2604_22782_b200 import harness
     dw = harness.setup(w, lens=lens)
+    dw.cache.skv_set_prefill_variant(variant)
     if poison:
         dw.cache.pool[256:].view(torch.int16).fill_(0x7FC1)
     harness.prefill(dw, upto_offset=0)               # every token of every owner layer is cached
@@ -48,12 +49,13 @@ def _check(o, layer, inp, out, rows=None, scale=None):
     return err.max().item()
 
 
-@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 64), (4, 2, 64), (2, 1, 128)])
-def test_whole_prompts_ragged(Hq, Hkv, D):
+@pytest.mark.parametrize("variant", [1, 0])       # the mma.sync kernel; automatic (tcgen05 kernel where it applies)
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 64), (4, 2, 64), (2, 1, 128), (6, 2, 128)])
+def test_whole_prompts_ragged(Hq, Hkv, D, variant):
     """Every token of every sequence is a query (q_len = seq_len): lengths around page and tile edges."""
     lens = torch.tensor([1, 15, 16, 17, 63, 64, 65, 100, 257, 700], dtype=torch.int32)
     w = W.Workload("pf", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=61)
-    harness, dw = _setup(w, lens)
+    harness, dw = _setup(w, lens, variant=variant)
     o = _oracle(dw, range(3))
     for layer in range(3):
         inp, out = _run(harness, dw, layer, lens)
@@ -62,12 +64,13 @@ def test_whole_prompts_ragged(Hq, Hkv, D):
     assert dw.cache.skv_get_status() == 0
 
 
-def test_chunks_of_a_prompt_and_single_rows():
+@pytest.mark.parametrize("variant", [1, 2])
+def test_chunks_of_a_prompt_and_single_rows(variant):
     """Chunked pre-fill (the last q_len tokens only), sequences with no query at all, and one row per
     sequence, which must agree with the decode step's entry point."""
     lens = torch.tensor([900, 33, 128, 2049, 5, 300], dtype=torch.int32)
     w = W.Workload("pf_chunk", 2, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=67)
-    harness, dw = _setup(w, lens, poison=True)
+    harness, dw = _setup(w, lens, poison=True, variant=variant)
     o = _oracle(dw, [1])
     for q_lens in ([100, 33, 0, 513, 1, 17], [1, 1, 1, 1, 1, 1], [0, 0, 128, 0, 5, 0]):
         ql = torch.tensor(q_lens, dtype=torch.int32)
@@ -84,11 +87,12 @@ def test_chunks_of_a_prompt_and_single_rows():
     assert dw.cache.skv_get_status() == 0
 
 
-def test_explicit_scale_and_bad_lengths():
+@pytest.mark.parametrize("variant", [1, 2])
+def test_explicit_scale_and_bad_lengths(variant):
     from paper_2604_22782_b200.binding import SKV_ERR_BOUNDS
     lens = torch.tensor([70, 40], dtype=torch.int32)
     w = W.Workload("pf_scale", 1, 4, 2, 128, 16, 2, 0, 0, "explicit", explicit_r=(0,), seed=71)
-    harness, dw = _setup(w, lens)
+    harness, dw = _setup(w, lens, variant=variant)
     o = _oracle(dw, [0])
     inp, out = _run(harness, dw, 0, lens, scale=0.05)
     _check(o, 0, inp, out, scale=0.05)
@@ -102,13 +106,14 @@ def test_explicit_scale_and_bad_lengths():
     assert bool((out[:80] == 7.0).all())
 
 
-def test_llama3_8b_shape_prompts_sampled_rows():
+@pytest.mark.parametrize("variant", [1, 2])
+def test_llama3_8b_shape_prompts_sampled_rows(variant):
     """Llama-3-8B head shape, 4 prompts of 1024..4096 tokens in layer 1 (reads layer 0): sampled rows
     (first, last, tile edges, seeded picks of every sequence) against the oracle; all rows finite and bounded."""
     w0 = W.get_workload("llama3_8b")
     w = W.Workload("pf_l3", 2, w0.q_heads, w0.kv_heads, w0.head_dim, 16, 4, 1024, 4096, "groups", group=2, seed=73)
     lens = W.seq_lens(w)
-    harness, dw = _setup(w, lens)
+    harness, dw = _setup(w, lens, variant=variant)
     inp, out = _run(harness, dw, 1, lens)
     assert dw.cache.skv_get_status() == 0
     from oracle import Oracle
@@ -125,3 +130,14 @@ def test_llama3_8b_shape_prompts_sampled_rows():
     _check(o, 1, inp, out, rows=torch.tensor(rows))
     f = out.float()
     assert torch.isfinite(f).all() and f.abs().max().item() <= 5.0
+
+
+def test_tcgen05_variant_is_refused_where_it_does_not_apply():
+    from paper_2604_22782_b200.binding import SKV_ERR_UNSUPPORTED, SkvError
+    lens = torch.tensor([20], dtype=torch.int32)
+    w = W.Workload("pf_no", 1, 6, 2, 64, 16, 1, 0, 0, "explicit", explicit_r=(0,), seed=79)     # head_dim 64, G = 3
+    harness, dw = _setup(w, lens, variant=2)
+    inp = harness.prefill_inputs(dw, 0, lens)
+    with pytest.raises(SkvError) as e:
+        dw.cache.skv_prefill_attn(0, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, torch.empty_like(inp["Q"]), 20)
+    assert e.value.status == SKV_ERR_UNSUPPORTED
