@@ -2,21 +2,29 @@
 // skv_prefill.cu with both contractions issued as UMMA instructions and their accumulators in
 // tensor memory.
 //
-// One CTA (128 threads, 2 CTAs per SM) owns 128 query rows: 128/G tokens x the G query heads of
-// one kv head, row r = token r/G, head r%G, and thread r owns row r (= TMEM lane r).
-//   Q tile   shared memory, K-major core-matrix layout [D/8 chunks][128 rows][16 B]
-//   K, V     pages of the owner layer, 64 keys (4 pages) per stage, 2 stages, linear bulk copies;
-//            the pool's page layout IS the UMMA no-swizzle core-matrix layout: a K half is
-//            K-major [chunk][key][16 B], a V half read as the B operand of P V is MN-major
-//   S = Q K^T  TMEM columns [0,64):   per page one M128 N16 K16 instruction per 16 dims
-//   P          TMEM columns [64,96):  bf16 pairs, written by the softmax threads, A operand of P V
-//   O += P V   TMEM columns [128,128+D): per page one M128 N=D K16 instruction
-// Softmax state (running max, sum) lives in the row's thread.  O is rescaled lazily: the running
-// max used for the exponentials only moves when the true max has grown by more than 8 (in log2
-// units), so most key blocks cost no pass over O; the final division uses the same max, so the
-// result is the exact softmax.
-// Every wait is bounded; on a timeout the CTA flags the status word, lets its copies land,
-// frees its tensor memory and returns.
+// One CTA (2 per SM) owns 128 query rows: 128/G tokens x the G query heads of one kv head, row
+// r = token r/G, head r%G.  Five warps:
+//   warps 0-3  softmax: thread r owns row r (= TMEM lane r)
+//   warp 4     all lanes issue the bulk copies, lane 0 issues the UMMA instructions
+// Shared memory
+//   Q tile   K-major core-matrix layout [D/8 chunks][128 rows][16 B]
+//   K ring   2 stages of 64 keys, [D/8 chunks][64 keys][16 B]: a page's K half is
+//            [chunk][16 keys][16 B]; warp 4 moves it with 16-byte cp.async copies that interleave
+//            the four pages of a stage by chunk, which makes the 64 keys ONE N=64 operand
+//   V ring   2 stages of 4 pages, each page's V half copied as it is (4 KB): read as the B operand
+//            of P V it is the MN-major core-matrix layout
+// Tensor memory (256 columns)
+//   [0,64), [64,128)   two score buffers: S = Q K^T of a key block (fp32), overwritten in place by
+//                      its P (bf16 pairs, 32 columns), the A operand of P V
+//   [128,128+D)        O += P V
+// Per key block kb: Q K^T(kb+1) is issued before the softmax of block kb has finished, so the
+// tensor core works on the next scores (and on P V of the block before) while the softmax warps
+// are busy.  Softmax state (running max, sum) lives in the row's thread.  O is rescaled lazily:
+// the max used for the exponentials only moves when the true max has grown by more than 8 (in
+// log2 units), so most key blocks cost no pass over O; the final division uses the same max, so
+// the result is the exact softmax.
+// Every wait is bounded; on a timeout the warp flags the status word and goes to the common exit,
+// where copies are given time to land and the tensor memory is freed.
 #include "skv_common.cuh"
 
 #include <math.h>
@@ -28,8 +36,9 @@ namespace {
 constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr int ROWS = 128;
 constexpr int KB = 4;                 // pages per key block
+constexpr int KEYS = KB * PAGE;       // 64
 constexpr int NSTAGE = 2;
-constexpr int COL_S = 0, COL_P = 64, COL_O = 128;
+constexpr int COL_O = 128;            // score buffers at columns 0 and 64
 constexpr int TMEM_COLS = 256;
 constexpr float RESCALE_STEP = 8.f;
 
@@ -115,29 +124,40 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
            ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+constexpr int THREADS = 160;
+
 template <int D>
-__global__ void __launch_bounds__(128, 2) prefill_umma_kernel(PrefillParams p, int G)
+__global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams p, int G)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = block_bytes(D), HALF = half_bytes(D), CH = D / 8;
     constexpr int Q_BYTES = ROWS * D * 2;
-    constexpr uint32_t IDESC_QK = instr_desc(ROWS, PAGE, false), IDESC_PV = instr_desc(ROWS, D, true);
-    const int tid = threadIdx.x, warp = tid >> 5;
+    constexpr int K_STAGE = KEYS * D * 2, V_STAGE = KB * HALF;
+    constexpr uint32_t IDESC_QK = instr_desc(ROWS, KEYS, false), IDESC_PV = instr_desc(ROWS, D, true);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.z, h = blockIdx.y;
     const int TQ = ROWS / G;
 
     const uint32_t base = smem_u32(smem_raw);
     const uint32_t pad = (128u - (base & 127u)) & 127u;
     const uint32_t q_smem = base + pad;
-    const uint32_t ring = q_smem + Q_BYTES;
-    const uint32_t bars = ring + NSTAGE * KB * BLOCK;          // full[NSTAGE], mma_done
-    const uint32_t bar_mma = bars + 8 * NSTAGE;
-    const uint32_t slot = bar_mma + 8;
-    volatile uint32_t *slot_ptr = reinterpret_cast<volatile uint32_t *>(smem_raw + pad + Q_BYTES + NSTAGE * KB * BLOCK + 8 * NSTAGE + 8);
+    const uint32_t k_ring = q_smem + Q_BYTES;
+    const uint32_t v_ring = k_ring + NSTAGE * K_STAGE;
+    const uint32_t bars = v_ring + NSTAGE * V_STAGE;
+    const uint32_t full_v = bars + 16, s_ready = bars + 32, p_ready = bars + 48, o_done = bars + 64;
+    const uint32_t slot = bars + 72;
+    volatile uint32_t *slot_ptr =
+        reinterpret_cast<volatile uint32_t *>(smem_raw + pad + Q_BYTES + NSTAGE * K_STAGE + NSTAGE * V_STAGE + 72);
+    volatile uint32_t *gave_up = slot_ptr + 1;     // set by a warp whose wait ran out
 
     if (tid == 0) {
-        for (int s = 0; s < NSTAGE; ++s) mbar_init(bars + 8 * s, 1);
-        mbar_init(bar_mma, 1);
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(full_v + 8 * s, 1);
+            mbar_init(s_ready + 8 * s, 1);
+            mbar_init(p_ready + 8 * s, ROWS);
+        }
+        mbar_init(o_done, 1);
+        *gave_up = 0;
         fence_barrier_init();
     }
     pdl_wait();
@@ -155,43 +175,62 @@ __global__ void __launch_bounds__(128, 2) prefill_umma_kernel(PrefillParams p, i
     const int n_pages = (n_keys + PAGE - 1) / PAGE;
     const int n_kb = (n_pages + KB - 1) / KB;
 
-    if (warp == 0) {
+    if (warp == 4) {
         tmem_alloc(slot, TMEM_COLS);
         tmem_relinquish();
     }
 
-    // copies: key block kb -> stage kb % NSTAGE (thread 0)
-    auto issue_copy = [&](int kb) {
+    // ---- copies (warp 4, all lanes) ----
+    // K of key block kb: 16-byte asynchronous copies, the four pages interleaved by chunk; completion is
+    // awaited by the issuing lanes themselves (cp.async groups), one group per block
+    auto copy_k = [&](int kb) {
         const int s = kb % NSTAGE, pg0 = kb * KB;
         const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
-        int ids[KB];
+        for (int j = 0; j < np; ++j) {
+            int id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + j);
+            if (id < 0 || (int64_t)id >= p.max_pages) {
+                if (lane == 0) atomicOr(p.status, STATUS_BOUNDS);
+                id = 0;
+            }
+            const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK;
+            const uint32_t dst = k_ring + (uint32_t)(s * K_STAGE + j * PAGE * 16);
 #pragma unroll
-        for (int j = 0; j < KB; ++j) ids[j] = j < np ? __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + j) : 0;
-        const uint32_t bar = bars + 8 * s;
-        mbar_expect_tx(bar, (uint32_t)(np * BLOCK));
-#pragma unroll
-        for (int j = 0; j < KB; ++j) {
-            if (j < np) {
-                int id = ids[j];
-                if (id < 0 || (int64_t)id >= p.max_pages) {
-                    atomicOr(p.status, STATUS_BOUNDS);
-                    id = 0;
-                }
-                bulk_copy_g2s(ring + (uint32_t)((s * KB + j) * BLOCK),
-                              p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK, BLOCK, bar);
+            for (int i = lane; i < CH * PAGE; i += 32) {          // piece i = (chunk i / 16, key i % 16)
+                const uint32_t d = dst + (uint32_t)((i / PAGE) * KEYS * 16 + (i % PAGE) * 16);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + i * 16) : "memory");
             }
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    int copies = 0;
-    if (tid == 0)
-        for (; copies < NSTAGE && copies < n_kb; ++copies) issue_copy(copies);
+    // V of key block kb: one 4 KB copy per page
+    auto copy_v = [&](int kb) {
+        const int s = kb % NSTAGE, pg0 = kb * KB;
+        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+        const uint32_t bar = full_v + 8 * s;
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(np * HALF));
+        __syncwarp();
+        if (lane < np) {
+            int id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + lane);
+            if (id < 0 || (int64_t)id >= p.max_pages) {
+                atomicOr(p.status, STATUS_BOUNDS);
+                id = 0;
+            }
+            bulk_copy_g2s(v_ring + (uint32_t)(s * V_STAGE + lane * HALF),
+                          p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK + HALF, HALF, bar);
+        }
+    };
+    int k_copies = 0, v_copies = 0;                // blocks whose copies have been issued (warp 4)
+    if (warp == 4) {
+        for (; k_copies < NSTAGE && k_copies < n_kb; ++k_copies) copy_k(k_copies);
+        copy_v(v_copies++);
+    }
 
-    // this thread's row: Q into shared memory in core-matrix layout (rows outside the tile are zero)
+    // ---- this thread's row (softmax warps): Q into shared memory in core-matrix layout ----
     const int qi = tid / G, g = tid - qi * G;
-    const bool row_ok = q0 + qi < q_end;
+    const bool row_ok = warp < 4 && q0 + qi < q_end;
     const int pos = row_ok ? pos0 + q0 + qi : 0x7FFFFFFF;
     const int64_t row_off = ((int64_t)(q_begin + q0 + qi) * p.Hq + (int64_t)h * G + g) * D;
-    {
+    if (warp < 4) {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + row_off);
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
@@ -199,171 +238,195 @@ __global__ void __launch_bounds__(128, 2) prefill_umma_kernel(PrefillParams p, i
             asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(q_smem + (uint32_t)(c * ROWS * 16 + tid * 16)),
                          "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
         }
+        fence_proxy_async();           // the tensor core reads Q through the async proxy
     }
-    fence_proxy_async();               // the tensor core reads Q through the async proxy
     tc_fence_before();
     __syncthreads();                   // Q tile complete, TMEM address published
     tc_fence_after();
     const uint32_t tmem = *slot_ptr;
-    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's 32 lanes
 
-    // S(kb) = Q K^T: per present page, D/16 instructions of K=16 (thread 0)
-    auto issue_qk = [&](int kb) {
-        const int s = kb % NSTAGE, pg0 = kb * KB;
-        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
-        for (int j = 0; j < np; ++j) {
-            const uint32_t k_page = ring + (uint32_t)((s * KB + j) * BLOCK);
+    if (warp == 4) {
+        // =================== copy + MMA warp ===================
+        bool ok = true;
+        // S(kb) = Q K^T: D/16 instructions M128 N64 K16 into score buffer kb % 2 (lane 0)
+        auto issue_qk = [&](int kb) {
+            const int s = kb % NSTAGE;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 const uint64_t a = smem_desc(q_smem + (uint32_t)(ks * 2 * ROWS * 16), ROWS * 16, 128);
-                const uint64_t bd = smem_desc(k_page + (uint32_t)(ks * 2 * PAGE * 16), PAGE * 16, 128);
-                umma_ss(tmem + COL_S + PAGE * j, a, bd, IDESC_QK, ks > 0);
+                const uint64_t bd = smem_desc(k_ring + (uint32_t)(s * K_STAGE + ks * 2 * KEYS * 16), KEYS * 16, 128);
+                umma_ss(tmem + (uint32_t)(s * KEYS), a, bd, IDESC_QK, ks > 0);
             }
+            tc_commit(s_ready + 8 * s);
+        };
+        // O += P V: one instruction M128 N=D K16 per present page (lane 0)
+        auto issue_pv = [&](int kb) {
+            const int s = kb % NSTAGE, pg0 = kb * KB;
+            const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+            for (int j = 0; j < np; ++j) {
+                const uint64_t bd = smem_desc(v_ring + (uint32_t)(s * V_STAGE + j * HALF), 128, PAGE * 16);
+                umma_ts(tmem + COL_O, tmem + (uint32_t)(s * KEYS + 8 * j), bd, IDESC_PV, (kb > 0 || j > 0) ? 1u : 0u);
+            }
+            tc_commit(o_done);
+        };
+        // K(0) has landed (K(1) may still be on its way): make it visible to the tensor core's proxy
+        if (n_kb > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) issue_qk(0);
+        for (int kb = 0; ok && kb < n_kb; ++kb) {
+            // P V of block kb-1 complete: its V stage, the K stage of block kb (Q K^T(kb) was issued before
+            // it) and the score buffer of block kb+1 are free
+            if (kb >= 1) {
+                if (lane == 0) ok = mbar_wait_bounded(o_done, (uint32_t)((kb - 1) & 1));
+                ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                if (v_copies < n_kb) copy_v(v_copies++);          // V(kb+1) -> stage of block kb-1
+            } else if (v_copies < n_kb) {
+                copy_v(v_copies++);                               // V(1): its stage has not been used yet
+            }
+            if (kb + 1 < n_kb) {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");      // K(kb+1), issued one block ago
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) { tc_fence_after(); issue_qk(kb + 1); }
+            }
+            if (lane == 0) {
+                ok = mbar_wait_bounded(p_ready + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1)) &&
+                     mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
+                if (ok) { tc_fence_after(); issue_pv(kb); }
+            }
+            ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            // Q K^T(kb) has been consumed by the softmax warps (p_ready): its K stage takes block kb+2
+            if (k_copies < n_kb) copy_k(k_copies++);
         }
-        tc_commit(bar_mma);
-    };
-    // O += P V: per present page one instruction of K=16 keys (thread 0)
-    auto issue_pv = [&](int kb) {
-        const int s = kb % NSTAGE, pg0 = kb * KB;
-        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
-        for (int j = 0; j < np; ++j) {
-            const uint32_t v_page = ring + (uint32_t)((s * KB + j) * BLOCK) + HALF;
-            const uint64_t bd = smem_desc(v_page, 128, PAGE * 16);
-            umma_ts(tmem + COL_O, tmem + COL_P + 8 * j, bd, IDESC_PV, (kb > 0 || j > 0) ? 1u : 0u);
+        if (!ok && lane == 0) {
+            atomicOr(p.status, STATUS_TIMEOUT);
+            *gave_up = 1;
         }
-    };
-
-    bool failed = false;
-    // first key block's scores
-    if (tid == 0) {
-        const bool ok = mbar_wait_bounded(bars, 0);
-        if (ok) { tc_fence_after(); issue_qk(0); }
-        else atomicOr(p.status, STATUS_TIMEOUT);
-    }
-
-    float m_used = -INFINITY, l_sum = 0.f;
-    for (int kb = 0; kb < n_kb; ++kb) {
-        const int s = kb % NSTAGE, pg0 = kb * KB;
-        const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
-        // S(kb) is complete, and with it every instruction issued before it: P V of block kb-1
-        const bool ok = mbar_wait_bounded(bar_mma, (uint32_t)(kb & 1));
-        if (__syncthreads_or(!ok)) {
-            if (tid == 0) atomicOr(p.status, STATUS_TIMEOUT);
-            failed = true;
-            break;
-        }
-        tc_fence_after();
-        // the stage of block kb-1 is free again
-        if (tid == 0 && kb >= 1 && copies < n_kb) issue_copy(copies++);
-        // slots of the sequence's last page that were never written may hold anything: zero their V rows
-        const int last_valid = n_b - (pg0 + np - 1) * PAGE;
-        if (last_valid < PAGE) {
-            const uint32_t sV = ring + (uint32_t)((s * KB + np - 1) * BLOCK) + HALF;
-            for (int i = tid; i < CH * PAGE; i += ROWS)
-                if ((i & (PAGE - 1)) >= last_valid)
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(sV + (uint32_t)(i * 16)), "r"(0u) : "memory");
-            fence_proxy_async();
-        }
-        // this row's 64 scores
-        uint32_t raw[2][32];
-        tmem_ld32(lane_base + COL_S, raw[0]);
-        tmem_ld32(lane_base + COL_S + 32, raw[1]);
-        tmem_wait_ld();
-        const int t_base = pg0 * PAGE;
-        const int n_there = np * PAGE;
-        float mx = -INFINITY;
+    } else {
+        // =================== softmax warps ===================
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        float m_used = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int kb = 0; kb < n_kb; ++kb) {
+            const int s = kb % NSTAGE, pg0 = kb * KB;
+            const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+            ok = mbar_wait_bounded(s_ready + 8 * s, (uint32_t)((kb / NSTAGE) & 1));
+            if (!__all_sync(FULL, ok)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t raw[2][32];
+            tmem_ld32(lane_base + (uint32_t)(s * KEYS), raw[0]);
+            tmem_ld32(lane_base + (uint32_t)(s * KEYS + 32), raw[1]);
+            tmem_wait_ld();
+            const int t_base = pg0 * PAGE, n_there = np * PAGE;
+            float mx = -INFINITY;
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh)
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const int col = hh * 32 + c;
+                    const float v = (col < n_there && t_base + col <= pos) ? __uint_as_float(raw[hh][c]) * p.scale_log2 : -INFINITY;
+                    raw[hh][c] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+            // lazy rescaling: move the reference max only when the true max has run away from it
+            float alpha = 1.f;
+            const bool move = mx > m_used + RESCALE_STEP;      // also true for the first block with a visible key
+            if (move) {
+                alpha = fast_exp2(m_used - mx);                // 0 when m_used = -inf
+                m_used = mx;
+            }
+            if (kb > 0 && __any_sync(FULL, move)) {
+                // O must hold every block up to kb-1 before it is scaled
+                ok = mbar_wait_bounded(o_done, (uint32_t)((kb - 1) & 1));
+                if (!__all_sync(FULL, ok)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int q4 = 0; q4 < D / 32; ++q4) {
+                    uint32_t ov[32];
+                    tmem_ld32(lane_base + COL_O + 32 * q4, ov);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                    tmem_st32(lane_base + COL_O + 32 * q4, ov);
+                }
+            }
+            l_sum *= alpha;
+            uint32_t pk[32];
+            float sum = 0.f;
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-                const int col = hh * 32 + c;
-                const float v = (col < n_there && t_base + col <= pos) ? __uint_as_float(raw[hh][c]) * p.scale_log2 : -INFINITY;
-                raw[hh][c] = __float_as_uint(v);
-                mx = fmaxf(mx, v);
+                const int hh = c >> 4, cc = (2 * c) & 31;
+                const float p0 = fast_exp2(__uint_as_float(raw[hh][cc]) - m_used);
+                const float p1 = fast_exp2(__uint_as_float(raw[hh][cc + 1]) - m_used);
+                sum += p0 + p1;
+                pk[c] = pack_bf16x2(p0, p1);
             }
-        // lazy rescaling: move the reference max only when the true max has run away from it
-        float alpha = 1.f;
-        const bool move = mx > m_used + RESCALE_STEP;          // also true for the first block with a visible key
-        if (move) {
-            alpha = fast_exp2(m_used - mx);                    // 0 when m_used = -inf
-            m_used = mx;
+            l_sum += sum;
+            tmem_st32(lane_base + (uint32_t)(s * KEYS), pk);    // P over the first half of its own scores
+            // slots of the sequence's last page that were never written may hold anything: zero their V rows
+            const int last_valid = n_b - (pg0 + np - 1) * PAGE;
+            if (last_valid < PAGE) {
+                ok = mbar_wait_bounded(full_v + 8 * s, (uint32_t)((kb / NSTAGE) & 1));
+                if (!__all_sync(FULL, ok)) { ok = false; break; }
+                const uint32_t sV = v_ring + (uint32_t)(s * V_STAGE + (np - 1) * HALF);
+                for (int i = tid; i < CH * PAGE; i += ROWS)
+                    if ((i & (PAGE - 1)) >= last_valid)
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(sV + (uint32_t)(i * 16)), "r"(0u) : "memory");
+                fence_proxy_async();
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(p_ready + 8 * s) : "memory");
         }
-        if (kb > 0 && __any_sync(FULL, move)) {                // O of blocks 0..kb-1 is complete (see the wait above)
+        if (ok) {
+            ok = mbar_wait_bounded(o_done, (uint32_t)((n_kb - 1) & 1));          // the last P V
+            ok = __all_sync(FULL, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l_sum;
+            uint16_t *dst = p.out + row_off;
 #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {
                 uint32_t ov[32];
                 tmem_ld32(lane_base + COL_O + 32 * q4, ov);
                 tmem_wait_ld();
+                if (row_ok) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-                tmem_st32(lane_base + COL_O + 32 * q4, ov);
-            }
-        }
-        l_sum *= alpha;
-        uint32_t pk[32];
-        float sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const int hh = c >> 4, cc = (2 * c) & 31;
-            const float p0 = fast_exp2(__uint_as_float(raw[hh][cc]) - m_used);
-            const float p1 = fast_exp2(__uint_as_float(raw[hh][cc + 1]) - m_used);
-            sum += p0 + p1;
-            pk[c] = pack_bf16x2(p0, p1);
-        }
-        l_sum += sum;
-        tmem_st32(lane_base + COL_P, pk);
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();               // every row's P (and rescaled O) is in tensor memory; V rows zeroed
-        if (tid == 0) {
-            tc_fence_after();
-            issue_pv(kb);
-            if (kb + 1 < n_kb) {
-                const int s1 = (kb + 1) % NSTAGE;
-                const bool ok1 = mbar_wait_bounded(bars + 8 * s1, (uint32_t)(((kb + 1) / NSTAGE) & 1));
-                if (ok1) issue_qk(kb + 1);                      // its commit also covers P V of block kb
-                else { atomicOr(p.status, STATUS_TIMEOUT); tc_commit(bar_mma); }
-            } else {
-                tc_commit(bar_mma);
-            }
-        }
-    }
-    if (!failed) {
-        const bool ok = mbar_wait_bounded(bar_mma, (uint32_t)(n_kb & 1));   // the last P V
-        if (__syncthreads_or(!ok)) {
-            if (tid == 0) atomicOr(p.status, STATUS_TIMEOUT);
-            failed = true;
-        }
-    }
-    if (!failed) {
-        tc_fence_after();
-        pdl_trigger();
-        const float inv = 1.f / l_sum;
-        uint16_t *dst = p.out + row_off;
-#pragma unroll
-        for (int q4 = 0; q4 < D / 32; ++q4) {
-            uint32_t ov[32];
-            tmem_ld32(lane_base + COL_O + 32 * q4, ov);
-            tmem_wait_ld();
-            if (row_ok) {
-#pragma unroll
-                for (int c = 0; c < 32; c += 8) {
-                    uint4 w;
-                    w.x = pack_bf16x2(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
-                    w.y = pack_bf16x2(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
-                    w.z = pack_bf16x2(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
-                    w.w = pack_bf16x2(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
-                    *reinterpret_cast<uint4 *>(dst + 32 * q4 + c) = w;
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(dst + 32 * q4 + c) = w;
+                    }
                 }
             }
+        } else if (lane == 0) {
+            atomicOr(p.status, STATUS_TIMEOUT);
+            *gave_up = 1;
         }
-    } else if (tid == 0) {
-        // let copies that are still in flight land before the shared memory goes away (bounded)
-        for (int kb = 0; kb < copies; ++kb) mbar_wait_bounded(bars + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
     }
+    // ---- common exit ----
+    pdl_trigger();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+    if (warp == 4) {
+        // after a timeout the last copies issued may still be in flight: give them their (bounded) wait
+        // before the shared memory goes away
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (lane == 0 && *gave_up) {
+            for (int kb = (v_copies > NSTAGE ? v_copies - NSTAGE : 0); kb < v_copies; ++kb)
+                mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
+        }
+        __syncwarp();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
 }
 
 }  // namespace
@@ -371,7 +434,7 @@ __global__ void __launch_bounds__(128, 2) prefill_umma_kernel(PrefillParams p, i
 size_t prefill_umma_smem_bytes(int D)
 {
     if (D != 128) return 0;
-    return 128 + (size_t)ROWS * D * 2 + (size_t)NSTAGE * KB * block_bytes(D) + 8 * NSTAGE + 8 + 16;
+    return 128 + (size_t)ROWS * D * 2 + (size_t)NSTAGE * KB * block_bytes(D) + 72 + 16;
 }
 
 bool prefill_umma_supported(int D, int G) { return D == 128 && G >= 1 && G <= 8 && ROWS % G == 0; }
@@ -384,7 +447,7 @@ cudaError_t launch_prefill_umma(const PrefillParams &p, int D, int G, int q_tile
     if (smem == 0 || q_tiles <= 0 || !prefill_umma_supported(D, G)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)q_tiles, (unsigned)p.Hkv, (unsigned)p.B);
-    cfg.blockDim = dim3(128);
+    cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
