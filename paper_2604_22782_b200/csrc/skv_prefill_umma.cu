@@ -3,9 +3,10 @@
 // tensor memory.
 //
 // One CTA (2 per SM) owns 128 query rows: 128/G tokens x the G query heads of one kv head, row
-// r = token r/G, head r%G.  Five warps:
+// r = token r/G, head r%G.  Six warps:
 //   warps 0-3  softmax: thread r owns row r (= TMEM lane r)
-//   warp 4     all lanes issue the bulk copies, lane 0 issues the UMMA instructions
+//   warp 4     lane 0 issues the UMMA instructions
+//   warp 5     copies K and V of the next key blocks into the rings
 // Shared memory
 //   Q tile   K-major core-matrix layout [D/8 chunks][128 rows][16 B]
 //   K ring   2 stages of 64 keys, [D/8 chunks][64 keys][16 B]: a page's K half is
@@ -23,6 +24,10 @@
 // the max used for the exponentials only moves when the true max has grown by more than 8 (in
 // log2 units), so most key blocks cost no pass over O; the final division uses the same max, so
 // the result is the exact softmax.
+// Barriers are all per stage / per score buffer (two of each): a parity wait only means "phase k is
+// over" if the waiter knows phase k-1 of that barrier is over and phase k+1 cannot have happened,
+// and with a period of two key blocks per barrier every waiter here can show both (a single
+// barrier counting every block let a fast softmax warp pass the final wait one phase early).
 // Every wait is bounded; on a timeout the warp flags the status word and goes to the common exit,
 // where copies are given time to land and the tensor memory is freed.
 #include "skv_common.cuh"
@@ -40,7 +45,29 @@ constexpr int KEYS = KB * PAGE;       // 64
 constexpr int NSTAGE = 2;
 constexpr int COL_O = 128;            // score buffers at columns 0 and 64
 constexpr int TMEM_COLS = 256;
-constexpr float RESCALE_STEP = 8.f;
+#ifndef SKV_RESCALE_STEP
+#define SKV_RESCALE_STEP 8.f
+#endif
+constexpr float RESCALE_STEP = SKV_RESCALE_STEP;
+#ifndef SKV_EXP_EMU
+#define SKV_EXP_EMU 2                 // of every 4 exponentials, how many run on the FMA pipe instead of the MUFU
+#endif
+
+// 2^x for x <= RESCALE_STEP on the FMA and integer pipes: round x to the nearest integer i with the
+// 1.5 * 2^23 trick, a cubic for 2^(x - i) on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16
+// rounding of the probabilities), then i added into the exponent field.  The special-function unit
+// is the busiest pipe of this kernel; a share of the exponentials goes here to unload it.
+__device__ __forceinline__ float exp2_fma(float x)
+{
+    x = fmaxf(x, -125.f);                          // masked scores are -inf: they end up as 2^-125, i.e. 0 in bf16
+    const float magic = 12582912.f;
+    const float t = x + magic;
+    const float f = x - (t - magic);
+    float pl = fmaf(0.055171460f, f, 0.24261086f);
+    pl = fmaf(pl, f, 0.69326097f);
+    pl = fmaf(pl, f, 0.99992812f);
+    return __int_as_float(__float_as_int(pl) + (__float_as_int(t) << 23));
+}
 
 // ---- tcgen05 wrappers ---------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols)
@@ -124,7 +151,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
            ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-constexpr int THREADS = 160;
+constexpr int THREADS = 192;
 
 template <int D>
 __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams p, int G)
@@ -144,19 +171,20 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     const uint32_t k_ring = q_smem + Q_BYTES;
     const uint32_t v_ring = k_ring + NSTAGE * K_STAGE;
     const uint32_t bars = v_ring + NSTAGE * V_STAGE;
-    const uint32_t full_v = bars + 16, s_ready = bars + 32, p_ready = bars + 48, o_done = bars + 64;
-    const uint32_t slot = bars + 72;
+    const uint32_t full_k = bars, full_v = bars + 16, s_ready = bars + 32, p_ready = bars + 48, pv_done = bars + 64;
+    const uint32_t slot = bars + 80;
     volatile uint32_t *slot_ptr =
-        reinterpret_cast<volatile uint32_t *>(smem_raw + pad + Q_BYTES + NSTAGE * K_STAGE + NSTAGE * V_STAGE + 72);
+        reinterpret_cast<volatile uint32_t *>(smem_raw + pad + Q_BYTES + NSTAGE * K_STAGE + NSTAGE * V_STAGE + 80);
     volatile uint32_t *gave_up = slot_ptr + 1;     // set by a warp whose wait ran out
 
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(full_k + 8 * s, 1);
             mbar_init(full_v + 8 * s, 1);
             mbar_init(s_ready + 8 * s, 1);
             mbar_init(p_ready + 8 * s, ROWS);
+            mbar_init(pv_done + 8 * s, 1);
         }
-        mbar_init(o_done, 1);
         *gave_up = 0;
         fence_barrier_init();
     }
@@ -180,18 +208,25 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
         tmem_relinquish();
     }
 
-    // ---- copies (warp 4, all lanes) ----
-    // K of key block kb: 16-byte asynchronous copies, the four pages interleaved by chunk; completion is
-    // awaited by the issuing lanes themselves (cp.async groups), one group per block
-    auto copy_k = [&](int kb) {
+    // ---- copies (warp 5, all lanes).  Lane j < KB carries the id of page j of a block. ----
+    auto load_ids = [&](int kb) -> int {
+        const int pg = kb * KB + lane;
+        int id = 0;
+        if (lane < KB && pg < n_pages) {
+            id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg);
+            if (id < 0 || (int64_t)id >= p.max_pages) {
+                atomicOr(p.status, STATUS_BOUNDS);
+                id = 0;
+            }
+        }
+        return id;
+    };
+    // K of key block kb: 16-byte asynchronous copies, the four pages interleaved by chunk (one cp.async group)
+    auto copy_k = [&](int kb, int ids) {
         const int s = kb % NSTAGE, pg0 = kb * KB;
         const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
         for (int j = 0; j < np; ++j) {
-            int id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + j);
-            if (id < 0 || (int64_t)id >= p.max_pages) {
-                if (lane == 0) atomicOr(p.status, STATUS_BOUNDS);
-                id = 0;
-            }
+            const int id = __shfl_sync(FULL, ids, j);
             const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK;
             const uint32_t dst = k_ring + (uint32_t)(s * K_STAGE + j * PAGE * 16);
 #pragma unroll
@@ -202,28 +237,24 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // V of key block kb: one 4 KB copy per page
-    auto copy_v = [&](int kb) {
+    // V of key block kb: one 4 KB bulk copy per page
+    auto copy_v = [&](int kb, int ids) {
         const int s = kb % NSTAGE, pg0 = kb * KB;
         const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
         const uint32_t bar = full_v + 8 * s;
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)(np * HALF));
         __syncwarp();
-        if (lane < np) {
-            int id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + lane);
-            if (id < 0 || (int64_t)id >= p.max_pages) {
-                atomicOr(p.status, STATUS_BOUNDS);
-                id = 0;
-            }
+        if (lane < np)
             bulk_copy_g2s(v_ring + (uint32_t)(s * V_STAGE + lane * HALF),
-                          p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK + HALF, HALF, bar);
-        }
+                          p.layer_base + (int64_t)ids * p.page_stride + (int64_t)h * BLOCK + HALF, HALF, bar);
     };
-    int k_copies = 0, v_copies = 0;                // blocks whose copies have been issued (warp 4)
-    if (warp == 4) {
-        for (; k_copies < NSTAGE && k_copies < n_kb; ++k_copies) copy_k(k_copies);
-        copy_v(v_copies++);
-    }
+    // this warp's copies of K(kb) have landed: make them visible to the tensor core's proxy, tell the MMA warp
+    auto publish_k = [&](int kb) {
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_k + 8 * (kb % NSTAGE)) : "memory");
+    };
+    int v_copies = 0;                              // V blocks issued (warp 5)
 
     // ---- this thread's row (softmax warps): Q into shared memory in core-matrix layout ----
     const int qi = tid / G, g = tid - qi * G;
@@ -245,67 +276,107 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     tc_fence_after();
     const uint32_t tmem = *slot_ptr;
 
-    if (warp == 4) {
-        // =================== copy + MMA warp ===================
+    if (warp == 5) {
+        // =================== copy warp ===================
         bool ok = true;
-        // S(kb) = Q K^T: D/16 instructions M128 N64 K16 into score buffer kb % 2 (lane 0)
-        auto issue_qk = [&](int kb) {
-            const int s = kb % NSTAGE;
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint64_t a = smem_desc(q_smem + (uint32_t)(ks * 2 * ROWS * 16), ROWS * 16, 128);
-                const uint64_t bd = smem_desc(k_ring + (uint32_t)(s * K_STAGE + ks * 2 * KEYS * 16), KEYS * 16, 128);
-                umma_ss(tmem + (uint32_t)(s * KEYS), a, bd, IDESC_QK, ks > 0);
-            }
-            tc_commit(s_ready + 8 * s);
-        };
-        // O += P V: one instruction M128 N=D K16 per present page (lane 0)
-        auto issue_pv = [&](int kb) {
-            const int s = kb % NSTAGE, pg0 = kb * KB;
-            const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
-            for (int j = 0; j < np; ++j) {
-                const uint64_t bd = smem_desc(v_ring + (uint32_t)(s * V_STAGE + j * HALF), 128, PAGE * 16);
-                umma_ts(tmem + COL_O, tmem + (uint32_t)(s * KEYS + 8 * j), bd, IDESC_PV, (kb > 0 || j > 0) ? 1u : 0u);
-            }
-            tc_commit(o_done);
-        };
-        // K(0) has landed (K(1) may still be on its way): make it visible to the tensor core's proxy
-        if (n_kb > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
-        else asm volatile("cp.async.wait_group 0;" ::: "memory");
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) issue_qk(0);
-        for (int kb = 0; ok && kb < n_kb; ++kb) {
-            // P V of block kb-1 complete: its V stage, the K stage of block kb (Q K^T(kb) was issued before
-            // it) and the score buffer of block kb+1 are free
-            if (kb >= 1) {
-                if (lane == 0) ok = mbar_wait_bounded(o_done, (uint32_t)((kb - 1) & 1));
+        int ids = load_ids(0);
+        copy_v(0, ids);
+        copy_k(0, ids);
+        v_copies = 1;
+        if (n_kb > 1) {
+            ids = load_ids(1);
+            copy_v(1, ids);
+            copy_k(1, ids);
+            v_copies = 2;
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            publish_k(0);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            publish_k(1);
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            publish_k(0);
+        }
+        // page ids are fetched ahead of their use: ids_prev, ids_cur, ids_next belong to blocks kb+1, kb+2, kb+3
+        int ids_prev = ids, ids_cur = load_ids(2), ids_next = load_ids(3);
+        for (int kb = 0; kb + 1 < n_kb; ++kb) {
+            // Q K^T(kb) complete (its scores are ready): the K stage of block kb takes K(kb+2).
+            // P V of block kb-1 complete: the V stage of block kb-1 takes V(kb+1) (V(1) went out above).
+            // Each wait is on a per-stage barrier whose next completion needs the very copy issued after it,
+            // so this warp can never fall a whole phase behind.
+            const bool more_k = kb + 2 < n_kb;
+            if (more_k) {
+                if (lane == 0) ok = mbar_wait_bounded(s_ready + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
                 ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                if (v_copies < n_kb) copy_v(v_copies++);          // V(kb+1) -> stage of block kb-1
-            } else if (v_copies < n_kb) {
-                copy_v(v_copies++);                               // V(1): its stage has not been used yet
+                copy_k(kb + 2, ids_cur);
             }
-            if (kb + 1 < n_kb) {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");      // K(kb+1), issued one block ago
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) { tc_fence_after(); issue_qk(kb + 1); }
+            if (kb >= 1) {
+                if (lane == 0) ok = mbar_wait_bounded(pv_done + 8 * ((kb - 1) % NSTAGE), (uint32_t)(((kb - 1) / NSTAGE) & 1));
+                ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                copy_v(kb + 1, ids_prev);
+                v_copies = kb + 2;
             }
-            if (lane == 0) {
-                ok = mbar_wait_bounded(p_ready + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1)) &&
-                     mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
-                if (ok) { tc_fence_after(); issue_pv(kb); }
+            const int ids_new = load_ids(kb + 4);
+            if (more_k) {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                publish_k(kb + 2);
             }
-            ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
-            // Q K^T(kb) has been consumed by the softmax warps (p_ready): its K stage takes block kb+2
-            if (k_copies < n_kb) copy_k(k_copies++);
+            ids_prev = ids_cur;
+            ids_cur = ids_next;
+            ids_next = ids_new;
         }
         if (!ok && lane == 0) {
             atomicOr(p.status, STATUS_TIMEOUT);
             *gave_up = 1;
         }
+    } else if (warp == 4) {
+        // =================== MMA warp: lane 0 issues ===================
+        if (lane == 0) {
+            // S(kb) = Q K^T: D/16 instructions M128 N64 K16 into score buffer kb % 2
+            auto issue_qk = [&](int kb) {
+                const int s = kb % NSTAGE;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint64_t a = smem_desc(q_smem + (uint32_t)(ks * 2 * ROWS * 16), ROWS * 16, 128);
+                    const uint64_t bd = smem_desc(k_ring + (uint32_t)(s * K_STAGE + ks * 2 * KEYS * 16), KEYS * 16, 128);
+                    umma_ss(tmem + (uint32_t)(s * KEYS), a, bd, IDESC_QK, ks > 0);
+                }
+                tc_commit(s_ready + 8 * s);
+            };
+            // O += P V: one instruction M128 N=D K16 per present page
+            auto issue_pv = [&](int kb) {
+                const int s = kb % NSTAGE, pg0 = kb * KB;
+                const int np = (n_pages - pg0) < KB ? (n_pages - pg0) : KB;
+                for (int j = 0; j < np; ++j) {
+                    const uint64_t bd = smem_desc(v_ring + (uint32_t)(s * V_STAGE + j * HALF), 128, PAGE * 16);
+                    umma_ts(tmem + COL_O, tmem + (uint32_t)(s * KEYS + 8 * j), bd, IDESC_PV, (kb > 0 || j > 0) ? 1u : 0u);
+                }
+                tc_commit(pv_done + 8 * s);
+            };
+            bool ok = mbar_wait_bounded(full_k, 0);
+            if (ok) { tc_fence_after(); issue_qk(0); }
+            for (int kb = 0; ok && kb < n_kb; ++kb) {
+                if (kb + 1 < n_kb) {
+                    // K(kb+1) in shared memory; score buffer of block kb+1 free (P V of block kb-1 complete)
+                    ok = mbar_wait_bounded(full_k + 8 * ((kb + 1) % NSTAGE), (uint32_t)(((kb + 1) / NSTAGE) & 1));
+                    if (ok && kb >= 1) ok = mbar_wait_bounded(pv_done + 8 * ((kb - 1) % NSTAGE), (uint32_t)(((kb - 1) / NSTAGE) & 1));
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(kb + 1);
+                }
+                ok = mbar_wait_bounded(p_ready + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1)) &&
+                     mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(kb);
+            }
+            if (!ok) {
+                atomicOr(p.status, STATUS_TIMEOUT);
+                *gave_up = 1;
+            }
+        }
+        __syncwarp();
     } else {
         // =================== softmax warps ===================
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
@@ -322,16 +393,24 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
             tmem_ld32(lane_base + (uint32_t)(s * KEYS + 32), raw[1]);
             tmem_wait_ld();
             const int t_base = pg0 * PAGE, n_there = np * PAGE;
+            // causal mask (and absent pages of the last block) on the raw scores; most blocks are fully visible
             float mx = -INFINITY;
+            if (n_there == KEYS && t_base + KEYS - 1 <= pos) {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh)
+                for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const int col = hh * 32 + c;
-                    const float v = (col < n_there && t_base + col <= pos) ? __uint_as_float(raw[hh][c]) * p.scale_log2 : -INFINITY;
-                    raw[hh][c] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
-                }
+                    for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[hh][c]));
+            } else {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const int col = hh * 32 + c;
+                        if (!(col < n_there && t_base + col <= pos)) raw[hh][c] = 0xFF800000u;   // -inf
+                        mx = fmaxf(mx, __uint_as_float(raw[hh][c]));
+                    }
+            }
+            mx *= p.scale_log2;                                // the scale is positive
             // lazy rescaling: move the reference max only when the true max has run away from it
             float alpha = 1.f;
             const bool move = mx > m_used + RESCALE_STEP;      // also true for the first block with a visible key
@@ -341,7 +420,7 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
             }
             if (kb > 0 && __any_sync(FULL, move)) {
                 // O must hold every block up to kb-1 before it is scaled
-                ok = mbar_wait_bounded(o_done, (uint32_t)((kb - 1) & 1));
+                ok = mbar_wait_bounded(pv_done + 8 * ((kb - 1) % NSTAGE), (uint32_t)(((kb - 1) / NSTAGE) & 1));
                 if (!__all_sync(FULL, ok)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
@@ -357,11 +436,14 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
             l_sum *= alpha;
             uint32_t pk[32];
             float sum = 0.f;
+            const float neg_m = -m_used;
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
                 const int hh = c >> 4, cc = (2 * c) & 31;
-                const float p0 = fast_exp2(__uint_as_float(raw[hh][cc]) - m_used);
-                const float p1 = fast_exp2(__uint_as_float(raw[hh][cc + 1]) - m_used);
+                const float x0 = fmaf(__uint_as_float(raw[hh][cc]), p.scale_log2, neg_m);
+                const float x1 = fmaf(__uint_as_float(raw[hh][cc + 1]), p.scale_log2, neg_m);
+                const float p0 = ((2 * c) & 3) < SKV_EXP_EMU ? exp2_fma(x0) : fast_exp2(x0);
+                const float p1 = ((2 * c + 1) & 3) < SKV_EXP_EMU ? exp2_fma(x1) : fast_exp2(x1);
                 sum += p0 + p1;
                 pk[c] = pack_bf16x2(p0, p1);
             }
@@ -383,7 +465,8 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(p_ready + 8 * s) : "memory");
         }
         if (ok) {
-            ok = mbar_wait_bounded(o_done, (uint32_t)((n_kb - 1) & 1));          // the last P V
+            // the last P V (the phase before it on this barrier, block n_kb-3, is known to be over)
+            ok = mbar_wait_bounded(pv_done + 8 * ((n_kb - 1) % NSTAGE), (uint32_t)(((n_kb - 1) / NSTAGE) & 1));
             ok = __all_sync(FULL, ok);
         }
         if (ok) {
@@ -416,14 +499,16 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     pdl_trigger();
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 5) {
         // after a timeout the last copies issued may still be in flight: give them their (bounded) wait
         // before the shared memory goes away
         asm volatile("cp.async.wait_group 0;" ::: "memory");
-        if (lane == 0 && *gave_up) {
+        if (lane == 0 && *gave_up)
             for (int kb = (v_copies > NSTAGE ? v_copies - NSTAGE : 0); kb < v_copies; ++kb)
                 mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
-        }
+    }
+    __syncthreads();
+    if (warp == 4) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
     }
@@ -434,7 +519,7 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
 size_t prefill_umma_smem_bytes(int D)
 {
     if (D != 128) return 0;
-    return 128 + (size_t)ROWS * D * 2 + (size_t)NSTAGE * KB * block_bytes(D) + 72 + 16;
+    return 128 + (size_t)ROWS * D * 2 + (size_t)NSTAGE * KB * block_bytes(D) + 96 + 16;
 }
 
 bool prefill_umma_supported(int D, int G) { return D == 128 && G >= 1 && G <= 8 && ROWS % G == 0; }

@@ -141,3 +141,20 @@ def test_tcgen05_variant_is_refused_where_it_does_not_apply():
     with pytest.raises(SkvError) as e:
         dw.cache.skv_prefill_attn(0, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, torch.empty_like(inp["Q"]), 20)
     assert e.value.status == SKV_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 2)])
+def test_tcgen05_repeated_calls_stay_correct(Hq, Hkv):
+    """The warps of the tcgen05 kernel run far apart (softmax, tensor-core issue, copies): many calls on
+    tiles of one and two key blocks (where a warp that is a phase early shows up) must all give the
+    oracle's rows, and the same bits every time."""
+    lens = torch.tensor([1, 15, 16, 17, 63, 64, 65, 100, 257, 700], dtype=torch.int32)
+    w = W.Workload("pf_rep", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=83)
+    harness, dw = _setup(w, lens, variant=2)
+    o = _oracle(dw, [1])
+    inp, first = _run(harness, dw, 1, lens)
+    _check(o, 1, inp, first)
+    for _ in range(40):
+        _, again = _run(harness, dw, 1, lens)
+        assert torch.equal(again.view(torch.int16), first.view(torch.int16))
+    assert dw.cache.skv_get_status() == 0
