@@ -45,30 +45,7 @@ constexpr int KEYS = KB * PAGE;       // 64
 constexpr int NSTAGE = 2;
 constexpr int COL_O = 128;            // score buffers at columns 0 and 64
 constexpr int TMEM_COLS = 256;
-#ifndef SKV_RESCALE_STEP
-#define SKV_RESCALE_STEP 8.f
-#endif
-constexpr float RESCALE_STEP = SKV_RESCALE_STEP;
-#ifndef SKV_EXP_EMU
-#define SKV_EXP_EMU 2                 // of every 4 exponentials, how many run on the FMA pipe instead of the MUFU
-#endif
-
-// 2^x for x <= RESCALE_STEP on the FMA and integer pipes: round x to the nearest integer i with the
-// 1.5 * 2^23 trick, a cubic for 2^(x - i) on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16
-// rounding of the probabilities), then i added into the exponent field.  The special-function unit
-// is the busiest pipe of this kernel; a share of the exponentials goes here to unload it.
-__device__ __forceinline__ float exp2_fma(float x)
-{
-    x = fmaxf(x, -125.f);                          // masked scores are -inf: they end up as 2^-125, i.e. 0 in bf16
-    const float magic = 12582912.f;
-    const float t = x + magic;
-    const float f = x - (t - magic);
-    float pl = fmaf(0.055171460f, f, 0.24261086f);
-    pl = fmaf(pl, f, 0.69326097f);
-    pl = fmaf(pl, f, 0.99992812f);
-    return __int_as_float(__float_as_int(pl) + (__float_as_int(t) << 23));
-}
-
+constexpr float RESCALE_STEP = 8.f;
 // ---- tcgen05 wrappers ---------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols)
 {
@@ -442,8 +419,7 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
                 const int hh = c >> 4, cc = (2 * c) & 31;
                 const float x0 = fmaf(__uint_as_float(raw[hh][cc]), p.scale_log2, neg_m);
                 const float x1 = fmaf(__uint_as_float(raw[hh][cc + 1]), p.scale_log2, neg_m);
-                const float p0 = ((2 * c) & 3) < SKV_EXP_EMU ? exp2_fma(x0) : fast_exp2(x0);
-                const float p1 = ((2 * c + 1) & 3) < SKV_EXP_EMU ? exp2_fma(x1) : fast_exp2(x1);
+                const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                 sum += p0 + p1;
                 pk[c] = pack_bf16x2(p0, p1);
             }
