@@ -353,10 +353,63 @@ def main():
         del dw, cache, t, hb, staging
         torch.cuda.empty_cache()
         line["sharing_sweep"] = sharing_sweep(args, dev)
+        line["prefill"] = prefill_leg(args, dev)
     print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def prefill_leg(args, dev):
+    """Pre-fill (the phase before decoding): Llama-3-8B head shape, 8 prompts of 4096 tokens.  Times the
+    multi-token update of the owner layer and the causal attention of all prompt tokens over the routed
+    owner's pages (layer 1 reads layer 0), for the tcgen05 kernel and the mma.sync kernel.  A dense
+    contraction: the bound is the tensor core, flops = 4 * q_heads * head_dim * sum over rows of (pos + 1)."""
+    from paper_2604_22782_b200 import harness
+    B, T = 8, 4096
+    w = W.Workload("prefill_llama3_8b", 2, 32, 8, 128, 16, B, T, T, "groups", group=2, seed=1, family="Llama-3-8B")
+    lens = torch.full((B,), T, dtype=torch.int32)
+    dw = harness.setup(w, device=dev, lens=lens)
+    seq_idx, pos = W.token_index(lens)
+    slots = W.slot_map_for(dw.page_table_cpu, seq_idx, pos, w.page_size).to(dev)
+    K, V = W.draw_kv(w, 0, seq_idx, pos, device=dev)
+    n_rep = max(3, args.steps // 2)
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_rep):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / n_rep
+
+    ms_append = timed(lambda: dw.cache.skv_append(0, K, V, slots))
+    inp = harness.prefill_inputs(dw, 1, lens)
+    out = torch.empty_like(inp["Q"])
+    flops = 4.0 * w.q_heads * w.head_dim * B * (T * (T + 1) / 2)
+    res = {"workload": w.name, "batch": B, "prompt_tokens": T, "flops_per_call": flops,
+           "append_ms": ms_append, "append_gbs": 2 * K.numel() * 2 * 2 / (ms_append * 1e-3) / 1e9}
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak = float(json.load(f)["bf16_tflops"])
+            peak_kind = "measured"
+    except Exception:
+        peak, peak_kind = 1590.0, "fallback"
+    for variant, name in ((2, "tcgen05"), (1, "mma_sync")):
+        dw.cache.skv_set_prefill_variant(variant)
+        ms = timed(lambda: dw.cache.skv_prefill_attn(1, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, out, T))
+        res[name] = {"ms_per_call": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                     "tokens_per_s": B * T / (ms * 1e-3)}
+    res["roofline"] = {"bound": "tensor", "kernel": "prefill_umma_kernel", "achieved": res["tcgen05"]["tflops"],
+                       "peak": peak, "peak_kind": peak_kind, "unit": "TFLOP/s",
+                       "frac": res["tcgen05"]["tflops"] / peak}
+    if dw.cache.skv_get_status() != 0:
+        raise SystemExit("device status after the pre-fill leg")
+    return res
 
 
 def sharing_sweep(args, dev):
