@@ -24,6 +24,13 @@
  *                       the source layer's tokens 0..pos of its sequence (a
  *                       decoder is causal).  One decode step is the special case
  *                       of one row per sequence at pos = seq_len - 1.
+ *   oracle_rcla_map     Section 3.2 (R-CLA, training time): per layer and forward pass
+ *                       d ~ Bernoulli(p); d = 1 keeps the layer's own K,V, d = 0 takes
+ *                       a layer drawn uniformly from those before it.  The random
+ *                       numbers are inputs (u for the coin, v for the choice).
+ *   oracle_rdcla_map    Section 4.2 ablation (RD-CLA@k): the fixed groups of k layers,
+ *                       but each layer flips a coin between the group's first layer
+ *                       and its own K,V.
  *   oracle_mu           Eq. (3.2): owner set S -> map mu (0-based layers).
  *   oracle_group_map    Section 4.3: groups of g consecutive layers share the
  *                       first layer's cache.
@@ -241,6 +248,39 @@ int oracle_attn_rows(const oracle_t *o, int layer, const uint16_t *Q, const int6
         }
     }
     return fail ? -2 : 0;
+}
+
+/* Section 3.2, one forward pass of R-CLA training, 0-based layers: for every layer l draw
+ * d ~ Bernoulli(p_self) as (u[l] < p_self); d = 1: the layer attends its own K,V (map[l] = l);
+ * d = 0: it attends layer l' uniform on {0, .., l-1}, taken as floor(v[l] * l).  Layer 0 has no
+ * layer before it and always attends itself.  u, v in [0, 1). */
+int oracle_rcla_map(int L, double p_self, const double *u, const double *v, int32_t *map_out)
+{
+    if (L <= 0 || p_self < 0.0 || p_self > 1.0) return -1;
+    for (int l = 0; l < L; ++l) {
+        if (u[l] < 0.0 || u[l] >= 1.0 || v[l] < 0.0 || v[l] >= 1.0) return -1;
+        if (l == 0 || u[l] < p_self) {
+            map_out[l] = l;
+        } else {
+            int pick = (int)floor(v[l] * (double)l);
+            if (pick > l - 1) pick = l - 1;
+            map_out[l] = pick;
+        }
+    }
+    return 0;
+}
+
+/* Section 4.2 ablation, RD-CLA@k: groups of k consecutive layers share the first one's K,V as in
+ * CLA@k, but at each forward step each layer flips a coin: u[l] < p_self keeps its own K,V,
+ * otherwise it attends the first layer of its group. */
+int oracle_rdcla_map(int L, int k, double p_self, const double *u, int32_t *map_out)
+{
+    if (L <= 0 || k <= 0 || p_self < 0.0 || p_self > 1.0) return -1;
+    for (int l = 0; l < L; ++l) {
+        if (u[l] < 0.0 || u[l] >= 1.0) return -1;
+        map_out[l] = (u[l] < p_self) ? l : (l / k) * k;
+    }
+    return 0;
 }
 
 /* Eq. (3.2), 0-based: mu(l) = l if l in S, else the largest member of S below

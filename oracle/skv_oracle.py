@@ -45,6 +45,8 @@ def _load():
                                             ctypes.c_int64, ctypes.c_double, f64p]
         lib.oracle_decode_attn.argtypes = [vp, ctypes.c_int, u16p, i32p, ctypes.c_double, f64p]
         lib.oracle_attn_rows.argtypes = [vp, ctypes.c_int, u16p, i64p, i64p, ctypes.c_int64, ctypes.c_double, f64p]
+        lib.oracle_rcla_map.argtypes = [ctypes.c_int, ctypes.c_double, f64p, f64p, i32p]
+        lib.oracle_rdcla_map.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double, f64p, i32p]
         lib.oracle_mu.argtypes = [ctypes.c_int, i32p, ctypes.c_int, i32p]
         lib.oracle_group_map.argtypes = [ctypes.c_int, ctypes.c_int, i32p]
         lib.oracle_count_owners.argtypes = [ctypes.c_int, i32p]
@@ -69,6 +71,23 @@ def mu_from_owners(n_layers: int, owners: Sequence[int]):
     ow = _i32(owners)
     out = torch.empty(n_layers, dtype=torch.int32)
     rc = _load().oracle_mu(n_layers, ow.data_ptr(), ow.numel(), out.data_ptr())
+    return out.tolist() if rc == 0 else None
+
+
+def rcla_map(p_self: float, u: Sequence[float], v: Sequence[float]):
+    """Section 3.2: one forward pass of R-CLA training (u: coins, v: choices, both in [0,1))."""
+    uu = torch.as_tensor(list(u), dtype=torch.float64).contiguous()
+    vv = torch.as_tensor(list(v), dtype=torch.float64).contiguous()
+    out = torch.empty(uu.numel(), dtype=torch.int32)
+    rc = _load().oracle_rcla_map(uu.numel(), p_self, uu.data_ptr(), vv.data_ptr(), out.data_ptr())
+    return out.tolist() if rc == 0 else None
+
+
+def rdcla_map(k: int, p_self: float, u: Sequence[float]):
+    """Section 4.2 ablation, RD-CLA@k."""
+    uu = torch.as_tensor(list(u), dtype=torch.float64).contiguous()
+    out = torch.empty(uu.numel(), dtype=torch.int32)
+    rc = _load().oracle_rdcla_map(uu.numel(), k, p_self, uu.data_ptr(), out.data_ptr())
     return out.tolist() if rc == 0 else None
 
 

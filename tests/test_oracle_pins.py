@@ -430,3 +430,42 @@ def test_prefill_brute_force_tiny():
             for d in range(D):
                 want = sum(w * float(store[0][1][b, t, 0, d]) for t, w in enumerate(ws)) / sum(ws)
                 assert abs(float(got[i, h, d]) - want) < 1e-12
+
+
+# ------------------------------------------------------------------ training-time routing samplers (Section 3.2)
+def test_rcla_map_cases_and_distribution():
+    from oracle import rcla_map
+    # hand cases: coin below p keeps the layer; otherwise floor(v * l) picks among the l layers before it
+    assert rcla_map(0.5, [0.9, 0.9, 0.1, 0.9, 0.9], [0.0, 0.99, 0.5, 0.0, 0.999]) == [0, 0, 2, 0, 3]
+    assert rcla_map(1.0, [0.3] * 6, [0.7] * 6) == list(range(6))          # p = 1: standard self-attention
+    assert rcla_map(0.0, [0.0] * 4, [0.0, 0.0, 0.5, 0.9]) == [0, 0, 1, 2]   # p = 0: always a previous layer
+    assert rcla_map(0.5, [1.0], [0.0]) is None                             # draws must lie in [0, 1)
+    # distribution over many passes: P(self) = p for l >= 1, the choice is uniform on {0..l-1}
+    g = torch.Generator().manual_seed(3)
+    L, n, p = 9, 20000, 0.6
+    self_count = torch.zeros(L)
+    picks = torch.zeros(L, L)
+    for _ in range(n // 100):
+        U, V = torch.rand(100, L, generator=g, dtype=torch.float64), torch.rand(100, L, generator=g, dtype=torch.float64)
+        for i in range(100):
+            m = rcla_map(p, U[i].tolist(), V[i].tolist())
+            for l, s in enumerate(m):
+                assert 0 <= s <= l
+                if s == l:
+                    self_count[l] += 1
+                else:
+                    picks[l, s] += 1
+    assert self_count[0] == n
+    for l in range(1, L):
+        # self includes d = 1 only (a cross pick is always < l)
+        assert abs(self_count[l] / n - p) < 0.02
+        cross = picks[l, :l]
+        assert (cross / cross.sum() - 1.0 / l).abs().max() < 0.03
+
+
+def test_rdcla_map_mixes_the_group_leader_and_the_layer_itself():
+    from oracle import rdcla_map
+    assert rdcla_map(4, 0.5, [0.9] * 8) == group_map(8, 4)                 # every coin says "shared": CLA@4
+    assert rdcla_map(4, 0.5, [0.1] * 8) == list(range(8))                  # every coin says "own"
+    assert rdcla_map(2, 0.6, [0.7, 0.7, 0.2, 0.9, 0.59, 0.61]) == [0, 0, 2, 2, 4, 4]
+    assert rdcla_map(3, 0.6, [0.7, 0.2, 0.9, 0.2, 0.7, 0.61]) == [0, 1, 0, 3, 3, 3]
