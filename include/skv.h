@@ -77,6 +77,22 @@ int skv_routing_from_owners(int n_layers, const int32_t *owners, int n_owners, i
  * their group, r_out[l] = l - (l mod g); the last group may be short. */
 int skv_routing_groups(int n_layers, int g, int32_t *r_out);
 
+/* Section 3.2, training time: the cache source of every layer for ONE forward
+ * pass of R-CLA.  For each layer l a decision d ~ Bernoulli(p_self) is drawn as
+ * (u[l] < p_self): d = 1 keeps the layer's own K,V (map_out[l] = l), d = 0 takes
+ * layer floor(v[l] * l), i.e. uniform over the l layers before it.  Layer 0 has
+ * nothing before it and always reads itself.  The random numbers are the
+ * caller's: u, v host arrays of n_layers doubles in [0, 1) (SKV_ERR_ARG else).
+ * The map need not be a valid skv_cache_create map (a layer may read a layer
+ * that itself reads elsewhere): at training time every layer's K,V exists, see
+ * skv_prefill_attn_src. */
+int skv_routing_rcla(int n_layers, double p_self, const double *u, const double *v, int32_t *map_out);
+
+/* Section 4.2 ablation "RD-CLA@k": the fixed groups of skv_routing_groups(k),
+ * applied stochastically: u[l] < p_self keeps the layer's own K,V, otherwise the
+ * layer reads the first layer of its group. */
+int skv_routing_rdcla(int n_layers, int k, double p_self, const double *u, int32_t *map_out);
+
 /* ---- cache -------------------------------------------------------------- */
 
 /* Bytes of device memory the caller must provide for the page pool:
@@ -241,6 +257,16 @@ int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *
 int skv_prefill_attn(skv_cache *cache, int layer, const void *Q, const int32_t *cu_q_lens,
                      const int32_t *page_table, const int32_t *seq_lens, void *out, int batch,
                      int max_q_len, int q_heads, int pt_stride, float scale, void *stream);
+
+/* skv_prefill_attn with the source named by the caller instead of the routing
+ * map: the rows attend the pages of `src_layer`, which must be an owner
+ * (SKV_ERR_LAYER otherwise).  This is the routed attention of a training-time
+ * forward pass (Section 3.2): with a cache in which every layer owns its pages
+ * (identity map), layer l of a pass calls it with src_layer = map[l] from
+ * skv_routing_rcla / skv_routing_rdcla.  Forward only. */
+int skv_prefill_attn_src(skv_cache *cache, int src_layer, const void *Q, const int32_t *cu_q_lens,
+                         const int32_t *page_table, const int32_t *seq_lens, void *out, int batch,
+                         int max_q_len, int q_heads, int pt_stride, float scale, void *stream);
 
 /* One whole decode step of Algorithm 2 with inputs already on the device:
  * for l = 0..L-1: append (owners only) then decode attention, on `stream`.

@@ -7,10 +7,12 @@ this package only marshals arguments.  There is no CPU fallback: importing
 """
 from .binding import (  # noqa: F401
     SkvError, SkvCache, lib, lib_path, exported_symbols,
-    skv_routing_from_owners, skv_routing_groups, skv_cache_pool_bytes, skv_strerror,
+    skv_routing_from_owners, skv_routing_groups, skv_routing_rcla, skv_routing_rdcla, skv_cache_pool_bytes,
+    skv_strerror,
 )
 
 __all__ = [
     "SkvError", "SkvCache", "lib", "lib_path", "exported_symbols",
-    "skv_routing_from_owners", "skv_routing_groups", "skv_cache_pool_bytes", "skv_strerror",
+    "skv_routing_from_owners", "skv_routing_groups", "skv_routing_rcla", "skv_routing_rdcla",
+    "skv_cache_pool_bytes", "skv_strerror",
 ]

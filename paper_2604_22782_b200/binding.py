@@ -45,6 +45,8 @@ lib.skv_strerror.restype = ctypes.c_char_p
 lib.skv_strerror.argtypes = [_int]
 lib.skv_routing_from_owners.argtypes = [_int, _i32p, _int, _i32p]
 lib.skv_routing_groups.argtypes = [_int, _int, _i32p]
+lib.skv_routing_rcla.argtypes = [_int, ctypes.c_double, _vp, _vp, _i32p]
+lib.skv_routing_rdcla.argtypes = [_int, _int, ctypes.c_double, _vp, _i32p]
 lib.skv_cache_pool_bytes.argtypes = [_int, _i32p, _int, _int, _int, _i64, _szp]
 lib.skv_cache_create.argtypes = [ctypes.POINTER(_vp), _int, _i32p, _int, _int, _int, _i64, _vp, _sz, _vp]
 lib.skv_cache_destroy.restype = None
@@ -58,6 +60,7 @@ lib.skv_decode_workspace_bytes.argtypes = [_vp, _int, _int, _szp]
 lib.skv_decode_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_attn_static.argtypes = [_vp, _int, _vp, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp]
 lib.skv_prefill_attn.argtypes = [_vp, _int, _vp, _i32p, _i32p, _i32p, _vp, _int, _int, _int, _int, _f32, _vp]
+lib.skv_prefill_attn_src.argtypes = [_vp, _int, _vp, _i32p, _i32p, _i32p, _vp, _int, _int, _int, _int, _f32, _vp]
 lib.skv_decode_splitk.argtypes = [_vp, _int, _vp, _i32p, _i32p, _int, _int, _int, _f32, _vp, _sz, _vp]
 lib.skv_decode_merge.argtypes = [_vp, _vp, _int, _int, _vp, _sz, _vp]
 lib.skv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _i64p, _i32p, _i32p, _vp, _int, _int, _int, _f32, _vp, _sz, _vp]
@@ -114,6 +117,24 @@ def skv_routing_groups(n_layers: int, g: int) -> List[int]:
     out = (ctypes.c_int32 * max(n_layers, 1))()
     _check(lib.skv_routing_groups(n_layers, g, out), "skv_routing_groups")
     return list(out)[:n_layers]
+
+
+def _f64_array(xs: Sequence[float]):
+    return (ctypes.c_double * len(xs))(*xs)
+
+
+def skv_routing_rcla(p_self: float, u: Sequence[float], v: Sequence[float]) -> List[int]:
+    n = len(u)
+    out = (ctypes.c_int32 * n)()
+    _check(lib.skv_routing_rcla(n, p_self, _f64_array(list(u)), _f64_array(list(v)), out), "skv_routing_rcla")
+    return list(out)
+
+
+def skv_routing_rdcla(k: int, p_self: float, u: Sequence[float]) -> List[int]:
+    n = len(u)
+    out = (ctypes.c_int32 * n)()
+    _check(lib.skv_routing_rdcla(n, k, p_self, _f64_array(list(u)), out), "skv_routing_rdcla")
+    return list(out)
 
 
 def skv_cache_pool_bytes(r: Sequence[int], kv_heads: int, head_dim: int, page_size: int, max_pages: int) -> int:
@@ -255,6 +276,15 @@ class SkvCache:
                                   _ptr(out), batch, max_q_len, q_heads, page_table.shape[1], scale,
                                   _stream_ptr(stream))
         _check(rc, "skv_prefill_attn")
+
+    def skv_prefill_attn_src(self, src_layer: int, Q: torch.Tensor, cu_q_lens: torch.Tensor, page_table: torch.Tensor,
+                             seq_lens: torch.Tensor, out: torch.Tensor, max_q_len: int, scale: float = 0.0,
+                             stream=None) -> None:
+        batch, q_heads = seq_lens.shape[0], Q.shape[1]
+        rc = lib.skv_prefill_attn_src(self._h, src_layer, _ptr(Q), _ptr(cu_q_lens), _ptr(page_table), _ptr(seq_lens),
+                                      _ptr(out), batch, max_q_len, q_heads, page_table.shape[1], scale,
+                                      _stream_ptr(stream))
+        _check(rc, "skv_prefill_attn_src")
 
     def skv_decode_splitk(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
                           workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:

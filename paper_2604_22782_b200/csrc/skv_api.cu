@@ -168,6 +168,33 @@ int skv_routing_groups(int n_layers, int g, int32_t *r_out)
     return SKV_OK;
 }
 
+int skv_routing_rcla(int n_layers, double p_self, const double *u, const double *v, int32_t *map_out)
+{
+    if (n_layers <= 0 || !u || !v || !map_out || !(p_self >= 0.0 && p_self <= 1.0)) return SKV_ERR_ARG;
+    for (int l = 0; l < n_layers; ++l)
+        if (!(u[l] >= 0.0 && u[l] < 1.0) || !(v[l] >= 0.0 && v[l] < 1.0)) return SKV_ERR_ARG;
+    map_out[0] = 0;                                       // nothing precedes the first layer
+    for (int l = 1; l < n_layers; ++l) {
+        if (u[l] < p_self) {
+            map_out[l] = l;                               // d = 1: the layer's own K,V
+        } else {
+            const int pick = (int)(v[l] * l);             // d = 0: uniform over the l layers before it
+            map_out[l] = pick < l ? pick : l - 1;
+        }
+    }
+    return SKV_OK;
+}
+
+int skv_routing_rdcla(int n_layers, int k, double p_self, const double *u, int32_t *map_out)
+{
+    if (n_layers <= 0 || k <= 0 || !u || !map_out || !(p_self >= 0.0 && p_self <= 1.0)) return SKV_ERR_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!(u[l] >= 0.0 && u[l] < 1.0)) return SKV_ERR_ARG;
+        map_out[l] = u[l] < p_self ? l : l - l % k;
+    }
+    return SKV_OK;
+}
+
 int skv_cache_pool_bytes(int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size,
                          int64_t max_pages, size_t *out_bytes)
 {
@@ -554,12 +581,45 @@ int skv_decode_step(skv_cache *c, const void *Q, const void *K, const void *V, c
 }
 
 // ---- pre-fill attention -------------------------------------------------------
+}  // extern "C"
+
+namespace {
+// pre-fill attention over the pages of owner layer `src` (already resolved and checked)
+int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens, const int32_t *page_table,
+                 const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
+                 float scale, void *stream);
+}  // namespace
+
+extern "C" {
+
 int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q_lens, const int32_t *page_table,
                      const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
                      float scale, void *stream)
 {
-    int rc = check_decode_args(c, layer, batch, q_heads);
+    const int rc = check_decode_args(c, layer, batch, q_heads);
     if (rc) return rc;
+    return prefill_over(c, c->r[(size_t)layer], Q, cu_q_lens, page_table, seq_lens, out, batch, max_q_len, q_heads,
+                        pt_stride, scale, stream);
+}
+
+int skv_prefill_attn_src(skv_cache *c, int src_layer, const void *Q, const int32_t *cu_q_lens,
+                         const int32_t *page_table, const int32_t *seq_lens, void *out, int batch, int max_q_len,
+                         int q_heads, int pt_stride, float scale, void *stream)
+{
+    const int rc = check_decode_args(c, src_layer, batch, q_heads);
+    if (rc) return rc;
+    if (c->slot[(size_t)src_layer] < 0) return SKV_ERR_LAYER;        // only layers that keep their K,V can be read
+    return prefill_over(c, src_layer, Q, cu_q_lens, page_table, seq_lens, out, batch, max_q_len, q_heads, pt_stride,
+                        scale, stream);
+}
+
+}  // extern "C"
+
+namespace {
+int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens, const int32_t *page_table,
+                 const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
+                 float scale, void *stream)
+{
     if (!Q || !cu_q_lens || !page_table || !seq_lens || !out || pt_stride <= 0 || max_q_len <= 0) return SKV_ERR_ARG;
     if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
     if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
@@ -570,7 +630,7 @@ int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q
     const bool umma = c->prefill_variant == 2 || (c->prefill_variant == 0 && can_umma);
     if (!umma && prefill_smem_bytes(c->head_dim) > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     PrefillParams p;
-    p.layer_base = c->layer_base(c->slot[(size_t)c->r[(size_t)layer]]);
+    p.layer_base = c->layer_base(c->slot[(size_t)src]);
     p.page_stride = (int64_t)c->page_bytes;
     p.max_pages = c->max_pages;
     p.Q = static_cast<const uint16_t *>(Q);
@@ -596,6 +656,9 @@ int skv_prefill_attn(skv_cache *c, int layer, const void *Q, const int32_t *cu_q
     c->launches += 1;
     return SKV_OK;
 }
+}  // namespace
+
+extern "C" {
 
 // ---- whole decode step from host buffers -------------------------------------
 namespace {

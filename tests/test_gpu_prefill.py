@@ -158,3 +158,33 @@ def test_tcgen05_repeated_calls_stay_correct(Hq, Hkv):
         _, again = _run(harness, dw, 1, lens)
         assert torch.equal(again.view(torch.int16), first.view(torch.int16))
     assert dw.cache.skv_get_status() == 0
+
+
+@pytest.mark.parametrize("sampler", ["rcla", "rdcla"])
+def test_training_time_routed_forward(sampler):
+    """Section 3.2: one forward pass in which every layer draws its K,V source.  Every layer keeps its own
+    K,V (identity map in the cache); layer l attends the layer the sampler gave it.  The oracle applies the
+    sampled map by indexing (it may send a layer to a layer that itself reads elsewhere)."""
+    from oracle import Oracle
+    from paper_2604_22782_b200 import skv_routing_rcla, skv_routing_rdcla
+    L, Hq, Hkv, D = 8, 8, 2, 128
+    lens = torch.tensor([200, 77, 513], dtype=torch.int32)
+    w = W.Workload("train_fwd", L, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=tuple(range(L)), seed=89)
+    harness, dw = _setup(w, lens)
+    si, pos = W.token_index(lens)
+    g = torch.Generator().manual_seed(11)
+    for trial in range(3):
+        u, v = torch.rand(L, generator=g, dtype=torch.float64).tolist(), torch.rand(L, generator=g, dtype=torch.float64).tolist()
+        m = skv_routing_rcla(0.4, u, v) if sampler == "rcla" else skv_routing_rdcla(4, 0.4, u)
+        assert any(s != l for l, s in enumerate(m))                 # the pass really routes somewhere
+        o = Oracle(L, m, Hq, Hkv, D, lens.numel(), int(lens.max()))
+        for src in sorted(set(m)):
+            K, V = W.draw_kv(w, src, si, pos)
+            o.append(src, K, V, si, pos)
+        for l in range(L):
+            inp = harness.prefill_inputs(dw, l, lens)
+            out = torch.full_like(inp["Q"], float("nan"))
+            dw.cache.skv_prefill_attn_src(m[l], inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, out, int(lens.max()))
+            torch.cuda.synchronize()
+            _check(o, l, inp, out)
+    assert dw.cache.skv_get_status() == 0

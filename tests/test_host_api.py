@@ -173,3 +173,25 @@ def test_work_partition_is_a_balanced_exact_cover():
             assert b <= x < e
     with pytest.raises(skv.SkvError):
         B.skv_plan_worker_of(10, 4, 10)
+
+
+def test_training_time_samplers_agree_with_the_oracle():
+    """R-CLA (Section 3.2) and RD-CLA@k (Section 4.2): library and oracle on the same random draws."""
+    from oracle import rcla_map, rdcla_map
+    rnd = random.Random(7)
+    for _ in range(200):
+        L = rnd.randint(1, 40)
+        p = rnd.choice([0.0, 0.25, 0.5, 0.6, 0.75, 1.0])
+        u = [rnd.random() for _ in range(L)]
+        v = [rnd.random() for _ in range(L)]
+        m = skv.skv_routing_rcla(p, u, v)
+        assert m == rcla_map(p, u, v)
+        assert m[0] == 0 and all(0 <= s <= l for l, s in enumerate(m))
+        k = rnd.randint(1, 6)
+        assert skv.skv_routing_rdcla(k, p, u) == rdcla_map(k, p, u)
+    with pytest.raises(skv.SkvError):
+        skv.skv_routing_rcla(0.5, [1.0], [0.0])
+    with pytest.raises(skv.SkvError):
+        skv.skv_routing_rcla(1.5, [0.1], [0.0])
+    with pytest.raises(skv.SkvError):
+        skv.skv_routing_rdcla(0, 0.5, [0.1])
