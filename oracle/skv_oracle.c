@@ -31,6 +31,8 @@
  *   oracle_rdcla_map    Section 4.2 ablation (RD-CLA@k): the fixed groups of k layers,
  *                       but each layer flips a coin between the group's first layer
  *                       and its own K,V.
+ *   oracle_append_fp8   the same Update through an FP8 (E4M3, per-row scale) quantiser; the
+ *                       attention then sees the dequantised values (scheme stated below).
  *   oracle_mu           Eq. (3.2): owner set S -> map mu (0-based layers).
  *   oracle_group_map    Section 4.3: groups of g consecutive layers share the
  *                       first layer's cache.
@@ -53,6 +55,8 @@ typedef struct {
     int32_t *r;          /* [L] routing map, 0-based, r[l] <= l */
     uint16_t **K;        /* [L] -> [B][n_max][Hkv][D] bf16 bits, NULL until first append */
     uint16_t **V;
+    double **Kq;         /* [L] -> same shape, fp64: layers appended through the fp8 quantiser hold their */
+    double **Vq;         /*        DEQUANTISED values here instead (code value x row scale), NULL otherwise */
 } oracle_t;
 
 static double bf16_to_f64(uint16_t bits)
@@ -76,6 +80,8 @@ oracle_t *oracle_create(int L, const int32_t *r, int Hq, int Hkv, int D, int B, 
     o->r = (int32_t *)malloc(sizeof(int32_t) * (size_t)L);
     o->K = (uint16_t **)calloc((size_t)L, sizeof *o->K);
     o->V = (uint16_t **)calloc((size_t)L, sizeof *o->V);
+    o->Kq = (double **)calloc((size_t)L, sizeof *o->Kq);
+    o->Vq = (double **)calloc((size_t)L, sizeof *o->Vq);
     memcpy(o->r, r, sizeof(int32_t) * (size_t)L);
     return o;
 }
@@ -83,9 +89,15 @@ oracle_t *oracle_create(int L, const int32_t *r, int Hq, int Hkv, int D, int B, 
 void oracle_destroy(oracle_t *o)
 {
     if (!o) return;
-    for (int l = 0; l < o->L; ++l) { free(o->K[l]); free(o->V[l]); }
-    free(o->K); free(o->V); free(o->r); free(o);
+    for (int l = 0; l < o->L; ++l) { free(o->K[l]); free(o->V[l]); free(o->Kq[l]); free(o->Vq[l]); }
+    free(o->K); free(o->V); free(o->Kq); free(o->Vq); free(o->r); free(o);
 }
+
+static int has_store(const oracle_t *o, int l) { return o->Kq[l] || o->K[l]; }
+
+/* element of a layer's K (or V) store as fp64: exact bf16 value, or the dequantised fp8 value */
+static double k_at(const oracle_t *o, int l, size_t i) { return o->Kq[l] ? o->Kq[l][i] : bf16_to_f64(o->K[l][i]); }
+static double v_at(const oracle_t *o, int l, size_t i) { return o->Vq[l] ? o->Vq[l][i] : bf16_to_f64(o->V[l][i]); }
 
 static size_t row_index(const oracle_t *o, int64_t b, int64_t t)
 {
@@ -100,6 +112,7 @@ int oracle_append(oracle_t *o, int layer, const uint16_t *K, const uint16_t *V,
                   const int64_t *seq_idx, const int64_t *pos, int64_t n_tok)
 {
     if (!o || layer < 0 || layer >= o->L) return -1;
+    if (o->Kq[layer]) return -4;                          /* a layer is either bf16 or fp8, not both */
     size_t row = (size_t)o->Hkv * (size_t)o->D;
     if (!o->K[layer]) {
         size_t elems = (size_t)o->B * (size_t)o->n_max * row;
@@ -114,6 +127,113 @@ int oracle_append(oracle_t *o, int layer, const uint16_t *K, const uint16_t *V,
         memcpy(o->V[layer] + at, V + (size_t)i * row, row * sizeof(uint16_t));
     }
     return 0;
+}
+
+/* ---- fp8 pages (quantisation is orthogonal to depth-wise sharing: Section 2, Section 5) ----------
+ * The paper names KV quantisation as composable with its method and fixes no scheme.  The one used
+ * here: OCP FP8 E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, subnormals, largest
+ * finite value 448, no infinities) with one fp32 scale per (token, kv head) row, separately for K
+ * and V:   amax = max |x| over the row;  scale = amax / 448;  code = E4M3(x * (448 / amax)),
+ * round to nearest even, saturating at +-448; a row of zeros has scale 0 and zero codes.  The
+ * divisions and the product are single fp32 operations (both sides take the decision in fp32).
+ * The value the attention sees is  code value x scale. */
+
+/* value of an E4M3 code (NaN codes 0x7f / 0xff never come out of the quantiser) */
+static double e4m3_value(uint8_t c)
+{
+    int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v = (e == 0) ? ldexp((double)m, -9) : ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* fp32 -> E4M3, round to nearest even, saturating */
+static uint8_t e4m3_encode(float y)
+{
+    uint8_t sign = (y < 0.0f || (y == 0.0f && 1.0f / y < 0.0f)) ? 0x80 : 0x00;
+    double a = fabs((double)y);
+    if (a >= 464.0) return sign | 0x7e;                 /* >= the midpoint above 448 (and beyond): saturate */
+    if (a < ldexp(1.0, -6)) {                           /* subnormal range: multiples of 2^-9 */
+        double q = a * 512.0;                           /* exact */
+        double f = floor(q);
+        double r = q - f;
+        int n = (int)f;
+        if (r > 0.5 || (r == 0.5 && (n & 1))) ++n;      /* ties to even */
+        return sign | (uint8_t)n;                       /* n = 8 is the smallest normal, code 0x08 */
+    }
+    int e;
+    double fr = frexp(a, &e);                           /* a = fr * 2^e, fr in [0.5, 1) */
+    double mant = fr * 2.0;                             /* [1, 2) */
+    int ex = e - 1;                                     /* a = mant * 2^ex */
+    double q = (mant - 1.0) * 8.0;                      /* exact in fp64 */
+    double f = floor(q);
+    double r = q - f;
+    int n = (int)f;
+    if (r > 0.5 || (r == 0.5 && (n & 1))) ++n;
+    if (n == 8) { n = 0; ++ex; }
+    int code = ((ex + 7) << 3) | n;
+    if (code > 0x7e) code = 0x7e;
+    return sign | (uint8_t)code;
+}
+
+/* Quantise n rows of D bf16 values: codes [n][D], scales [n]. */
+void oracle_quantize_e4m3(const uint16_t *x, int64_t n, int D, uint8_t *codes, float *scales)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        const uint16_t *row = x + (size_t)i * (size_t)D;
+        float amax = 0.0f;
+        for (int d = 0; d < D; ++d) {
+            float v = (float)fabs(bf16_to_f64(row[d]));
+            if (v > amax) amax = v;
+        }
+        volatile float inv = amax > 0.0f ? 448.0f / amax : 0.0f;
+        volatile float sc = amax / 448.0f;
+        scales[i] = sc;
+        for (int d = 0; d < D; ++d) {
+            volatile float y = (float)bf16_to_f64(row[d]) * inv;     /* one fp32 product */
+            codes[(size_t)i * (size_t)D + (size_t)d] = e4m3_encode(y);
+        }
+    }
+}
+
+double oracle_e4m3_value(int code) { return e4m3_value((uint8_t)code); }
+
+/* "Update" through the quantiser: the layer's store receives the DEQUANTISED rows (code value x
+ * scale, exact in fp64); optionally hands back the codes and scales ([n][Hkv][D] and [n][Hkv]). */
+int oracle_append_fp8(oracle_t *o, int layer, const uint16_t *K, const uint16_t *V,
+                      const int64_t *seq_idx, const int64_t *pos, int64_t n_tok,
+                      uint8_t *K_codes, uint8_t *V_codes, float *K_scales, float *V_scales)
+{
+    if (!o || layer < 0 || layer >= o->L) return -1;
+    if (o->K[layer]) return -4;                          /* a layer is either bf16 or fp8, not both */
+    size_t row = (size_t)o->Hkv * (size_t)o->D;
+    if (!o->Kq[layer]) {
+        size_t elems = (size_t)o->B * (size_t)o->n_max * row;
+        o->Kq[layer] = (double *)calloc(elems, sizeof(double));
+        o->Vq[layer] = (double *)calloc(elems, sizeof(double));
+        if (!o->Kq[layer] || !o->Vq[layer]) return -2;
+    }
+    uint8_t *ck = (uint8_t *)malloc(row), *cv = (uint8_t *)malloc(row);
+    float *sk = (float *)malloc(sizeof(float) * (size_t)o->Hkv), *sv = (float *)malloc(sizeof(float) * (size_t)o->Hkv);
+    if (!ck || !cv || !sk || !sv) { free(ck); free(cv); free(sk); free(sv); return -2; }
+    int rc = 0;
+    for (int64_t i = 0; i < n_tok && rc == 0; ++i) {
+        if (seq_idx[i] < 0 || seq_idx[i] >= o->B || pos[i] < 0 || pos[i] >= o->n_max) { rc = -3; break; }
+        oracle_quantize_e4m3(K + (size_t)i * row, o->Hkv, o->D, ck, sk);
+        oracle_quantize_e4m3(V + (size_t)i * row, o->Hkv, o->D, cv, sv);
+        size_t at = row_index(o, seq_idx[i], pos[i]);
+        for (int h = 0; h < o->Hkv; ++h)
+            for (int d = 0; d < o->D; ++d) {
+                size_t j = (size_t)h * (size_t)o->D + (size_t)d;
+                o->Kq[layer][at + j] = e4m3_value(ck[j]) * (double)sk[h];
+                o->Vq[layer][at + j] = e4m3_value(cv[j]) * (double)sv[h];
+            }
+        if (K_codes) memcpy(K_codes + (size_t)i * row, ck, row);
+        if (V_codes) memcpy(V_codes + (size_t)i * row, cv, row);
+        if (K_scales) memcpy(K_scales + (size_t)i * (size_t)o->Hkv, sk, sizeof(float) * (size_t)o->Hkv);
+        if (V_scales) memcpy(V_scales + (size_t)i * (size_t)o->Hkv, sv, sizeof(float) * (size_t)o->Hkv);
+    }
+    free(ck); free(cv); free(sk); free(sv);
+    return rc;
 }
 
 /* Read back one stored row (bit patterns) of a layer's own store. */
@@ -134,15 +254,14 @@ static int weights_of(const oracle_t *o, int layer, const uint16_t *Q, int b, in
                       int64_t n, double scale, double *w)
 {
     int src = o->r[layer];
-    const uint16_t *Ks = o->K[src];
-    if (!Ks) return -1;
+    if (!has_store(o, src)) return -1;
     int G = o->Hq / o->Hkv, kv = h / G, D = o->D;
     const uint16_t *q = Q + ((size_t)b * (size_t)o->Hq + (size_t)h) * (size_t)D;
     double smax = -INFINITY;
     for (int64_t t = 0; t < n; ++t) {
-        const uint16_t *k = Ks + row_index(o, b, t) + (size_t)kv * (size_t)D;
+        size_t k0 = row_index(o, b, t) + (size_t)kv * (size_t)D;
         double s = 0.0;
-        for (int d = 0; d < D; ++d) s += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+        for (int d = 0; d < D; ++d) s += bf16_to_f64(q[d]) * k_at(o, src, k0 + (size_t)d);
         s *= scale;
         w[t] = s;
         if (s > smax) smax = s;
@@ -169,7 +288,7 @@ int oracle_decode_attn(const oracle_t *o, int layer, const uint16_t *Q, const in
 {
     if (!o || layer < 0 || layer >= o->L) return -1;
     int src = o->r[layer];
-    if (!o->K[src] || !o->V[src]) return -1;
+    if (!has_store(o, src)) return -1;
     int G = o->Hq / o->Hkv, D = o->D;
     for (int b = 0; b < o->B; ++b)
         if (seq_lens[b] < 0 || seq_lens[b] > o->n_max) return -3;
@@ -190,8 +309,8 @@ int oracle_decode_attn(const oracle_t *o, int layer, const uint16_t *Q, const in
             }
             int kv = h / G;
             for (int64_t t = 0; t < n; ++t) {
-                const uint16_t *v = o->V[src] + row_index(o, b, t) + (size_t)kv * (size_t)D;
-                for (int d = 0; d < D; ++d) y[d] += w[t] * bf16_to_f64(v[d]);
+                size_t v0 = row_index(o, b, t) + (size_t)kv * (size_t)D;
+                for (int d = 0; d < D; ++d) y[d] += w[t] * v_at(o, src, v0 + (size_t)d);
             }
             free(w);
         }
@@ -210,7 +329,7 @@ int oracle_attn_rows(const oracle_t *o, int layer, const uint16_t *Q, const int6
 {
     if (!o || layer < 0 || layer >= o->L) return -1;
     int src = o->r[layer];
-    if (!o->K[src] || !o->V[src]) return -1;
+    if (!has_store(o, src)) return -1;
     int G = o->Hq / o->Hkv, D = o->D;
     for (int64_t i = 0; i < n_q; ++i)
         if (q_seq[i] < 0 || q_seq[i] >= o->B || q_pos[i] < 0 || q_pos[i] >= o->n_max) return -3;
@@ -230,9 +349,9 @@ int oracle_attn_rows(const oracle_t *o, int layer, const uint16_t *Q, const int6
             }
             double smax = -INFINITY;
             for (int64_t t = 0; t < n; ++t) {
-                const uint16_t *k = o->K[src] + row_index(o, b, t) + (size_t)kv * (size_t)D;
+                size_t k0 = row_index(o, b, t) + (size_t)kv * (size_t)D;
                 double acc = 0.0;
-                for (int d = 0; d < D; ++d) acc += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+                for (int d = 0; d < D; ++d) acc += bf16_to_f64(q[d]) * k_at(o, src, k0 + (size_t)d);
                 s[t] = scale * acc;
                 if (s[t] > smax) smax = s[t];
             }
@@ -240,9 +359,9 @@ int oracle_attn_rows(const oracle_t *o, int layer, const uint16_t *Q, const int6
             for (int64_t t = 0; t < n; ++t) { s[t] = exp(s[t] - smax); denom += s[t]; }
             for (int d = 0; d < D; ++d) y[d] = 0.0;
             for (int64_t t = 0; t < n; ++t) {
-                const uint16_t *v = o->V[src] + row_index(o, b, t) + (size_t)kv * (size_t)D;
+                size_t v0 = row_index(o, b, t) + (size_t)kv * (size_t)D;
                 double w = s[t] / denom;
-                for (int d = 0; d < D; ++d) y[d] += w * bf16_to_f64(v[d]);
+                for (int d = 0; d < D; ++d) y[d] += w * v_at(o, src, v0 + (size_t)d);
             }
             free(s);
         }

@@ -45,6 +45,11 @@ def _load():
                                             ctypes.c_int64, ctypes.c_double, f64p]
         lib.oracle_decode_attn.argtypes = [vp, ctypes.c_int, u16p, i32p, ctypes.c_double, f64p]
         lib.oracle_attn_rows.argtypes = [vp, ctypes.c_int, u16p, i64p, i64p, ctypes.c_int64, ctypes.c_double, f64p]
+        lib.oracle_quantize_e4m3.restype = None
+        lib.oracle_quantize_e4m3.argtypes = [u16p, ctypes.c_int64, ctypes.c_int, vp, vp]
+        lib.oracle_e4m3_value.restype = ctypes.c_double
+        lib.oracle_e4m3_value.argtypes = [ctypes.c_int]
+        lib.oracle_append_fp8.argtypes = [vp, ctypes.c_int, u16p, u16p, i64p, i64p, ctypes.c_int64, vp, vp, vp, vp]
         lib.oracle_rcla_map.argtypes = [ctypes.c_int, ctypes.c_double, f64p, f64p, i32p]
         lib.oracle_rdcla_map.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double, f64p, i32p]
         lib.oracle_mu.argtypes = [ctypes.c_int, i32p, ctypes.c_int, i32p]
@@ -72,6 +77,21 @@ def mu_from_owners(n_layers: int, owners: Sequence[int]):
     out = torch.empty(n_layers, dtype=torch.int32)
     rc = _load().oracle_mu(n_layers, ow.data_ptr(), ow.numel(), out.data_ptr())
     return out.tolist() if rc == 0 else None
+
+
+def quantize_e4m3(x: torch.Tensor):
+    """FP8 E4M3 codes (uint8, same shape) and one fp32 scale per row (last dim) of a bf16 tensor."""
+    xb = _bf16_bits(x)
+    D = xb.shape[-1]
+    n = xb.numel() // D
+    codes = torch.empty(xb.shape, dtype=torch.uint8)
+    scales = torch.empty(xb.shape[:-1], dtype=torch.float32)
+    _load().oracle_quantize_e4m3(xb.data_ptr(), n, D, codes.data_ptr(), scales.data_ptr())
+    return codes, scales
+
+
+def e4m3_value(code: int) -> float:
+    return float(_load().oracle_e4m3_value(int(code)))
 
 
 def rcla_map(p_self: float, u: Sequence[float], v: Sequence[float]):
@@ -139,6 +159,23 @@ class Oracle:
         rc = self.lib.oracle_append(self.h, layer, kb.data_ptr(), vb.data_ptr(), s.data_ptr(), p.data_ptr(), n)
         if rc != 0:
             raise RuntimeError(f"oracle_append failed: {rc}")
+
+    def append_fp8(self, layer: int, K: torch.Tensor, V: torch.Tensor, seq_idx: torch.Tensor, pos: torch.Tensor):
+        """Update through the FP8 quantiser; returns (K codes, V codes, K scales, V scales) of the rows."""
+        kb, vb = _bf16_bits(K), _bf16_bits(V)
+        n = kb.shape[0]
+        assert kb.shape == (n, self.Hkv, self.D) and vb.shape == kb.shape
+        s = seq_idx.to(torch.int64).contiguous()
+        p = pos.to(torch.int64).contiguous()
+        kc = torch.empty((n, self.Hkv, self.D), dtype=torch.uint8)
+        vc = torch.empty_like(kc)
+        ks = torch.empty((n, self.Hkv), dtype=torch.float32)
+        vs = torch.empty_like(ks)
+        rc = self.lib.oracle_append_fp8(self.h, layer, kb.data_ptr(), vb.data_ptr(), s.data_ptr(), p.data_ptr(), n,
+                                        kc.data_ptr(), vc.data_ptr(), ks.data_ptr(), vs.data_ptr())
+        if rc != 0:
+            raise RuntimeError(f"oracle_append_fp8 failed: {rc}")
+        return kc, vc, ks, vs
 
     def read(self, layer: int, b: int, t: int):
         k = torch.empty((self.Hkv, self.D), dtype=torch.int16)

@@ -469,3 +469,71 @@ def test_rdcla_map_mixes_the_group_leader_and_the_layer_itself():
     assert rdcla_map(4, 0.5, [0.1] * 8) == list(range(8))                  # every coin says "own"
     assert rdcla_map(2, 0.6, [0.7, 0.7, 0.2, 0.9, 0.59, 0.61]) == [0, 0, 2, 2, 4, 4]
     assert rdcla_map(3, 0.6, [0.7, 0.2, 0.9, 0.2, 0.7, 0.61]) == [0, 1, 0, 3, 3, 3]
+
+
+# ------------------------------------------------------------------ fp8 pages: the quantiser and attention over it
+def test_e4m3_code_values_and_roundtrip():
+    """All 254 finite codes: the value formula of the format (bias 7, 3 mantissa bits, subnormals, max 448),
+    and torch's own float8_e4m3fn decoding of the same bits."""
+    from oracle import e4m3_value
+    codes = [c for c in range(256) if (c & 0x7f) != 0x7f]
+    mine = torch.tensor([e4m3_value(c) for c in codes], dtype=torch.float64)
+    theirs = torch.tensor(codes, dtype=torch.uint8).view(torch.float8_e4m3fn).double()
+    assert torch.equal(mine, theirs)
+    assert e4m3_value(0x7e) == 448.0 and e4m3_value(0x01) == 2.0 ** -9 and e4m3_value(0x08) == 2.0 ** -6
+    assert e4m3_value(0xc5) == -(1 + 5 / 8) * 2.0
+
+
+def test_e4m3_quantiser_matches_library_rounding_and_saturates():
+    """Rows with amax = 448 have inv = 1, so codes = E4M3(x): torch's cast (round to nearest even) pins the
+    rounding on random and on tie values; larger scales pin scale = amax/448 and saturation of the row maximum."""
+    from oracle import quantize_e4m3
+    g = torch.Generator().manual_seed(9)
+    x = (torch.randn(64, 128, generator=g) * 40).clamp(-440, 440)
+    x[:, 0] = 448.0                                                     # pins amax, so inv = 1 exactly
+    ties = torch.tensor([2.0 ** -10, 1.5 * 2.0 ** -9, 2.5 * 2.0 ** -9, 17.0, 19.0, 0.0, -0.0, 2.0 ** -6 - 2.0 ** -10])
+    x[0, 1:1 + ties.numel()] = ties
+    xb = x.to(torch.bfloat16)
+    codes, scales = quantize_e4m3(xb)
+    want = xb.float().to(torch.float8_e4m3fn).view(torch.uint8)
+    assert torch.equal(codes, want) and bool((scales == 1.0).all())
+    # general scale: dequantised value within half a code step of the input, the row maximum maps to +-448
+    y = (torch.randn(32, 64, generator=g) * 3).to(torch.bfloat16)
+    c, s = quantize_e4m3(y)
+    amax = y.float().abs().max(dim=1).values
+    assert torch.equal(s, amax / 448.0)
+    deq = c.view(torch.float8_e4m3fn).float() * s[:, None]
+    assert bool(((deq - y.float()).abs() <= (amax[:, None] / 448.0) * 16.0 * 1.001 + 1e-6).all())    # coarsest step is 32 at the top binade
+    top = y.float().abs().argmax(dim=1)
+    assert bool((c[torch.arange(32), top] & 0x7f == 0x7e).all())
+    z, sz = quantize_e4m3(torch.zeros(2, 16, dtype=torch.bfloat16))
+    assert int(z.sum()) == 0 and bool((sz == 0).all())
+
+
+def test_attention_over_fp8_layers_is_attention_over_the_dequantised_values():
+    """A layer appended through the quantiser behaves exactly like a layer holding code x scale."""
+    L, B, n, Hq, Hkv, D = 2, 2, 21, 4, 2, 32
+    o = Oracle(L, [0, 0], Hq, Hkv, D, B, n)
+    b_idx = torch.arange(B).repeat_interleave(n)
+    t_idx = torch.arange(n).repeat(B)
+    K = _rand_bf16((B * n, Hkv, D), 1, std=2.0)
+    V = _rand_bf16((B * n, Hkv, D), 2, std=0.5)
+    kc, vc, ks, vs = o.append_fp8(0, K, V, b_idx, t_idx)
+    Kd = (kc.view(torch.float8_e4m3fn).double() * ks.double()[..., None]).view(B, n, Hkv, D)
+    Vd = (vc.view(torch.float8_e4m3fn).double() * vs.double()[..., None]).view(B, n, Hkv, D)
+    lens = torch.tensor([21, 8], dtype=torch.int32)
+    Q = _rand_bf16((B, Hq, D), 3)
+    G = Hq // Hkv
+    got = o.decode_attn(1, Q, lens, 0.3)
+    for b in range(B):
+        nb = int(lens[b])
+        q = Q[b].double()[None, :, None, :]
+        k = Kd[b, :nb].permute(1, 0, 2).repeat_interleave(G, 0)[None]
+        v = Vd[b, :nb].permute(1, 0, 2).repeat_interleave(G, 0)[None]
+        want = torch.nn.functional.scaled_dot_product_attention(q, k, v, scale=0.3)[0, :, 0, :]
+        assert torch.allclose(got[b], want, rtol=1e-12, atol=1e-13)
+    # and it is close to, but not the same as, attention over the unquantised rows
+    o2 = Oracle(L, [0, 0], Hq, Hkv, D, B, n)
+    o2.append(0, K, V, b_idx, t_idx)
+    ref = o2.decode_attn(1, Q, lens, 0.3)
+    assert not torch.equal(got, ref) and (got - ref).abs().max() < 0.1
