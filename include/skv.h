@@ -115,6 +115,25 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
                      int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes,
                      void *stream);
 
+/* The same cache with FP8 pages (the paper names KV quantisation as composable
+ * with depth-wise sharing, Sections 2 and 5, and fixes no scheme; this is the
+ * library's): OCP E4M3 codes and one fp32 scale per (token, kv head) row, for K
+ * and for V separately.  skv_append quantises on the way in:
+ *   amax = max |x| over the row's head_dim values,  scale = amax / 448,
+ *   code = E4M3(x * (448 / amax)), round to nearest even, saturating at +-448
+ * (a row of zeros: scale 0, codes 0; each step is one fp32 operation), and the
+ * attention sees  code value x scale.  Cache bytes per token become
+ * 2 x |owners| x kv_heads x (head_dim + 4).  skv_decode_attn, skv_decode_step and
+ * skv_decode_step_host work on such a cache as on a bf16 one (any q_heads /
+ * kv_heads <= 8, tensor cores in f16, scales applied outside the contractions);
+ * skv_gather and the pre-fill calls return SKV_ERR_UNSUPPORTED.  Same
+ * arguments and errors as skv_cache_pool_bytes / skv_cache_create. */
+int skv_cache_pool_bytes_fp8(int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                             int page_size, int64_t max_pages, size_t *out_bytes);
+int skv_cache_create_fp8(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                         int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes,
+                         void *stream);
+
 /* Frees host state (and the handle's copy stream and events, if
  * skv_decode_step_host created them); never touches device_pool. */
 void skv_cache_destroy(skv_cache *cache);
@@ -127,7 +146,8 @@ int skv_is_owner(const skv_cache *cache, int layer);
 /* Byte accounting; any out pointer may be NULL.
  *   page_bytes      bytes of one page of one owner layer
  *   kv_bytes        |owners| * max_pages * page_bytes (the KV storage proper)
- *   bytes_per_token 2 * |owners| * kv_heads * head_dim * 2 */
+ *   bytes_per_token 2 * |owners| * kv_heads * head_dim * 2
+ *                   (FP8 cache: 2 * |owners| * kv_heads * (head_dim + 4)) */
 int skv_cache_stats(const skv_cache *cache, int *n_owners, size_t *page_bytes, size_t *kv_bytes,
                     size_t *bytes_per_token);
 
@@ -151,6 +171,13 @@ int skv_append(skv_cache *cache, int layer, const void *K, const void *V, const 
  *   K_out, V_out device bf16 [n][kv_heads][head_dim] */
 int skv_gather(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t n, void *K_out,
                void *V_out, void *stream);
+
+/* Read-back of an FP8 cache (skv_cache_create_fp8): the stored codes and scales.
+ *   K_codes, V_codes  device uint8 [n][kv_heads][head_dim]
+ *   K_scales, V_scales device fp32 [n][kv_heads]
+ * SKV_ERR_UNSUPPORTED on a bf16 cache. */
+int skv_gather_fp8(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t n, void *K_codes,
+                   void *V_codes, float *K_scales, float *V_scales, void *stream);
 
 /* ---- Algorithm 2 "Load + Attn": decode attention -------------------------- */
 

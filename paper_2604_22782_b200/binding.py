@@ -49,6 +49,9 @@ lib.skv_routing_rcla.argtypes = [_int, ctypes.c_double, _vp, _vp, _i32p]
 lib.skv_routing_rdcla.argtypes = [_int, _int, ctypes.c_double, _vp, _i32p]
 lib.skv_cache_pool_bytes.argtypes = [_int, _i32p, _int, _int, _int, _i64, _szp]
 lib.skv_cache_create.argtypes = [ctypes.POINTER(_vp), _int, _i32p, _int, _int, _int, _i64, _vp, _sz, _vp]
+lib.skv_cache_create_fp8.argtypes = lib.skv_cache_create.argtypes
+lib.skv_cache_pool_bytes_fp8.argtypes = [_int, _i32p, _int, _int, _int, _i64, _szp]
+lib.skv_gather_fp8.argtypes = [_vp, _int, _i64p, _i64, _vp, _vp, _vp, _vp, _vp]
 lib.skv_cache_destroy.restype = None
 lib.skv_cache_destroy.argtypes = [_vp]
 lib.skv_layer_owner.argtypes = [_vp, _int]
@@ -144,6 +147,13 @@ def skv_cache_pool_bytes(r: Sequence[int], kv_heads: int, head_dim: int, page_si
     return out.value
 
 
+def skv_cache_pool_bytes_fp8(r: Sequence[int], kv_heads: int, head_dim: int, page_size: int, max_pages: int) -> int:
+    out = _sz(0)
+    _check(lib.skv_cache_pool_bytes_fp8(len(r), _i32_array(r), kv_heads, head_dim, page_size, max_pages,
+                                        ctypes.byref(out)), "skv_cache_pool_bytes_fp8")
+    return out.value
+
+
 def skv_plan_worker_range(n_blocks: int, n_workers: int, w: int):
     b, e = _i64(0), _i64(0)
     _check(lib.skv_plan_worker_range(n_blocks, n_workers, w, ctypes.byref(b), ctypes.byref(e)),
@@ -178,27 +188,28 @@ class SkvCache:
 
     def __init__(self, r: Sequence[int], kv_heads: int, head_dim: int, page_size: int, max_pages: int,
                  device_pool: Optional[torch.Tensor] = None, allocate: bool = False,
-                 accounting_only: bool = False, stream=None):
+                 accounting_only: bool = False, stream=None, fp8: bool = False):
+        self.fp8 = fp8
+        create = lib.skv_cache_create_fp8 if fp8 else lib.skv_cache_create
         self.r = [int(x) for x in r]
         self.n_layers = len(self.r)
         self.kv_heads, self.head_dim, self.page_size, self.max_pages = kv_heads, head_dim, page_size, max_pages
         self._h = _vp()
         self.pool = None
         if accounting_only:
-            rc = lib.skv_cache_create(ctypes.byref(self._h), self.n_layers, _i32_array(self.r), kv_heads, head_dim,
-                                      page_size, max_pages, None, 0, None)
+            rc = create(ctypes.byref(self._h), self.n_layers, _i32_array(self.r), kv_heads, head_dim,
+                        page_size, max_pages, None, 0, None)
             _check(rc, "skv_cache_create")
             return
-        need = skv_cache_pool_bytes(self.r, kv_heads, head_dim, page_size, max_pages)
+        need = (skv_cache_pool_bytes_fp8 if fp8 else skv_cache_pool_bytes)(self.r, kv_heads, head_dim, page_size, max_pages)
         if device_pool is None:
             if not allocate:
                 raise ValueError("pass device_pool, allocate=True or accounting_only=True")
             device_pool = torch.empty(need, dtype=torch.uint8, device="cuda")
         assert device_pool.is_cuda and device_pool.dtype == torch.uint8 and device_pool.is_contiguous()
         self.pool = device_pool
-        rc = lib.skv_cache_create(ctypes.byref(self._h), self.n_layers, _i32_array(self.r), kv_heads, head_dim,
-                                  page_size, max_pages, device_pool.data_ptr(), device_pool.numel(),
-                                  _stream_ptr(stream))
+        rc = create(ctypes.byref(self._h), self.n_layers, _i32_array(self.r), kv_heads, head_dim,
+                    page_size, max_pages, device_pool.data_ptr(), device_pool.numel(), _stream_ptr(stream))
         _check(rc, "skv_cache_create")
 
     # -- lifetime
@@ -242,6 +253,12 @@ class SkvCache:
         rc = lib.skv_gather(self._h, layer, _ptr(slot_ids), slot_ids.numel(), _ptr(K_out), _ptr(V_out),
                             _stream_ptr(stream))
         _check(rc, "skv_gather")
+
+    def skv_gather_fp8(self, layer: int, slot_ids: torch.Tensor, K_codes: torch.Tensor, V_codes: torch.Tensor,
+                       K_scales: torch.Tensor, V_scales: torch.Tensor, stream=None) -> None:
+        rc = lib.skv_gather_fp8(self._h, layer, _ptr(slot_ids), slot_ids.numel(), _ptr(K_codes), _ptr(V_codes),
+                                _ptr(K_scales), _ptr(V_scales), _stream_ptr(stream))
+        _check(rc, "skv_gather_fp8")
 
     # -- Load + Attn
     def skv_decode_workspace_bytes(self, batch: int, q_heads: int) -> int:

@@ -23,6 +23,7 @@ struct skv_cache {
     int sm_count = 0;
     int max_smem_optin = 0;
     DecodeTuning tune{0, 2, 2, 4, 1};
+    bool fp8 = false;                // pages hold E4M3 codes + per-row scales instead of bf16
     int prefill_variant = 0;         // 0 auto (tcgen05 where supported), 1 mma.sync kernel, 2 tcgen05 kernel
     bool shape_is_default = true;    // until skv_set_decode_tuning is called: the CUDA-core kernel runs as 1 x 2 x 8
     int l2_keep_pct = 35;            // > 0: consecutive layers that read one owner walk it in opposite directions
@@ -66,7 +67,10 @@ int check_shape(int kv_heads, int head_dim, int page_size, int64_t max_pages)
     return SKV_OK;
 }
 
-size_t page_bytes_of(int kv_heads, int head_dim) { return (size_t)kv_heads * block_bytes(head_dim); }
+size_t page_bytes_of(int kv_heads, int head_dim, bool fp8)
+{
+    return (size_t)kv_heads * (fp8 ? fp8_block_bytes(head_dim) : block_bytes(head_dim));
+}
 
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -195,8 +199,11 @@ int skv_routing_rdcla(int n_layers, int k, double p_self, const double *u, int32
     return SKV_OK;
 }
 
-int skv_cache_pool_bytes(int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size,
-                         int64_t max_pages, size_t *out_bytes)
+}  // extern "C"
+
+namespace {
+int pool_bytes_impl(int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size, int64_t max_pages,
+                    bool fp8, size_t *out_bytes)
 {
     if (!out_bytes) return SKV_ERR_ARG;
     int rc = check_routing(n_layers, r);
@@ -205,17 +212,17 @@ int skv_cache_pool_bytes(int n_layers, const int32_t *r, int kv_heads, int head_
     if (rc) return rc;
     size_t owners = 0;
     for (int l = 0; l < n_layers; ++l) owners += (r[l] == l);
-    *out_bytes = HEADER_BYTES + owners * (size_t)max_pages * page_bytes_of(kv_heads, head_dim);
+    *out_bytes = HEADER_BYTES + owners * (size_t)max_pages * page_bytes_of(kv_heads, head_dim, fp8);
     return SKV_OK;
 }
 
-int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
-                     int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes, void *stream)
+int create_impl(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size,
+                int64_t max_pages, void *device_pool, size_t pool_bytes, void *stream, bool fp8)
 {
     if (!out) return SKV_ERR_ARG;
     *out = nullptr;
     size_t need = 0;
-    int rc = skv_cache_pool_bytes(n_layers, r, kv_heads, head_dim, page_size, max_pages, &need);
+    int rc = pool_bytes_impl(n_layers, r, kv_heads, head_dim, page_size, max_pages, fp8, &need);
     if (rc) return rc;
     if (device_pool) {
         if (!aligned(device_pool, 256)) return SKV_ERR_ARG;
@@ -238,7 +245,8 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
             c->owners.push_back(l);
         }
     c->n_owners = (int)c->owners.size();
-    c->page_bytes = page_bytes_of(kv_heads, head_dim);
+    c->fp8 = fp8;
+    c->page_bytes = page_bytes_of(kv_heads, head_dim, fp8);
     plan_walks(c);
     c->pool = static_cast<uint8_t *>(device_pool);
     c->pool_bytes = device_pool ? need : 0;
@@ -255,6 +263,34 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
     }
     *out = c;
     return SKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int skv_cache_pool_bytes(int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size,
+                         int64_t max_pages, size_t *out_bytes)
+{
+    return pool_bytes_impl(n_layers, r, kv_heads, head_dim, page_size, max_pages, false, out_bytes);
+}
+
+int skv_cache_pool_bytes_fp8(int n_layers, const int32_t *r, int kv_heads, int head_dim, int page_size,
+                             int64_t max_pages, size_t *out_bytes)
+{
+    return pool_bytes_impl(n_layers, r, kv_heads, head_dim, page_size, max_pages, true, out_bytes);
+}
+
+int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                     int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes, void *stream)
+{
+    return create_impl(out, n_layers, r, kv_heads, head_dim, page_size, max_pages, device_pool, pool_bytes, stream, false);
+}
+
+int skv_cache_create_fp8(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
+                         int page_size, int64_t max_pages, void *device_pool, size_t pool_bytes, void *stream)
+{
+    return create_impl(out, n_layers, r, kv_heads, head_dim, page_size, max_pages, device_pool, pool_bytes, stream, true);
 }
 
 void skv_cache_destroy(skv_cache *cache)
@@ -292,7 +328,9 @@ int skv_cache_stats(const skv_cache *c, int *n_owners, size_t *page_bytes, size_
     if (n_owners) *n_owners = c->n_owners;
     if (page_bytes) *page_bytes = c->page_bytes;
     if (kv_bytes) *kv_bytes = (size_t)c->n_owners * (size_t)c->max_pages * c->page_bytes;
-    if (bytes_per_token) *bytes_per_token = (size_t)2 * c->n_owners * c->kv_heads * c->head_dim * 2;
+    if (bytes_per_token)      // bf16: 2 bytes per value; fp8: 1 byte per value + one fp32 scale per row
+        *bytes_per_token = c->fp8 ? (size_t)2 * c->n_owners * c->kv_heads * (c->head_dim + 4)
+                                  : (size_t)2 * c->n_owners * c->kv_heads * c->head_dim * 2;
     return SKV_OK;
 }
 
@@ -307,6 +345,23 @@ int skv_append(skv_cache *c, int layer, const void *K, const void *V, const int6
     if (!c->pool) return SKV_ERR_ARG;
     if (n_tokens == 0) return SKV_OK;
     if (!K || !V || !slot_map || !aligned(K, 16) || !aligned(V, 16)) return SKV_ERR_ARG;
+    if (c->fp8) {
+        AppendFp8Params q;
+        q.layer_base = c->layer_base(s);
+        q.K = static_cast<const uint16_t *>(K);
+        q.V = static_cast<const uint16_t *>(V);
+        q.slot_map = slot_map;
+        q.n_tokens = n_tokens;
+        q.n_slots = c->max_pages * PAGE;
+        q.page_stride = (int64_t)c->page_bytes;
+        q.layer_stride = 0;
+        q.Hkv = c->kv_heads;
+        q.D = c->head_dim;
+        q.status = c->status_word();
+        if (launch_append_fp8(q, 1, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+        c->launches += 1;
+        return SKV_OK;
+    }
     AppendParams p;
     p.layer_base = c->layer_base(s);
     p.K = static_cast<const uint4 *>(K);
@@ -328,6 +383,7 @@ int skv_gather(skv_cache *c, int layer, const int64_t *slot_ids, int64_t n, void
 {
     if (!c || !c->pool) return SKV_ERR_ARG;
     if (layer < 0 || layer >= c->n_layers || c->slot[(size_t)layer] < 0) return SKV_ERR_LAYER;
+    if (c->fp8) return SKV_ERR_UNSUPPORTED;            // an FP8 cache is read back with skv_gather_fp8
     if (n < 0) return SKV_ERR_ARG;
     if (n == 0) return SKV_OK;
     if (!slot_ids || !K_out || !V_out || !aligned(K_out, 16) || !aligned(V_out, 16)) return SKV_ERR_ARG;
@@ -343,6 +399,33 @@ int skv_gather(skv_cache *c, int layer, const int64_t *slot_ids, int64_t n, void
     p.D = c->head_dim;
     p.status = c->status_word();
     if (launch_gather(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+    c->launches += 1;
+    return SKV_OK;
+}
+
+int skv_gather_fp8(skv_cache *c, int layer, const int64_t *slot_ids, int64_t n, void *K_codes, void *V_codes,
+                   float *K_scales, float *V_scales, void *stream)
+{
+    if (!c || !c->pool) return SKV_ERR_ARG;
+    if (layer < 0 || layer >= c->n_layers || c->slot[(size_t)layer] < 0) return SKV_ERR_LAYER;
+    if (!c->fp8) return SKV_ERR_UNSUPPORTED;
+    if (n < 0) return SKV_ERR_ARG;
+    if (n == 0) return SKV_OK;
+    if (!slot_ids || !K_codes || !V_codes || !K_scales || !V_scales) return SKV_ERR_ARG;
+    GatherFp8Params p;
+    p.layer_base = c->layer_base(c->slot[(size_t)layer]);
+    p.K_codes = static_cast<uint8_t *>(K_codes);
+    p.V_codes = static_cast<uint8_t *>(V_codes);
+    p.K_scales = K_scales;
+    p.V_scales = V_scales;
+    p.slot_ids = slot_ids;
+    p.n = n;
+    p.n_slots = c->max_pages * PAGE;
+    p.page_stride = (int64_t)c->page_bytes;
+    p.Hkv = c->kv_heads;
+    p.D = c->head_dim;
+    p.status = c->status_word();
+    if (launch_gather_fp8(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
     c->launches += 1;
     return SKV_OK;
 }
@@ -373,7 +456,7 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     const int W = n_workers_of(c);
     const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
-    const bool tensor_core = c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
+    const bool tensor_core = c->fp8 || c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
     // Default launch shapes (8 warps per SM, two 8 KB stages each, many small CTAs so that the CTAs of the
     // next launch can move in one by one): 2 warps x 4 CTAs per SM for the tensor-core kernel, 1 warp x 8
     // CTAs per SM for the CUDA-core kernel (measured best for each on B200).  Same worker count either way.
@@ -382,7 +465,7 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
         warps = 1;
         ctas = 8;
     }
-    const size_t smem = decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages);
+    const size_t smem = decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages, c->fp8);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
@@ -411,7 +494,7 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.status = c->status_word();
     p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
     const int grid = c->sm_count * ctas;
-    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, tensor_core, grid, warps, c->tune.stages,
+    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, c->fp8 ? 2 : tensor_core ? 1 : 0, grid, warps, c->tune.stages,
                                                 c->tune.pdl != 0, st);
     if (le != cudaSuccess) {
         (void)cudaGetLastError();
@@ -505,6 +588,26 @@ namespace {
 int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot_map, int batch, void *stream)
 {
     if (!aligned(K, 16) || !aligned(V, 16)) return SKV_ERR_ARG;
+    if (c->fp8) {
+        AppendFp8Params q;
+        q.layer_base = c->layer_base(0);
+        q.K = static_cast<const uint16_t *>(K);
+        q.V = static_cast<const uint16_t *>(V);
+        q.slot_map = slot_map;
+        q.n_tokens = batch;
+        q.n_slots = c->max_pages * PAGE;
+        q.page_stride = (int64_t)c->page_bytes;
+        q.layer_stride = (int64_t)c->max_pages * (int64_t)c->page_bytes;
+        q.Hkv = c->kv_heads;
+        q.D = c->head_dim;
+        q.status = c->status_word();
+        if (launch_append_fp8(q, c->n_owners, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SKV_ERR_CUDA;
+        }
+        c->launches += 1;
+        return SKV_OK;
+    }
     AppendParams ap;
     ap.layer_base = c->layer_base(0);
     ap.K = static_cast<const uint4 *>(K);
@@ -620,6 +723,7 @@ int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens,
                  const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
                  float scale, void *stream)
 {
+    if (c->fp8) return SKV_ERR_UNSUPPORTED;            // pre-fill reads bf16 pages only
     if (!Q || !cu_q_lens || !page_table || !seq_lens || !out || pt_stride <= 0 || max_q_len <= 0) return SKV_ERR_ARG;
     if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
     if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
@@ -813,7 +917,7 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     if (t.warps < 1 || t.warps > 16 || t.stages < 1 || t.stages > 8 || t.ctas_per_sm < 1 || t.ctas_per_sm > 16)
         return SKV_ERR_ARG;
     if (c->pool) {
-        const size_t smem = decode_smem_bytes(c->head_dim, 1, t.warps, t.stages);
+        const size_t smem = decode_smem_bytes(c->head_dim, 1, t.warps, t.stages, c->fp8);
         if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     }
     c->tune = t;

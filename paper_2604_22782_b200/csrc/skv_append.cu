@@ -77,6 +77,88 @@ __global__ void __launch_bounds__(COPY_THREADS) gather_kernel(GatherParams p)
     *dst = *reinterpret_cast<const uint4 *>(src);
 }
 
+// ---- FP8 pages -----------------------------------------------------------------------------
+// One warp per (token, kv head); grid.y picks K or V, grid.z the owner layer.  The row's D values
+// are spread over the lanes (D/32 each); amax by shuffles; scale = amax / 448, codes =
+// E4M3(x * (448 / amax)) round-to-nearest-even, saturating; every step a single fp32 operation.
+__global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * COPY_THREADS + threadIdx.x) >> 5;
+    if (warp >= p.n_tokens * p.Hkv) return;
+    const int64_t tok = warp / p.Hkv;
+    const int h = (int)(warp - tok * p.Hkv);
+    const int64_t slot = p.slot_map[tok];
+    if (slot < 0) return;
+    if (slot >= p.n_slots) {
+        if (h == 0 && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
+        return;
+    }
+    const int64_t page = slot / PAGE;
+    const int off = (int)(slot - page * PAGE);
+    const int which = blockIdx.y;
+    const int64_t layer = blockIdx.z;
+    const int D = p.D, PER = D / 32;                  // 4 values per lane at D = 128, 2 at D = 64
+    const uint16_t *src = (which ? p.V : p.K) + ((layer * p.n_tokens + tok) * p.Hkv + h) * D + lane * PER;
+    float x[4] = {0.f, 0.f, 0.f, 0.f};
+    if (PER == 4) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2 *>(src));
+        x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    } else {
+        const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(src));
+        x[0] = bf16_lo(w); x[1] = bf16_hi(w);
+    }
+    float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+    const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+    const uint32_t c01 = pack_e4m3x2(__fmul_rn(x[0], inv), __fmul_rn(x[1], inv));
+    const uint32_t c23 = pack_e4m3x2(__fmul_rn(x[2], inv), __fmul_rn(x[3], inv));
+    uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
+    if (which == 0) {                                  // K: token-major rows
+        uint8_t *dst = blk + off * D + lane * PER;
+        if (PER == 4) *reinterpret_cast<uint32_t *>(dst) = c01 | (c23 << 16);
+        else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)c01;
+    } else {                                           // V: dim-major, this token's column
+        uint8_t *dst = blk + fp8_v_off(D) + (lane * PER) * PAGE + off;
+        dst[0] = (uint8_t)(c01 & 0xFF);
+        dst[PAGE] = (uint8_t)(c01 >> 8);
+        if (PER == 4) {
+            dst[2 * PAGE] = (uint8_t)(c23 & 0xFF);
+            dst[3 * PAGE] = (uint8_t)(c23 >> 8);
+        }
+    }
+    if (lane == 0)
+        *reinterpret_cast<float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * off) = __fdiv_rn(amax, 448.f);
+}
+
+// read-back: codes as [n][Hkv][D] for both K and V, scales as [n][Hkv]
+__global__ void __launch_bounds__(COPY_THREADS) gather_fp8_kernel(GatherFp8Params p)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * COPY_THREADS + threadIdx.x) >> 5;
+    if (warp >= p.n * p.Hkv) return;
+    const int64_t tok = warp / p.Hkv;
+    const int h = (int)(warp - tok * p.Hkv);
+    const int64_t slot = p.slot_ids[tok];
+    if (slot < 0) return;
+    if (slot >= p.n_slots) {
+        if (h == 0 && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
+        return;
+    }
+    const int64_t page = slot / PAGE;
+    const int off = (int)(slot - page * PAGE);
+    const int which = blockIdx.y;
+    const int D = p.D;
+    const uint8_t *blk = p.layer_base + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
+    uint8_t *out = (which ? p.V_codes : p.K_codes) + (tok * p.Hkv + h) * D;
+    for (int d = lane; d < D; d += 32)
+        out[d] = which ? blk[fp8_v_off(D) + d * PAGE + off] : blk[off * D + d];
+    if (lane == 0)
+        (which ? p.V_scales : p.K_scales)[tok * p.Hkv + h] =
+            *reinterpret_cast<const float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * off);
+}
+
 // blocks needed for n tokens: one warp per (16 tokens, head, chunk pair)
 int64_t copy_blocks(int64_t n, int Hkv, int D)
 {
@@ -103,6 +185,30 @@ cudaError_t launch_gather(const GatherParams &p, cudaStream_t s)
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     gather_kernel<<<dim3((unsigned)blocks, 2), COPY_THREADS, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace skv
+
+namespace skv {
+
+cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s)
+{
+    const int64_t warps = p.n_tokens * p.Hkv;
+    const int64_t blocks = (warps * 32 + 255) / 256;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFll || n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
+    append_fp8_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), 256, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_fp8(const GatherFp8Params &p, cudaStream_t s)
+{
+    const int64_t warps = p.n * p.Hkv;
+    const int64_t blocks = (warps * 32 + 255) / 256;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
+    gather_fp8_kernel<<<dim3((unsigned)blocks, 2), 256, 0, s>>>(p);
     return cudaGetLastError();
 }
 

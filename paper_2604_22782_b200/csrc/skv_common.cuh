@@ -22,6 +22,15 @@ constexpr int HEADER_BYTES = 256;                // pool header (device status w
 __host__ __device__ constexpr int half_bytes(int D) { return PAGE * D * 2; }
 __host__ __device__ constexpr int block_bytes(int D) { return 2 * half_bytes(D); }
 
+// FP8 pages (E4M3 codes, one fp32 scale per (token, kv head) row for K and for V).  The block of
+// one (page, kv head):  K codes [PAGE tokens][D] | V codes [D dims][PAGE tokens] | K scales [PAGE]
+// fp32 | V scales [PAGE] fp32.  K is token-major and V dim-major so that the decode kernel's tensor-
+// core fragments are plain 32-bit / 128-bit shared-memory loads (see Fp8State in skv_decode.cu).
+__host__ __device__ constexpr int fp8_v_off(int D) { return PAGE * D; }
+__host__ __device__ constexpr int fp8_ks_off(int D) { return 2 * PAGE * D; }
+__host__ __device__ constexpr int fp8_vs_off(int D) { return 2 * PAGE * D + PAGE * 4; }
+__host__ __device__ constexpr int fp8_block_bytes(int D) { return 2 * PAGE * D + 2 * PAGE * 4; }
+
 // device status bits
 constexpr int STATUS_TIMEOUT = 1;
 constexpr int STATUS_BOUNDS = 2;
@@ -35,6 +44,33 @@ struct AppendParams {
     int64_t n_slots;            // max_pages * PAGE
     int64_t page_stride;        // bytes between pages of one layer
     int64_t layer_stride;       // bytes between consecutive owner layers in the pool (grid.z walks them)
+    int Hkv, D;
+    int *status;
+};
+
+struct AppendFp8Params {
+    uint8_t *layer_base;
+    const uint16_t *K;          // [n_layers_here][n_tokens][Hkv][D] bf16 bits
+    const uint16_t *V;
+    const int64_t *slot_map;
+    int64_t n_tokens;
+    int64_t n_slots;
+    int64_t page_stride;
+    int64_t layer_stride;
+    int Hkv, D;
+    int *status;
+};
+
+struct GatherFp8Params {
+    const uint8_t *layer_base;
+    uint8_t *K_codes;           // [n][Hkv][D]
+    uint8_t *V_codes;           // [n][Hkv][D]
+    float *K_scales;            // [n][Hkv]
+    float *V_scales;
+    const int64_t *slot_ids;
+    int64_t n;
+    int64_t n_slots;
+    int64_t page_stride;
     int Hkv, D;
     int *status;
 };
@@ -110,9 +146,12 @@ struct DecodeTuning {
 // host launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s);
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
+cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s);
+cudaError_t launch_gather_fp8(const GatherFp8Params &p, cudaStream_t s);
 // smem bytes the split-K kernel needs for this shape, or 0 if unsupported
-size_t decode_smem_bytes(int D, int B, int warps, int stages);
-cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid,
+size_t decode_smem_bytes(int D, int B, int warps, int stages, bool fp8);
+// kernel variant: 0 = CUDA-core (G = 1), 1 = tensor-core (bf16 pages), 2 = FP8 pages (tensor-core, any G)
+cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, int kernel, int grid,
                                  int warps, int stages, bool pdl, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 size_t prefill_smem_bytes(int D);
@@ -258,6 +297,41 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// D(16x8,f32) += A(16x16,f16,row) * B(16x8,f16,col)
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// four E4M3 codes (one 32-bit word) -> two f16x2 registers: lo = codes 0,1; hi = codes 2,3 (exact)
+__device__ __forceinline__ void e4m3x4_to_f16x2(uint32_t w, uint32_t &lo, uint32_t &hi)
+{
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(w));
+}
+
+// two fp32 -> packed f16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// two fp32 -> two E4M3 codes in the low 16 bits (lo in bits 0-7), round to nearest even, saturating at +-448
+__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return (uint32_t)r;
 }
 
 __device__ __forceinline__ float fast_exp2(float x)

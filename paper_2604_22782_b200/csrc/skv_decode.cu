@@ -81,6 +81,7 @@ __host__ __device__ inline size_t table_bytes(int B) { return (((size_t)(2 * B +
 // ---------------------------------------------------------------------------
 template <int D>
 struct TensorCoreState {
+    static constexpr int BLOCK = block_bytes(D);   // bytes of one (page, kv head) block
     static constexpr int KS = D / 16;   // k-steps of QK^T, and pairs of 8-dim tiles of PV
     uint32_t qa[KS][2];
     float o[D / 8][4];
@@ -101,9 +102,10 @@ struct TensorCoreState {
         l = 0.f;
     }
 
-    // one page: sK/sV = shared addresses of the K and V halves, valid = tokens in use (1..16)
-    __device__ __forceinline__ void page(uint32_t sK, uint32_t sV, int valid, float scale_log2, int lane)
+    // one page: blk = shared address of the block (K half, V half), valid = tokens in use (1..16)
+    __device__ __forceinline__ void page(uint32_t blk, int valid, float scale_log2, int lane)
     {
+        const uint32_t sK = blk, sV = blk + half_bytes(D);
         const int tig = lane & 3;
         float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
         // K fragments: matrices (chunk 2ks | 2ks+1) x (tokens 0-7 | 8-15)
@@ -182,6 +184,7 @@ struct TensorCoreState {
 // ---------------------------------------------------------------------------
 template <int D>
 struct CudaCoreState {
+    static constexpr int BLOCK = block_bytes(D);
     static constexpr int HC = D / 16;   // 16-byte chunks per dim half
     float q[D / 2];
     float o[D / 2];
@@ -205,8 +208,9 @@ struct CudaCoreState {
         l = 0.f;
     }
 
-    __device__ __forceinline__ void page(uint32_t sK, uint32_t sV, int valid, float scale_log2, int lane)
+    __device__ __forceinline__ void page(uint32_t blk, int valid, float scale_log2, int lane)
     {
+        const uint32_t sK = blk, sV = blk + half_bytes(D);
         const int t = lane & 15, hf = lane >> 4;
         const uint32_t off = (uint32_t)((hf * HC * PAGE + t) * 16);
         float acc0 = 0.f, acc1 = 0.f;
@@ -282,6 +286,153 @@ struct CudaCoreState {
         }
     }
 
+};
+
+// ---------------------------------------------------------------------------
+// FP8 pages (E4M3 codes + one fp32 scale per token for K and for V), any group size: tensor cores
+// in f16, which holds every E4M3 value exactly.  Per page  S = (Q/qmax) Kc^T  and  O += P' Vc  on
+// the raw codes; the per-token scales are applied outside the contractions:
+//   score_t = qmax * kscale_t * S_t,      P'_t = p_t * vscale_t / c,
+// with c a power of two >= every vscale seen so far (so P' <= 1 fits f16 whatever the magnitudes;
+// when c grows O is scaled down with the softmax's own rescaling factor), and O * c at the end.
+// Fragments come straight from shared memory without transposes because the contraction order
+// within a k-step is free as long as both operands agree: a thread's k-slots {2tig,2tig+1,
+// 2tig+8,2tig+9} carry FOUR CONSECUTIVE dims (QK^T) or tokens (PV), i.e. one 32-bit word of codes.
+//   QK^T: thread (g = lane/4, tig) reads token rows 4*(g/2) + g%2 (+2 for the second 8-column tile),
+//         bytes [D/4*tig, D/4*(tig+1)), so that its four scores are tokens 4tig .. 4tig+3;
+//   PV:   V is stored dim-major, the word at dim 8*tile + g, byte 4*tig holds tokens 4tig .. 4tig+3.
+// ---------------------------------------------------------------------------
+template <int D>
+struct Fp8State {
+    static constexpr int BLOCK = fp8_block_bytes(D);
+    static constexpr int KS = D / 16;
+    static constexpr int DT = D / 4;    // dims per thread of a quad
+    uint32_t qa[KS][2];                 // f16x2: dims DT*tig + 4ks + {0,1} and + {2,3} of Q / qmax
+    float o[D / 8][4];
+    float m, l, qmax, cs;
+
+    __device__ __forceinline__ void begin(const DecodeParams &p, int b, int h, int G, int lane)
+    {
+        const int g = lane >> 2, tig = lane & 3;
+        float q[DT];
+        float amax = 0.f;
+        if (g < G) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + ((int64_t)b * p.Hq + (int64_t)h * G + g) * D + DT * tig);
+#pragma unroll
+            for (int c = 0; c < DT / 8; ++c) {
+                const uint4 w = __ldg(src + c);
+                q[8 * c + 0] = bf16_lo(w.x); q[8 * c + 1] = bf16_hi(w.x);
+                q[8 * c + 2] = bf16_lo(w.y); q[8 * c + 3] = bf16_hi(w.y);
+                q[8 * c + 4] = bf16_lo(w.z); q[8 * c + 5] = bf16_hi(w.z);
+                q[8 * c + 6] = bf16_lo(w.w); q[8 * c + 7] = bf16_hi(w.w);
+            }
+#pragma unroll
+            for (int i = 0; i < DT; ++i) amax = fmaxf(amax, fabsf(q[i]));
+        } else {
+#pragma unroll
+            for (int i = 0; i < DT; ++i) q[i] = 0.f;
+        }
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
+        qmax = amax;
+        const float inv = amax > 0.f ? 1.f / amax : 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qa[ks][0] = pack_f16x2(q[4 * ks] * inv, q[4 * ks + 1] * inv);
+            qa[ks][1] = pack_f16x2(q[4 * ks + 2] * inv, q[4 * ks + 3] * inv);
+        }
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        m = -INFINITY;
+        l = 0.f;
+        cs = 0.f;
+    }
+
+    __device__ __forceinline__ void page(uint32_t blk, int valid, float scale_log2, int lane)
+    {
+        const int g = lane >> 2, tig = lane & 3;
+        // ---- scores of tokens 4tig .. 4tig+3 for query head g ----
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t k0 = blk + (uint32_t)((4 * (g >> 1) + (g & 1)) * D + DT * tig), k1 = k0 + 2 * D;
+        uint32_t w0[DT / 4], w1[DT / 4];
+#pragma unroll
+        for (int c = 0; c < DT / 16; ++c) {
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(w0[4 * c]), "=r"(w0[4 * c + 1]), "=r"(w0[4 * c + 2]), "=r"(w0[4 * c + 3]) : "r"(k0 + 16 * c));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(w1[4 * c]), "=r"(w1[4 * c + 1]), "=r"(w1[4 * c + 2]), "=r"(w1[4 * c + 3]) : "r"(k1 + 16 * c));
+        }
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t b0, b1;
+            e4m3x4_to_f16x2(w0[ks], b0, b1);
+            mma_f16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+            e4m3x4_to_f16x2(w1[ks], b0, b1);
+            mma_f16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+        }
+        float4 sk, sv;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(sk.x), "=f"(sk.y), "=f"(sk.z), "=f"(sk.w)
+                     : "r"(blk + (uint32_t)(fp8_ks_off(D) + 16 * tig)));
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(sv.x), "=f"(sv.y), "=f"(sv.z), "=f"(sv.w)
+                     : "r"(blk + (uint32_t)(fp8_vs_off(D) + 16 * tig)));
+        const float qs = qmax * scale_log2;
+        const int t0 = 4 * tig;
+        float v0 = s0[0] * (qs * sk.x), v1 = s0[1] * (qs * sk.y), v2 = s1[0] * (qs * sk.z), v3 = s1[1] * (qs * sk.w);
+        uint32_t vmask = 0xFFFFFFFFu;          // bytes of a V word (tokens 4tig..4tig+3) that are in use
+        if (valid < PAGE) {                    // slots past the sequence's end may hold anything
+            if (t0 >= valid) { v0 = -INFINITY; sv.x = 0.f; }
+            if (t0 + 1 >= valid) { v1 = -INFINITY; sv.y = 0.f; }
+            if (t0 + 2 >= valid) { v2 = -INFINITY; sv.z = 0.f; }
+            if (t0 + 3 >= valid) { v3 = -INFINITY; sv.w = 0.f; }
+            const int keep = valid - t0;       // leading bytes to keep
+            vmask = keep >= 4 ? 0xFFFFFFFFu : keep <= 0 ? 0u : (0xFFFFFFFFu >> (8 * (4 - keep)));
+        }
+        float mx = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
+        const float m_new = fmaxf(m, mx);                 // finite: every page has a valid token
+        float alpha = fast_exp2(m - m_new);
+        const float p0 = fast_exp2(v0 - m_new), p1 = fast_exp2(v1 - m_new);
+        const float p2 = fast_exp2(v2 - m_new), p3 = fast_exp2(v3 - m_new);
+        l = l * alpha + ((p0 + p1) + (p2 + p3));
+        m = m_new;
+        // reference scale of the V side: the smallest power of two >= every vscale so far
+        float svmax = fmaxf(fmaxf(sv.x, sv.y), fmaxf(sv.z, sv.w));
+        svmax = fmaxf(svmax, __shfl_xor_sync(FULL, svmax, 1));
+        svmax = fmaxf(svmax, __shfl_xor_sync(FULL, svmax, 2));
+        const float up = __uint_as_float((__float_as_uint(svmax) + 0x007FFFFFu) & 0x7F800000u);
+        const float cs_new = fmaxf(cs, up);
+        const float inv_cs = cs_new > 0.f ? 1.f / cs_new : 0.f;          // exact: a power of two
+        alpha *= cs * inv_cs;                                             // 1 unless the reference grew
+        cs = cs_new;
+        const uint32_t pa0 = pack_f16x2(p0 * (sv.x * inv_cs), p1 * (sv.y * inv_cs));
+        const uint32_t pa2 = pack_f16x2(p2 * (sv.z * inv_cs), p3 * (sv.w * inv_cs));
+        // ---- O += P' Vc ----
+        const uint32_t v_lane = blk + (uint32_t)(fp8_v_off(D) + g * PAGE + 4 * tig);
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) {
+            uint32_t w;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(v_lane + (uint32_t)(nt * 8 * PAGE)));
+            uint32_t b0, b1;
+            e4m3x4_to_f16x2(w & vmask, b0, b1);
+            o[nt][0] *= alpha; o[nt][1] *= alpha;
+            mma_f16_16816(o[nt], pa0, 0u, pa2, 0u, b0, b1);
+        }
+    }
+
+    __device__ __forceinline__ void finish(const DecodeParams &p, int64_t slot, int G, int lane)
+    {
+        const int g = lane >> 2, tig = lane & 3;
+        l += __shfl_xor_sync(FULL, l, 1);
+        l += __shfl_xor_sync(FULL, l, 2);
+        if (g < G) {
+            float *po = p.part_o + (slot * G + g) * D + 2 * tig;
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i)
+                *reinterpret_cast<float2 *>(po + 8 * i) = make_float2(o[i][0] * cs, o[i][1] * cs);
+            if (tig == 0) *reinterpret_cast<float2 *>(p.part_ml + (slot * G + g) * 2) = make_float2(m, l);
+        }
+    }
 };
 
 // ---------------------------------------------------------------------------
@@ -378,7 +529,7 @@ template <int D, class State>
 __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    constexpr int BLOCK = block_bytes(D);
+    constexpr int BLOCK = State::BLOCK;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint64_t t_entry = p.trace ? global_timer_ns() : 0;
     uint64_t t_first = 0;
@@ -521,9 +672,8 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
                     break;
                 }
                 if (p.trace && consumed == 0) t_first = global_timer_ns();
-                const uint32_t sK = ring + (uint32_t)(c_stage * BLOCK);
                 const int left = n_b - cons.pg * PAGE;
-                st.page(sK, sK + half_bytes(D), left < PAGE ? left : PAGE, p.scale_log2, lane);
+                st.page(ring + (uint32_t)(c_stage * BLOCK), left < PAGE ? left : PAGE, p.scale_log2, lane);
                 __syncwarp();                       // every lane is done reading this stage
                 --in_flight;
                 issue();                            // refill it
@@ -599,7 +749,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32) merge_kernel(MergeParams p)
 template <int D, class State>
 cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, int stages, bool pdl, cudaStream_t s)
 {
-    const size_t smem = decode_smem_bytes(D, p.B, warps, stages);
+    const size_t smem = 128 + table_bytes(p.B) + (size_t)warps * stages * State::BLOCK + (size_t)warps * stages * 8 + 16;
     auto kern = decode_splitk_kernel<D, State>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -618,22 +768,25 @@ cudaError_t launch_splitk_t(const DecodeParams &p, int G, int grid, int warps, i
 
 }  // namespace
 
-size_t decode_smem_bytes(int D, int B, int warps, int stages)
+size_t decode_smem_bytes(int D, int B, int warps, int stages, bool fp8)
 {
     if (D != 64 && D != 128) return 0;
+    const size_t blk = fp8 ? fp8_block_bytes(D) : block_bytes(D);
     // 128 bytes of slack for aligning the ring base; 16 bytes for the arrival word
-    return 128 + table_bytes(B) + (size_t)warps * stages * block_bytes(D) + (size_t)warps * stages * 8 + 16;
+    return 128 + table_bytes(B) + (size_t)warps * stages * blk + (size_t)warps * stages * 8 + 16;
 }
 
-cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, bool tensor_core, int grid, int warps,
+cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, int kernel, int grid, int warps,
                                  int stages, bool pdl, cudaStream_t s)
 {
     if (D == 128) {
-        if (tensor_core) return launch_splitk_t<128, TensorCoreState<128>>(p, G, grid, warps, stages, pdl, s);
+        if (kernel == 2) return launch_splitk_t<128, Fp8State<128>>(p, G, grid, warps, stages, pdl, s);
+        if (kernel == 1) return launch_splitk_t<128, TensorCoreState<128>>(p, G, grid, warps, stages, pdl, s);
         return launch_splitk_t<128, CudaCoreState<128>>(p, G, grid, warps, stages, pdl, s);
     }
     if (D == 64) {
-        if (tensor_core) return launch_splitk_t<64, TensorCoreState<64>>(p, G, grid, warps, stages, pdl, s);
+        if (kernel == 2) return launch_splitk_t<64, Fp8State<64>>(p, G, grid, warps, stages, pdl, s);
+        if (kernel == 1) return launch_splitk_t<64, TensorCoreState<64>>(p, G, grid, warps, stages, pdl, s);
         return launch_splitk_t<64, CudaCoreState<64>>(p, G, grid, warps, stages, pdl, s);
     }
     return cudaErrorInvalidValue;

@@ -53,10 +53,11 @@ class DeviceWorkload:
 
     def kv_bytes_per_call(self) -> int:
         """Algorithmic bytes of one decode-attention call: the owner layer's K,V of
-        every attended token, plus Q in and out out."""
+        every attended token (bf16, or FP8 codes plus one fp32 scale per row), plus Q in and out out."""
         w = self.w
         tokens = int(self.lens_cpu.to(torch.int64).sum())
-        return tokens * w.kv_heads * w.head_dim * 2 * 2 + 2 * self.batch * w.q_heads * w.head_dim * 2
+        row = (w.head_dim + 4) if self.cache.fp8 else w.head_dim * 2
+        return tokens * w.kv_heads * row * 2 + 2 * self.batch * w.q_heads * w.head_dim * 2
 
     def append_bytes_per_call(self) -> int:
         """Algorithmic bytes of one owner-layer append of one token per sequence (read + write)."""
@@ -65,7 +66,7 @@ class DeviceWorkload:
 
 
 def setup(w: W.Workload, device="cuda", lens: Optional[torch.Tensor] = None, r: Optional[List[int]] = None,
-          extra_pages: int = 0, permute: Optional[bool] = None) -> DeviceWorkload:
+          extra_pages: int = 0, permute: Optional[bool] = None, fp8: bool = False) -> DeviceWorkload:
     device = torch.device(device)
     r = W.routing_map(w) if r is None else list(r)
     lens_cpu = (W.seq_lens(w) if lens is None else lens).to(torch.int32)
@@ -73,7 +74,7 @@ def setup(w: W.Workload, device="cuda", lens: Optional[torch.Tensor] = None, r: 
     table, total = W.page_layout(lens_cpu, w.page_size, w.permute_pages if permute is None else permute, w.seed,
                                  extra_pages=extra_pages)
     total = max(total, 1)
-    cache = SkvCache(r, w.kv_heads, w.head_dim, w.page_size, total, allocate=True)
+    cache = SkvCache(r, w.kv_heads, w.head_dim, w.page_size, total, allocate=True, fp8=fp8)
     ws = torch.empty(cache.skv_decode_workspace_bytes(B, w.q_heads), dtype=torch.uint8, device=device)
     b = torch.arange(B, dtype=torch.int64)
     last = (lens_cpu.to(torch.int64) - 1)

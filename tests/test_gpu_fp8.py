@@ -1,0 +1,125 @@
+"""FP8 pages (E4M3 codes + one fp32 scale per (token, kv head) row): cache contents bit for bit against
+the oracle's quantiser, decode attention against the oracle's attention over the dequantised values."""
+import pytest
+import torch
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 1e-2, 1e-2
+
+
+def _setup(w, lens, poison=False):
+    from paper_2604_22782_b200 import harness
+    dw = harness.setup(w, lens=lens, fp8=True)
+    if poison:       # every byte 0x7f: NaN codes and NaN scales in every slot that is never written
+        dw.cache.pool[256:].fill_(0x7F)
+    harness.prefill(dw, upto_offset=0)
+    return harness, dw
+
+
+def _oracle(dw, layers):
+    """Oracle with the source layers appended through its quantiser; also returns their codes and scales."""
+    from oracle import Oracle
+    w = dw.w
+    o = Oracle(w.n_layers, dw.r, w.q_heads, w.kv_heads, w.head_dim, dw.batch, max(1, int(dw.lens_cpu.max())))
+    si, pos = W.token_index(dw.lens_cpu)
+    stored = {}
+    for src in sorted({dw.r[l] for l in layers}):
+        K, V = W.draw_kv(w, src, si, pos)
+        stored[src] = o.append_fp8(src, K, V, si, pos)
+    return o, stored, si, pos
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 64), (4, 2, 64), (2, 2, 64)])
+def test_cache_codes_and_decode_outputs(Hq, Hkv, D):
+    lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3, 700, 2049], dtype=torch.int32)
+    w = W.Workload("fp8", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=97, kv_std=1.7)
+    harness, dw = _setup(w, lens, poison=True)
+    o, stored, si, pos = _oracle(dw, range(3))
+    # cache: codes and scales of every token of every owner layer, bit for bit
+    slots = W.slot_map_for(dw.page_table_cpu, si, pos, w.page_size).to(dw.device)
+    n = si.numel()
+    for l in dw.owners:
+        kc = torch.zeros((n, Hkv, D), dtype=torch.uint8, device=dw.device)
+        vc = torch.zeros_like(kc)
+        ks = torch.zeros((n, Hkv), dtype=torch.float32, device=dw.device)
+        vs = torch.zeros_like(ks)
+        dw.cache.skv_gather_fp8(l, slots, kc, vc, ks, vs)
+        torch.cuda.synchronize()
+        okc, ovc, oks, ovs = stored[l]
+        assert torch.equal(kc.cpu(), okc) and torch.equal(vc.cpu(), ovc)
+        assert torch.equal(ks.cpu().view(torch.int32), oks.view(torch.int32))
+        assert torch.equal(vs.cpu().view(torch.int32), ovs.view(torch.int32))
+    # attention of every layer
+    for l in range(3):
+        Q = harness.step_inputs(dw, l)["Q"]
+        out = torch.full((dw.batch, Hq, D), float("nan"), dtype=torch.bfloat16, device=dw.device)
+        dw.cache.skv_decode_attn(l, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+        torch.cuda.synchronize()
+        ref = o.decode_attn(l, Q.cpu(), dw.lens_cpu)
+        err = (out.cpu().double() - ref).abs()
+        assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {l}: max abs err {err.max().item()}"
+    assert dw.cache.skv_get_status() == 0
+    st = dw.cache.skv_cache_stats()
+    assert st["bytes_per_token"] == 2 * len(dw.owners) * Hkv * (D + 4)
+    assert st["page_bytes"] == Hkv * (2 * 16 * D + 128)
+
+
+def test_rows_of_very_different_magnitude():
+    """Per-row scales spanning 2^-20 .. 2^12 in one sequence: the scales are applied outside the f16
+    contractions, so neither overflow nor flush-to-zero may show.  With such a spread an output element
+    is a sum of terms thousands of times larger than itself wherever the big rows cancel, so the bound
+    here is taken relative to the largest element of the output row, not element by element."""
+    from paper_2604_22782_b200 import harness
+    from oracle import Oracle
+    lens = torch.tensor([300, 40], dtype=torch.int32)
+    w = W.Workload("fp8_mag", 1, 8, 2, 128, 16, 2, 0, 0, "explicit", explicit_r=(0,), seed=101)
+    dw = harness.setup(w, lens=lens, fp8=True)
+    si, pos = W.token_index(lens)
+    K, V = W.draw_kv(w, 0, si, pos)
+    g = torch.Generator().manual_seed(1)
+    mag = torch.exp2(torch.randint(-20, 13, (si.numel(), 1, 1), generator=g).float())
+    V = (V.float() * mag).to(torch.bfloat16)
+    K = (K.float() * torch.exp2(torch.randint(-3, 3, (si.numel(), 1, 1), generator=g).float())).to(torch.bfloat16)
+    slots = W.slot_map_for(dw.page_table_cpu, si, pos, w.page_size).to(dw.device)
+    dw.cache.skv_append(0, K.to(dw.device), V.to(dw.device), slots)
+    o = Oracle(1, [0], 8, 2, 128, 2, 300)
+    o.append_fp8(0, K, V, si, pos)
+    Q = harness.step_inputs(dw, 0)["Q"]
+    out = torch.empty((2, 8, 128), dtype=torch.bfloat16, device=dw.device)
+    dw.cache.skv_decode_attn(0, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+    torch.cuda.synchronize()
+    ref = o.decode_attn(0, Q.cpu(), lens)
+    err = (out.cpu().double() - ref).abs()
+    assert torch.isfinite(out.float()).all()
+    row_max = ref.abs().amax(dim=-1, keepdim=True)
+    assert bool((err <= ATOL + RTOL * row_max).all()), f"max abs err {err.max().item()} at |ref| up to {ref.abs().max().item()}"
+
+
+def test_whole_step_and_unsupported_calls():
+    from paper_2604_22782_b200 import harness
+    from paper_2604_22782_b200.binding import SKV_ERR_UNSUPPORTED, SkvError
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 0, 15], dtype=torch.int32)
+    w = W.Workload("fp8_step", 4, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2, 2), seed=103)
+    dw = harness.setup(w, lens=lens, fp8=True)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    o, _, _, _ = _oracle(dw, range(4))
+    for rep in range(2):
+        t["out"].fill_(float("nan"))
+        dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
+        torch.cuda.synchronize()
+        for l in range(4):
+            ref = o.decode_attn(l, t["Q"][l].cpu(), dw.lens_cpu)
+            err = (t["out"][l].cpu().double() - ref).abs()
+            assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"rep {rep} layer {l}: {err.max().item()}"
+    assert dw.cache.skv_get_status() == 0
+    with pytest.raises(SkvError) as e:
+        dw.cache.skv_gather(0, dw.slot_new, t["K"][0], t["V"][0])
+    assert e.value.status == SKV_ERR_UNSUPPORTED
+    inp = harness.prefill_inputs(dw, 0, torch.ones(lens.numel(), dtype=torch.int32))
+    with pytest.raises(SkvError) as e:
+        dw.cache.skv_prefill_attn(0, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, torch.empty_like(inp["Q"]), 1)
+    assert e.value.status == SKV_ERR_UNSUPPORTED
