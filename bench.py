@@ -354,6 +354,7 @@ def main():
         torch.cuda.empty_cache()
         line["sharing_sweep"] = sharing_sweep(args, dev)
         line["prefill"] = prefill_leg(args, dev)
+        line["fp8_pages"] = fp8_leg(args, dev)
     print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
@@ -410,6 +411,41 @@ def prefill_leg(args, dev):
     if dw.cache.skv_get_status() != 0:
         raise SystemExit("device status after the pre-fill leg")
     return res
+
+
+def fp8_leg(args, dev):
+    """The benchmark's workload with FP8 pages (E4M3 codes + one fp32 scale per token and kv head): whole
+    decode steps, cache bytes per token, and the rate in tokens attended per microsecond next to the bf16
+    cache's (the FP8 kernel converts codes on the way into the tensor cores and is bound by that, not by HBM)."""
+    from paper_2604_22782_b200 import harness
+    w = W.get_workload("llama3_8b")
+    dw = harness.setup(w, device=dev, fp8=True)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    cache = dw.cache
+
+    def step():
+        cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = max(3, args.steps // 2)
+    e0.record()
+    for _ in range(n):
+        step()
+    e1.record()
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / n
+    if cache.skv_get_status() != 0:
+        raise SystemExit("device status after the FP8 leg")
+    st = cache.skv_cache_stats()
+    tokens = int(dw.lens_cpu.sum())
+    return {"workload": w.name, "kv_bytes_per_token": st["bytes_per_token"], "ms_per_step": ms,
+            "us_per_attn_call": ms * 1e3 / w.n_layers,
+            "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
+            "tokens_attended_per_us": w.n_layers * tokens / (ms * 1e3)}
 
 
 def sharing_sweep(args, dev):
