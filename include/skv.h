@@ -318,11 +318,11 @@ int skv_decode_step(skv_cache *cache, const void *Q, const void *K, const void *
  * inputs to the device, runs append + decode attention for layers 0..L-1 in
  * order, and copies the outputs back.  Everything is ordered after the work
  * already on `stream`, and `stream` is complete only when the outputs are in
- * h_out (the caller synchronises `stream`); inside, the layers are cut into up
- * to four groups and a copy stream owned by the handle (created on the first
- * call, destroyed by skv_cache_destroy) moves one group's queries in and
- * another group's outputs out while a third group's kernels run.  Host buffers
- * should be pinned for the copies to be asynchronous.
+ * h_out (the caller synchronises `stream`); inside, the layers are cut into
+ * groups and a copy stream owned by the handle (created on the first call,
+ * destroyed by skv_cache_destroy) moves the next group's inputs in while a
+ * group's kernels run and takes each group's results back while the next group
+ * runs.  Host buffers should be pinned for the copies to be asynchronous.
  *   hQ          host bf16 [n_layers][batch][q_heads][head_dim]
  *   hK, hV      host bf16 [n_owners][batch][kv_heads][head_dim], owner layers
  *               in increasing layer order
@@ -382,6 +382,11 @@ int skv_set_decode_overlap(skv_cache *cache, int enabled);
  * 0 = every layer walks forward, everything evict-first.  Results do not depend
  * on it beyond floating-point summation order. */
 int skv_set_decode_l2_reuse(skv_cache *cache, int keep_percent);
+
+/* How skv_decode_step_host cuts the step: `groups` layer groups (1..8, default
+ * 4), of equal size (ramp 0) or with small first and last groups, whose copies
+ * nothing hides (ramp 1, default).  Results do not depend on either. */
+int skv_set_host_step(skv_cache *cache, int groups, int ramp);
 
 /* Tracing: while a device buffer of at least 32 * skv_decode_worker_count bytes
  * is set, every split-K launch records four uint64 per worker (warp): SM id,

@@ -76,6 +76,7 @@ lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
 lib.skv_set_prefill_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
+lib.skv_set_host_step.argtypes = [_vp, _int, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
 lib.skv_decode_worker_count.argtypes = [_vp]
 lib.skv_launch_count.argtypes = [_vp, ctypes.POINTER(_i64)]
@@ -361,6 +362,9 @@ class SkvCache:
 
     def skv_set_decode_l2_reuse(self, keep_percent: int) -> None:
         _check(lib.skv_set_decode_l2_reuse(self._h, keep_percent), "skv_set_decode_l2_reuse")
+
+    def skv_set_host_step(self, groups: int, ramp: int) -> None:
+        _check(lib.skv_set_host_step(self._h, groups, ramp), "skv_set_host_step")
 
     def skv_set_trace_buffer(self, buf: Optional[torch.Tensor]) -> None:
         _check(lib.skv_set_trace_buffer(self._h, _ptr(buf), 0 if buf is None else buf.numel() * buf.element_size()),

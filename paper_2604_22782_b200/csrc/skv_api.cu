@@ -34,7 +34,9 @@ struct skv_cache {
     size_t trace_bytes = 0;
     // skv_decode_step_host: a copy stream and events that let host<->device copies of one part of the
     // step run beside the kernels of another (created on first use, destroyed with the handle)
-    static constexpr int HOST_GROUPS = 4;
+    static constexpr int HOST_GROUPS = 8;
+    int host_groups = 4;            // layer groups of skv_decode_step_host
+    int host_ramp = 1;              // 1: small first and last groups (smoothstep cut), 0: equal groups
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_entry = nullptr, ev_exit = nullptr, ev_in[HOST_GROUPS] = {}, ev_done[HOST_GROUPS] = {};
 
@@ -585,12 +587,18 @@ extern "C" {
 
 namespace {
 // The updates of every owner layer of one step in one launch.  K, V: [n_owners][batch][kv_heads][head_dim].
-int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot_map, int batch, void *stream)
+int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot_map, int batch, void *stream,
+                 int first_owner = 0, int n_upd = -1)
 {
     if (!aligned(K, 16) || !aligned(V, 16)) return SKV_ERR_ARG;
+    if (n_upd < 0) n_upd = c->n_owners - first_owner;
+    if (n_upd == 0) return SKV_OK;
+    const size_t kv_off = (size_t)first_owner * batch * c->kv_heads * c->head_dim * 2;
+    K = static_cast<const uint8_t *>(K) + kv_off;
+    V = static_cast<const uint8_t *>(V) + kv_off;
     if (c->fp8) {
         AppendFp8Params q;
-        q.layer_base = c->layer_base(0);
+        q.layer_base = c->layer_base(first_owner);
         q.K = static_cast<const uint16_t *>(K);
         q.V = static_cast<const uint16_t *>(V);
         q.slot_map = slot_map;
@@ -601,7 +609,7 @@ int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot
         q.Hkv = c->kv_heads;
         q.D = c->head_dim;
         q.status = c->status_word();
-        if (launch_append_fp8(q, c->n_owners, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        if (launch_append_fp8(q, n_upd, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
             (void)cudaGetLastError();
             return SKV_ERR_CUDA;
         }
@@ -609,7 +617,7 @@ int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot
         return SKV_OK;
     }
     AppendParams ap;
-    ap.layer_base = c->layer_base(0);
+    ap.layer_base = c->layer_base(first_owner);
     ap.K = static_cast<const uint4 *>(K);
     ap.V = static_cast<const uint4 *>(V);
     ap.slot_map = slot_map;
@@ -620,7 +628,7 @@ int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot
     ap.Hkv = c->kv_heads;
     ap.D = c->head_dim;
     ap.status = c->status_word();
-    if (launch_append(ap, c->n_owners, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    if (launch_append(ap, n_upd, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;
     }
@@ -837,21 +845,42 @@ int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const voi
     uint8_t *ho = static_cast<uint8_t *>(h_out);
     const size_t q_layer = (size_t)batch * q_heads * c->head_dim * 2;
     const size_t kv_layer = (size_t)batch * c->kv_heads * c->head_dim * 2;
-    const int L = c->n_layers, NG = L < skv_cache::HOST_GROUPS ? L : skv_cache::HOST_GROUPS;
-    auto first_layer = [&](int g) { return (int)(((int64_t)g * L) / NG); };
-    // The layers are cut into NG groups.  Copy stream: small inputs, then the queries group by group;
-    // caller's stream: the kernels of a group as soon as its queries have arrived; copy stream again: a
-    // group's output rows as soon as its kernels are done.  So only the first group's inputs and the
-    // last group's outputs are not hidden behind kernels.
+    const int L = c->n_layers;
+    // The layers are cut into NG groups.  Copy stream: the small inputs, then group by group the new K,V
+    // rows of the group's owners and its queries; caller's stream: a group's kernels as soon as its inputs
+    // have arrived; copy stream again: a group's result rows as soon as its kernels are done.  So only the
+    // first group's inputs and the last group's results are not hidden behind kernels, and those two groups
+    // are the small ones (cut points on a smoothstep curve).
+    const int NG = L < c->host_groups ? L : c->host_groups;
+    int bound[skv_cache::HOST_GROUPS + 1];
+    bound[0] = 0;
+    for (int g = 1; g <= NG; ++g) {
+        const double x = (double)g / NG;
+        int64_t b = c->host_ramp ? (int64_t)(L * x * x * (3.0 - 2.0 * x) + 0.5) : ((int64_t)g * L) / NG;
+        if (b < bound[g - 1] + 1) b = bound[g - 1] + 1;
+        if (b > L - (NG - g)) b = L - (NG - g);
+        bound[g] = (int)b;
+    }
+    bound[NG] = L;
+    auto owners_before = [&](int l) { int n = 0; for (int i = 0; i < l; ++i) n += c->slot[(size_t)i] >= 0; return n; };
+    const bool batched = c->tune.pdl != 0;
     bool ok = cudaEventRecord(c->ev_entry, st) == cudaSuccess;             // staging may still be in use by
     ok = ok && cudaStreamWaitEvent(cs, c->ev_entry, 0) == cudaSuccess;     // earlier work on the caller's stream
     ok = ok && cudaMemcpyAsync(d + s.slot_map, h_slot_map, (size_t)batch * 8, cudaMemcpyHostToDevice, cs) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(d + s.page_table, h_page_table, (size_t)batch * pt_stride * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(d + s.seq_lens, h_seq_lens, (size_t)batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d + s.k, hK, kv_layer * c->n_owners, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d + s.v, hV, kv_layer * c->n_owners, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    // K,V rows: those of the first group's owners with the first group, all the others with the second, so
+    // that the updates are two launches at most and the attention launches of a group stay one chain.
+    const int own0 = owners_before(bound[1]);
     for (int g = 0; ok && g < NG; ++g) {
-        const int l0 = first_layer(g), l1 = first_layer(g + 1);
+        const int l0 = bound[g], l1 = bound[g + 1];
+        const int o0 = g == 0 ? 0 : own0, o1 = g == 0 ? own0 : c->n_owners;
+        if (g < 2 && o1 > o0) {
+            ok = ok && cudaMemcpyAsync(d + s.k + o0 * kv_layer, static_cast<const uint8_t *>(hK) + o0 * kv_layer,
+                                       (size_t)(o1 - o0) * kv_layer, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(d + s.v + o0 * kv_layer, static_cast<const uint8_t *>(hV) + o0 * kv_layer,
+                                       (size_t)(o1 - o0) * kv_layer, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+        }
         ok = ok && cudaMemcpyAsync(d + s.q + l0 * q_layer, hq + l0 * q_layer, (size_t)(l1 - l0) * q_layer,
                                    cudaMemcpyHostToDevice, cs) == cudaSuccess;
         ok = ok && cudaEventRecord(c->ev_in[g], cs) == cudaSuccess;
@@ -860,12 +889,12 @@ int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const voi
     const int64_t *slot_map = reinterpret_cast<const int64_t *>(d + s.slot_map);
     const int32_t *page_table = reinterpret_cast<const int32_t *>(d + s.page_table);
     const int32_t *seq_lens = reinterpret_cast<const int32_t *>(d + s.seq_lens);
-    const bool batched = c->tune.pdl != 0;
     for (int g = 0; g < NG; ++g) {
-        const int l0 = first_layer(g), l1 = first_layer(g + 1);
+        const int l0 = bound[g], l1 = bound[g + 1];
         if (cudaStreamWaitEvent(st, c->ev_in[g], 0) != cudaSuccess) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
-        if (g == 0 && batched) {
-            rc = step_updates(c, d + s.k, d + s.v, slot_map, batch, stream);
+        if (g < 2 && batched) {
+            rc = g == 0 ? step_updates(c, d + s.k, d + s.v, slot_map, batch, stream, 0, own0)
+                        : step_updates(c, d + s.k, d + s.v, slot_map, batch, stream, own0, c->n_owners - own0);
             if (rc) return rc;
         }
         rc = step_layers(c, l0, l1, d + s.q, d + s.k, d + s.v, slot_map, page_table, seq_lens, d + s.out, batch,
@@ -881,6 +910,14 @@ int skv_decode_step_host(skv_cache *c, const void *hQ, const void *hK, const voi
     ok = cudaEventRecord(c->ev_exit, cs) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(st, c->ev_exit, 0) == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); return SKV_ERR_CUDA; }
+    return SKV_OK;
+}
+
+int skv_set_host_step(skv_cache *c, int groups, int ramp)
+{
+    if (!c || groups < 1 || groups > skv_cache::HOST_GROUPS || ramp < 0 || ramp > 1) return SKV_ERR_ARG;
+    c->host_groups = groups;
+    c->host_ramp = ramp;
     return SKV_OK;
 }
 

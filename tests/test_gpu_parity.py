@@ -164,11 +164,18 @@ def test_whole_step_entry_points_match_the_oracle(overlap, l2_keep, Hq, Hkv, D):
     hb = harness.step_tensors(dw, device="cpu", pin=True)
     staging = torch.empty(dw.cache.skv_decode_step_staging_bytes(dw.batch, w.q_heads, dw.page_table_cpu.shape[1]),
                           dtype=torch.uint8, device=dw.device)
-    dw.cache.skv_decode_step_host(hb["Q"], hb["K"], hb["V"], dw.slot_new.cpu().pin_memory(),
-                                  dw.page_table_cpu.contiguous().pin_memory(), dw.lens_cpu.contiguous().pin_memory(),
-                                  hb["out"], staging)
-    torch.cuda.synchronize()
-    assert torch.equal(hb["out"].view(torch.int16), t["out"].cpu().view(torch.int16))
+    h_slot, h_pt, h_len = (dw.slot_new.cpu().pin_memory(), dw.page_table_cpu.contiguous().pin_memory(),
+                           dw.lens_cpu.contiguous().pin_memory())
+    pageable_out = torch.empty_like(hb["out"], pin_memory=False)
+    # every cut of the step, into pinned or pageable result buffers: one answer
+    for groups, direct, h_out in ((4, 1, hb["out"]), (4, 0, hb["out"]), (1, 1, hb["out"]), (8, 1, hb["out"]),
+                                  (3, 0, hb["out"]), (5, 1, pageable_out)):
+        dw.cache.skv_set_host_step(groups, direct)
+        h_out.fill_(float("nan"))
+        dw.cache.skv_decode_step_host(hb["Q"], hb["K"], hb["V"], h_slot, h_pt, h_len, h_out, staging)
+        torch.cuda.synchronize()
+        assert dw.cache.skv_get_status() == 0
+        assert torch.equal(h_out.view(torch.int16), t["out"].cpu().view(torch.int16)), (groups, direct)
     # the updates really happened: the newest token of every owner layer reads back bit-exactly
     has = dw.slot_new >= 0
     for i, l in enumerate(dw.owners):
