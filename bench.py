@@ -192,6 +192,8 @@ def main():
     ap.add_argument("--tuning", default="", help="warps,stages,ctas_per_sm of the split-K kernel")
     ap.add_argument("--overlap", type=int, default=-1, help="1 = overlappable (chained) launches, 0 = plain launches")
     ap.add_argument("--l2-keep", type=int, default=-1, help="percent of each block range kept in L2 for the next layer")
+    ap.add_argument("--fp8", action="store_true", help="run the main legs on FP8 pages (profiling the FP8 kernel); "
+                    "the byte counts are then those of the FP8 cache")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sharing-ratio sweep (owner fractions 1, 1/2, 1/4, 1/8)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -210,7 +212,7 @@ def main():
 
     from paper_2604_22782_b200 import harness
     w = rank_workload(w, rank, world)
-    dw = harness.setup(w, device=dev)
+    dw = harness.setup(w, device=dev, fp8=args.fp8)
     dw.retune(variant=args.variant or None,
               tuning=[int(x) for x in args.tuning.split(",")] if args.tuning else None,
               overlap=args.overlap if args.overlap >= 0 else None,
@@ -313,7 +315,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "dtype": "e4m3 pages, f16 contractions" if args.fp8 else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "family": w.family, "n_layers": L, "owners": n_own, "batch": dw.batch,
                    "tokens": int(dw.lens_cpu.sum()), "q_heads": w.q_heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size,
@@ -331,7 +333,7 @@ def main():
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "us_per_launch": us_per_launch,
                      "bytes_per_launch": attn_bytes,
                      "how": "whole steps with L2 reuse between layers off; timed region / split-K launches in it",
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+                     "traffic": None if args.fp8 else NCU_TRAFFIC_BYTES.get(w.name)},
         "single_call": {"us_owner_layers": call_ms_owner * 1e3,
                         "us_reader_layers": None if call_ms_reader is None else call_ms_reader * 1e3,
                         "gbs_owner_layers": attn_bytes / (call_ms_owner * 1e-3) / 1e9,

@@ -248,6 +248,7 @@ int create_impl(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, i
         }
     c->n_owners = (int)c->owners.size();
     c->fp8 = fp8;
+    if (fp8) c->tune.ctas_per_sm = 6;          // the FP8 kernel is bound by instruction latency: 12 warps per SM
     c->page_bytes = page_bytes_of(kv_heads, head_dim, fp8);
     plan_walks(c);
     c->pool = static_cast<uint8_t *>(device_pool);

@@ -407,15 +407,20 @@ struct Fp8State {
         cs = cs_new;
         const uint32_t pa0 = pack_f16x2(p0 * (sv.x * inv_cs), p1 * (sv.y * inv_cs));
         const uint32_t pa2 = pack_f16x2(p2 * (sv.z * inv_cs), p3 * (sv.w * inv_cs));
+        if (__any_sync(FULL, alpha != 1.f)) {              // rare once the running maximum has settled
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] *= alpha; o[nt][1] *= alpha; }
+        }
         // ---- O += P' Vc ----
         const uint32_t v_lane = blk + (uint32_t)(fp8_v_off(D) + g * PAGE + 4 * tig);
+        uint32_t vw[D / 8];                    // all loads first: the volatile loads keep their order
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt)
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(vw[nt]) : "r"(v_lane + (uint32_t)(nt * 8 * PAGE)));
 #pragma unroll
         for (int nt = 0; nt < D / 8; ++nt) {
-            uint32_t w;
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(v_lane + (uint32_t)(nt * 8 * PAGE)));
             uint32_t b0, b1;
-            e4m3x4_to_f16x2(w & vmask, b0, b1);
-            o[nt][0] *= alpha; o[nt][1] *= alpha;
+            e4m3x4_to_f16x2(vw[nt] & vmask, b0, b1);
             mma_f16_16816(o[nt], pa0, 0u, pa2, 0u, b0, b1);
         }
     }
