@@ -293,7 +293,7 @@ struct CudaCoreState {
 // in f16, which holds every E4M3 value exactly.  Per page  S = (Q/qmax) Kc^T  and  O += P' Vc  on
 // the raw codes; the per-token scales are applied outside the contractions:
 //   score_t = qmax * kscale_t * S_t,      P'_t = p_t * vscale_t / c,
-// with c a power of two >= every vscale seen so far (so P' <= 1 fits f16 whatever the magnitudes;
+// with c a power of two >= every vscale seen so far (so P' <= 256 fits f16 whatever the magnitudes;
 // when c grows O is scaled down with the softmax's own rescaling factor), and O * c at the end.
 // Fragments come straight from shared memory without transposes because the contraction order
 // within a k-step is free as long as both operands agree: a thread's k-slots {2tig,2tig+1,
@@ -390,7 +390,11 @@ struct Fp8State {
         float mx = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
         mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
-        const float m_new = fmaxf(m, mx);                 // finite: every page has a valid token
+        // The reference m only follows the running maximum when that has grown by more than 2^8 (m is then
+        // finite: every page has a valid token): until then the probabilities are at most 256, which f16
+        // and the fp32 sums hold easily, and nothing has to be rescaled.  The result does not depend on
+        // the reference.
+        const float m_new = mx > m + 8.f ? mx : m;
         float alpha = fast_exp2(m - m_new);
         const float p0 = fast_exp2(v0 - m_new), p1 = fast_exp2(v1 - m_new);
         const float p2 = fast_exp2(v2 - m_new), p3 = fast_exp2(v3 - m_new);
