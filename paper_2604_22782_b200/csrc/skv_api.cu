@@ -100,7 +100,14 @@ WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int
     return w;
 }
 
-int n_workers_of(const skv_cache *c) { return c->sm_count * c->tune.ctas_per_sm * c->tune.warps; }
+// FP8 pages go to the tcgen05 kernel (a worker is a CTA there) unless the mma.sync variant is asked for
+bool fp8_on_umma(const skv_cache *c) { return c->fp8 && c->tune.variant != 2 && decode_fp8_umma_supported(c->head_dim, 1); }
+
+int n_workers_of(const skv_cache *c)
+{
+    if (fp8_on_umma(c)) return c->sm_count * decode_fp8_umma_ctas_per_sm();
+    return c->sm_count * c->tune.ctas_per_sm * c->tune.warps;
+}
 
 // Walk directions for L2 reuse: a layer that reads the same owner as the layer before it walks every
 // block range in the opposite direction, so that it starts on the blocks its predecessor read last.
@@ -468,7 +475,9 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
         warps = 1;
         ctas = 8;
     }
-    const size_t smem = decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages, c->fp8);
+    const bool umma = fp8_on_umma(c) && decode_fp8_umma_supported(c->head_dim, G);
+    const size_t smem = umma ? decode_fp8_umma_smem_bytes(c->head_dim, batch)
+                             : decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages, c->fp8);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
@@ -497,8 +506,10 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.status = c->status_word();
     p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
     const int grid = c->sm_count * ctas;
-    const cudaError_t le = launch_decode_splitk(p, c->head_dim, G, c->fp8 ? 2 : tensor_core ? 1 : 0, grid, warps, c->tune.stages,
-                                                c->tune.pdl != 0, st);
+    const cudaError_t le =
+        umma ? launch_decode_fp8_umma(p, c->head_dim, G, W, c->tune.pdl != 0, st)
+             : launch_decode_splitk(p, c->head_dim, G, c->fp8 ? 2 : tensor_core ? 1 : 0, grid, warps, c->tune.stages,
+                                    c->tune.pdl != 0, st);
     if (le != cudaSuccess) {
         (void)cudaGetLastError();
         // a launch shape with more warps per CTA than the register file holds for this kernel variant

@@ -115,8 +115,8 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Param
     const uint32_t c01 = pack_e4m3x2(__fmul_rn(x[0], inv), __fmul_rn(x[1], inv));
     const uint32_t c23 = pack_e4m3x2(__fmul_rn(x[2], inv), __fmul_rn(x[3], inv));
     uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
-    if (which == 0) {                                  // K: token-major rows
-        uint8_t *dst = blk + off * D + lane * PER;
+    if (which == 0) {                                  // K: a lane's dims are neighbours inside one 16-byte piece
+        uint8_t *dst = blk + fp8_k_pos(D, off, lane * PER);
         if (PER == 4) *reinterpret_cast<uint32_t *>(dst) = c01 | (c23 << 16);
         else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)c01;
     } else {                                           // V: dim-major, this token's column
@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(COPY_THREADS) gather_fp8_kernel(GatherFp8Param
     const uint8_t *blk = p.layer_base + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
     uint8_t *out = (which ? p.V_codes : p.K_codes) + (tok * p.Hkv + h) * D;
     for (int d = lane; d < D; d += 32)
-        out[d] = which ? blk[fp8_v_off(D) + d * PAGE + off] : blk[off * D + d];
+        out[d] = which ? blk[fp8_v_off(D) + d * PAGE + off] : blk[fp8_k_pos(D, off, d)];
     if (lane == 0)
         (which ? p.V_scales : p.K_scales)[tok * p.Hkv + h] =
             *reinterpret_cast<const float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * off);

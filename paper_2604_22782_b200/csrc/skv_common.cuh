@@ -23,9 +23,14 @@ __host__ __device__ constexpr int half_bytes(int D) { return PAGE * D * 2; }
 __host__ __device__ constexpr int block_bytes(int D) { return 2 * half_bytes(D); }
 
 // FP8 pages (E4M3 codes, one fp32 scale per (token, kv head) row for K and for V).  The block of
-// one (page, kv head):  K codes [PAGE tokens][D] | V codes [D dims][PAGE tokens] | K scales [PAGE]
-// fp32 | V scales [PAGE] fp32.  K is token-major and V dim-major so that the decode kernel's tensor-
-// core fragments are plain 32-bit / 128-bit shared-memory loads (see Fp8State in skv_decode.cu).
+// one (page, kv head):  K codes | V codes | K scales [PAGE] fp32 | V scales [PAGE] fp32.
+//   K codes: [2 groups of 8 tokens][D/16 chunks of 16 dims][8 tokens][16 B]
+//   V codes: [D dims][PAGE tokens]  =  [D/8 groups of 8 dims][8 dims][16 B]
+// Both are the tensor cores' K-major core-matrix layout (8 rows x 16 bytes, contiguous) for the
+// operand they are used as: K with the tokens as rows and the dims contracted, V^T with the dims as
+// rows and the tokens contracted (see skv_decode_fp8_umma.cu); the mma.sync kernel reads the same
+// layout with plain shared-memory loads (Fp8State in skv_decode.cu).
+__host__ __device__ constexpr int fp8_k_pos(int D, int t, int d) { return (t >> 3) * 8 * D + (d >> 4) * 128 + (t & 7) * 16 + (d & 15); }
 __host__ __device__ constexpr int fp8_v_off(int D) { return PAGE * D; }
 __host__ __device__ constexpr int fp8_ks_off(int D) { return 2 * PAGE * D; }
 __host__ __device__ constexpr int fp8_vs_off(int D) { return 2 * PAGE * D + PAGE * 4; }
@@ -146,6 +151,11 @@ struct DecodeTuning {
 // host launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s);
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
+// decode attention over FP8 pages on tcgen05 (skv_decode_fp8_umma.cu): a worker is a CTA, grid = worker count
+bool decode_fp8_umma_supported(int D, int G);
+int decode_fp8_umma_ctas_per_sm();
+size_t decode_fp8_umma_smem_bytes(int D, int B);
+cudaError_t launch_decode_fp8_umma(const DecodeParams &p, int D, int G, int grid, bool pdl, cudaStream_t s);
 cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s);
 cudaError_t launch_gather_fp8(const GatherFp8Params &p, cudaStream_t s);
 // smem bytes the split-K kernel needs for this shape, or 0 if unsupported

@@ -14,6 +14,7 @@
 // kernel (one warp per segment) combines a segment's partials; it is launched
 // so that it is already resident, waiting, when the split-K kernel ends.
 #include "skv_common.cuh"
+#include "skv_walk.cuh"
 
 #include <math.h>
 
@@ -23,55 +24,6 @@ namespace {
 
 constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr int WIN = 128;   // page ids a warp keeps in registers (4 per lane)
-
-struct Cursor {        // a position in the flattened (b, h, page) list
-    int b, h, pg, pages;
-};
-
-__device__ __forceinline__ Cursor locate(const int32_t *prefix, int B, int Hkv, int64_t x)
-{
-    int lo = 0, hi = B - 1;   // smallest b with prefix[b+1]*Hkv > x
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if ((int64_t)prefix[mid + 1] * Hkv > x) hi = mid; else lo = mid + 1;
-    }
-    Cursor c;
-    c.b = lo;
-    c.pages = prefix[lo + 1] - prefix[lo];
-    const int64_t r = x - (int64_t)prefix[lo] * Hkv;
-    c.h = (int)(r / c.pages);
-    c.pg = (int)(r - (int64_t)c.h * c.pages);
-    return c;
-}
-
-// One position forward (or backward).  Only called while another position remains in that
-// direction, so b stays inside [0, B).
-__device__ __forceinline__ void step(Cursor &c, const int32_t *prefix, int Hkv, bool reverse)
-{
-    if (!reverse) {
-        if (++c.pg < c.pages) return;
-        c.pg = 0;
-        if (++c.h < Hkv) return;
-        c.h = 0;
-        do {
-            ++c.b;
-            c.pages = prefix[c.b + 1] - prefix[c.b];
-        } while (c.pages == 0);
-    } else {
-        if (--c.pg >= 0) return;
-        if (--c.h < 0) {
-            c.h = Hkv - 1;
-            do {
-                --c.b;
-                c.pages = prefix[c.b + 1] - prefix[c.b];
-            } while (c.pages == 0);
-        }
-        c.pg = c.pages - 1;
-    }
-}
-
-// Shared-memory carve-up (dynamic): prefix[B+1] | lens[B] | rings | barriers | CTA arrival word
-__host__ __device__ inline size_t table_bytes(int B) { return (((size_t)(2 * B + 1) * 4) + 127) & ~(size_t)127; }
 
 // ---------------------------------------------------------------------------
 // Per-warp compute state, tensor-core variant: the G query heads of one kv head
@@ -299,7 +251,8 @@ struct CudaCoreState {
 // within a k-step is free as long as both operands agree: a thread's k-slots {2tig,2tig+1,
 // 2tig+8,2tig+9} carry FOUR CONSECUTIVE dims (QK^T) or tokens (PV), i.e. one 32-bit word of codes.
 //   QK^T: thread (g = lane/4, tig) reads token rows 4*(g/2) + g%2 (+2 for the second 8-column tile),
-//         bytes [D/4*tig, D/4*(tig+1)), so that its four scores are tokens 4tig .. 4tig+3;
+//         dims [D/4*tig, D/4*(tig+1)) (K is stored in 8-token x 16-dim pieces, see fp8_k_pos), so
+//         that its four scores are tokens 4tig .. 4tig+3;
 //   PV:   V is stored dim-major, the word at dim 8*tile + g, byte 4*tig holds tokens 4tig .. 4tig+3.
 // ---------------------------------------------------------------------------
 template <int D>
@@ -353,14 +306,16 @@ struct Fp8State {
         const int g = lane >> 2, tig = lane & 3;
         // ---- scores of tokens 4tig .. 4tig+3 for query head g ----
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t k0 = blk + (uint32_t)((4 * (g >> 1) + (g & 1)) * D + DT * tig), k1 = k0 + 2 * D;
+        // token rows 4 (g/2) + g%2 and that + 2 (the same group of 8 tokens), 16-dim chunks (D/64) tig + c
+        const int tok = 4 * (g >> 1) + (g & 1);
+        const uint32_t k0 = blk + (uint32_t)((tok >> 3) * 8 * D + (DT / 16) * tig * 128 + (tok & 7) * 16), k1 = k0 + 2 * 16;
         uint32_t w0[DT / 4], w1[DT / 4];
 #pragma unroll
         for (int c = 0; c < DT / 16; ++c) {
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(w0[4 * c]), "=r"(w0[4 * c + 1]), "=r"(w0[4 * c + 2]), "=r"(w0[4 * c + 3]) : "r"(k0 + 16 * c));
+                         : "=r"(w0[4 * c]), "=r"(w0[4 * c + 1]), "=r"(w0[4 * c + 2]), "=r"(w0[4 * c + 3]) : "r"(k0 + 128 * c));
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(w1[4 * c]), "=r"(w1[4 * c + 1]), "=r"(w1[4 * c + 2]), "=r"(w1[4 * c + 3]) : "r"(k1 + 16 * c));
+                         : "=r"(w1[4 * c]), "=r"(w1[4 * c + 1]), "=r"(w1[4 * c + 2]), "=r"(w1[4 * c + 3]) : "r"(k1 + 128 * c));
         }
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
@@ -443,17 +398,6 @@ struct Fp8State {
         }
     }
 };
-
-// ---------------------------------------------------------------------------
-// Where the partials of a segment live.  The segment's blocks are [s0, s0 + pages) of the flattened
-// list.  Normally worker w writes the partial of its run inside segment seg to slot  w + seg, so a
-// segment's partials sit in consecutive slots.  When there are fewer blocks than workers every
-// non-empty range is a single block x, and its partial goes to slot  x + seg  (consecutive again).
-// ---------------------------------------------------------------------------
-__device__ __forceinline__ int partial_slot(int64_t T, int64_t W, int64_t w, int64_t x_any, int64_t seg)
-{
-    return (int)((T < W ? x_any : w) + seg);
-}
 
 __device__ __forceinline__ void segment_partials(int64_t T, int64_t W, int64_t seg, int64_t s0, int pages, int &slot0,
                                                  int &n)

@@ -32,11 +32,15 @@ def _oracle(dw, layers):
     return o, stored, si, pos
 
 
-@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 64), (4, 2, 64), (2, 2, 64)])
-def test_cache_codes_and_decode_outputs(Hq, Hkv, D):
-    lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3, 700, 2049], dtype=torch.int32)
+@pytest.mark.parametrize("variant", [0, 2])      # 0: tcgen05 kernel where it applies (head_dim 128), 2: mma.sync kernel
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 128), (6, 2, 64), (4, 2, 64), (2, 2, 64)])
+def test_cache_codes_and_decode_outputs(Hq, Hkv, D, variant):
+    if variant == 2 and D == 64:
+        pytest.skip("head_dim 64 runs the mma.sync kernel under either setting")
+    lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3, 700, 2049, 129, 256, 112], dtype=torch.int32)
     w = W.Workload("fp8", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=97, kv_std=1.7)
     harness, dw = _setup(w, lens, poison=True)
+    dw.retune(variant=variant)
     o, stored, si, pos = _oracle(dw, range(3))
     # cache: codes and scales of every token of every owner layer, bit for bit
     slots = W.slot_map_for(dw.page_table_cpu, si, pos, w.page_size).to(dw.device)
@@ -107,7 +111,8 @@ def test_whole_step_and_unsupported_calls():
     harness.prefill(dw, upto_offset=-1)
     t = harness.step_tensors(dw)
     o, _, _, _ = _oracle(dw, range(4))
-    for rep in range(2):
+    for rep in range(3):
+        dw.retune(l2_keep=(35, 0, 60)[rep])      # layers 1 and 3 walk backward unless L2 reuse is off
         t["out"].fill_(float("nan"))
         dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
         torch.cuda.synchronize()
