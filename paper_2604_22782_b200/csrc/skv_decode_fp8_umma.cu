@@ -138,6 +138,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity)
     if (try_wait_for(bar, parity, 2000u)) return true;
     const uint64_t t0 = global_timer_ns();
     for (;;) {
+        __nanosleep(64);
         if (try_wait_for(bar, parity, 10000u)) return true;
         if (global_timer_ns() - t0 > 2000000000ull) return false;
     }
@@ -148,7 +149,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-template <int D>
+template <int D, int GP>   // GP: the group size rounded up to a power of two (the softmax loops run over GP heads)
 // (bounds as for four CTAs per SM = 80 registers: shared memory admits three, and the registers left over let
 // a CTA of the merge kernel become resident beside them, which the launch chain needs to move on)
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kernel(DecodeParams p, int G)
@@ -428,6 +429,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                         tc_commit(k_empty + 8 * s);
                         qk_issued = true;
                     }
+                    if (!(qk_issued && pv_issued)) __nanosleep(32);
                     if ((spin & 63) == 63 && global_timer_ns() - t0 > 2000000000ull) ok = false;
                 }
                 if (!ok) break;
@@ -446,9 +448,9 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
         // ================= softmax (warps 0-3) =================
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         const int j = tid >> 4, tt = tid & 15;           // page slot and token-in-page of this thread's token
-        float m_ref[8], l_sum[8], qs[8];
+        float m_ref[GP], l_sum[GP], qs[GP];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) { m_ref[h] = -INFINITY; l_sum[h] = 0.f; qs[h] = 0.f; }
+        for (int h = 0; h < GP; ++h) { m_ref[h] = -INFINITY; l_sum[h] = 0.f; qs[h] = 0.f; }
         float cs = 0.f;
         int runs = 0;
         bool ok = true;
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 wait_bounded(q_full, (uint32_t)(runs & 1));     // already over: the scores used Q'
                 ++runs;
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
+                for (int h = 0; h < GP; ++h) {
                     m_ref[h] = -INFINITY;
                     l_sum[h] = 0.f;
                     qs[h] = reinterpret_cast<volatile float *>(qscale)[m.qbuf * 8 + h];
@@ -481,17 +483,15 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 ksc = *reinterpret_cast<const float *>(vpage + K_PAGE + 4 * tt);
                 vsc = *reinterpret_cast<const float *>(vpage + K_PAGE + 4 * PAGE + 4 * tt);
             }
-            float sc[8];
+            float sc[GP];                  // (heads G..GP-1 have zero queries: their scores are 0, their results unused)
 #pragma unroll
-            for (int h = 0; h < 8; ++h)
-                sc[h] = (valid && h < G) ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * (ksc * qs[h]) : -INFINITY;
+            for (int h = 0; h < GP; ++h)
+                sc[h] = valid ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * (ksc * qs[h]) : -INFINITY;
             // maxima over the tile's 128 tokens: per head, and of the V scales
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h < G) {
-                    const int mk = warp_max_s32(float_key(sc[h]));
-                    if (lane == 0) red[s * 64 + h * 4 + warp] = mk;
-                }
+            for (int h = 0; h < GP; ++h) {
+                const int mk = warp_max_s32(float_key(sc[h]));
+                if (lane == 0) red[s * 64 + h * 4 + warp] = mk;
             }
             {
                 const int mk = warp_max_s32(__float_as_int(vsc));      // scales are >= 0: their bits order them
@@ -500,18 +500,15 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
             ok = softmax_all(ok);          // the maxima are in place; and has every thread's wait ended normally?
             if (!ok) break;
             bool changed = false;
-            float alpha[8];                // factor that moves a head's sums to its new reference
+            float alpha[GP];               // factor that moves a head's sums to its new reference
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                alpha[h] = 1.f;
-                if (h < G) {
-                    const int4 r = *reinterpret_cast<const int4 *>(red + s * 64 + h * 4);      // the four warps' maxima
-                    const float mx = key_float(max(max(r.x, r.y), max(r.z, r.w)));           // finite: every tile has a valid token
-                    const float m_new = mx > m_ref[h] + RESCALE_STEP ? mx : m_ref[h];
-                    alpha[h] = fast_exp2(m_ref[h] - m_new);
-                    changed = changed || (m_new != m_ref[h]);
-                    m_ref[h] = m_new;
-                }
+            for (int h = 0; h < GP; ++h) {
+                const int4 r = *reinterpret_cast<const int4 *>(red + s * 64 + h * 4);      // the four warps' maxima
+                const float mx = key_float(max(max(r.x, r.y), max(r.z, r.w)));           // finite: every tile has a valid token
+                const float m_new = mx > m_ref[h] + RESCALE_STEP ? mx : m_ref[h];
+                alpha[h] = fast_exp2(m_ref[h] - m_new);
+                changed = changed || (m_new != m_ref[h]);
+                m_ref[h] = m_new;
             }
             float wp, ca;
             {
@@ -537,24 +534,23 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 tmem_ld16(lane_base + COL_O, ov);
                 tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 16; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * (alpha[c & 7] * ca));
+                for (int c = 0; c < 16; ++c)
+                    if ((c & 7) < GP) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * (alpha[(c & 7) % GP] * ca));
                 tmem_st16(lane_base + COL_O, ov);
                 tmem_wait_st();
             }
             // probabilities, split into two E4M3 terms; bytes of token (j, tt): [j][term][head][tt]
             uint8_t *parea = p_sm_ptr + s * P_BYTES + j * 256 + tt;
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h < G) {
-                    const float pr = fast_exp2(sc[h] - m_ref[h]);       // 0 for a token that is not in use
-                    const float pp = pr * (vsc * wp);
-                    const float lead = __uint_as_float(__float_as_uint(pp) & 0xFFF00000u);   // E4M3's three mantissa bits
-                    const float rem = (pp - lead) * REM_SCALE;                                 // < 8 * 32 at the top binade
-                    const uint32_t codes = pack_e4m3x2(lead, rem);       // low byte: leading term, high byte: remainder
-                    parea[h * 16] = (uint8_t)(codes & 0xFFu);
-                    parea[128 + h * 16] = (uint8_t)(codes >> 8);
-                    l_sum[h] = l_sum[h] * alpha[h] + pr;
-                }
+            for (int h = 0; h < GP; ++h) {
+                const float pr = fast_exp2(sc[h] - m_ref[h]);       // 0 for a token that is not in use
+                const float pp = pr * (vsc * wp);
+                const float lead = __uint_as_float(__float_as_uint(pp) & 0xFFF00000u);   // E4M3's three mantissa bits
+                const float rem = (pp - lead) * REM_SCALE;                                 // < 8 * 32 at the top binade
+                const uint32_t codes = pack_e4m3x2(lead, rem);       // low byte: leading term, high byte: remainder
+                parea[h * 16] = (uint8_t)(codes & 0xFFu);
+                parea[128 + h * 16] = (uint8_t)(codes >> 8);
+                l_sum[h] = l_sum[h] * alpha[h] + pr;
             }
             // V codes the tensor core will read but that belong to no token in use must be finite too: the
             // unused slots of the sequence's last page may hold anything, and an odd tile reads one page
@@ -588,27 +584,25 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 tmem_ld16(lane_base + COL_O, ov);
                 tmem_wait_ld();
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < G) {
-                        float v = l_sum[h];
+                for (int h = 0; h < GP; ++h) {
+                    float v = l_sum[h];
 #pragma unroll
-                        for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(FULL, v, d);
-                        if (lane == 0) red_l[warp * 8 + h] = v;
-                    }
+                    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(FULL, v, d);
+                    if (lane == 0) red_l[warp * 8 + h] = v;
                 }
                 softmax_sync();
                 const int64_t seg = (int64_t)m.b * p.Hkv + m.h;
                 const int64_t slot = partial_slot(T, W, w, x0, seg);
                 const float back = cs * (1.f / P_SCALE);
 #pragma unroll
-                for (int h = 0; h < 8; ++h)
+                for (int h = 0; h < GP; ++h)
                     if (h < G)
                         p.part_o[(slot * G + h) * D + tid] = (__uint_as_float(ov[h]) + __uint_as_float(ov[8 + h]) * (1.f / REM_SCALE)) * back;
                 if (tid < G) {
                     const volatile float *r = red_l + tid;
                     float mine = m_ref[0];
 #pragma unroll
-                    for (int h = 1; h < 8; ++h) mine = tid == h ? m_ref[h] : mine;
+                    for (int h = 1; h < GP; ++h) mine = tid == h ? m_ref[h] : mine;
                     *reinterpret_cast<float2 *>(p.part_ml + (slot * G + tid) * 2) = make_float2(mine, (r[0] + r[8]) + (r[16] + r[24]));
                 }
                 tc_fence_before();
@@ -660,7 +654,8 @@ cudaError_t launch_decode_fp8_umma(const DecodeParams &p, int D, int G, int grid
 {
     if (!decode_fp8_umma_supported(D, G)) return cudaErrorInvalidValue;
     const size_t smem = decode_fp8_umma_smem_bytes(D, p.B);
-    auto kern = decode_fp8_umma_kernel<128>;
+    auto kern = G <= 1 ? decode_fp8_umma_kernel<128, 1> : G <= 2 ? decode_fp8_umma_kernel<128, 2>
+              : G <= 4 ? decode_fp8_umma_kernel<128, 4> : decode_fp8_umma_kernel<128, 8>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
