@@ -48,7 +48,7 @@ constexpr int THREADS = 192;
 constexpr int COL_O = 32;              // S^T buffers at columns 0 and 16
 constexpr int TMEM_COLS = 64;
 constexpr float RESCALE_STEP = 3.5f;    // p <= 2^3.5 between moves of the reference: P' = 32 p vscale / c <= 362 fits E4M3 (max 448)
-constexpr float P_SCALE = 32.f, REM_SCALE = 8.f;
+constexpr float P_SCALE = 32.f, REM_SCALE = 16.f;
 constexpr int CTAS_PER_SM = 3;
 
 constexpr int TILE_FIRST = 1, TILE_LAST = 2, TILE_END = 4;
@@ -163,6 +163,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     constexpr int Q_BYTES = 16 * D;                    // the Q' operand: 16 rows (8 leading, 8 remainder) x D
     constexpr int P_BYTES = 16 * TP * PAGE;            // one P' operand: 16 rows x 128 tokens
     constexpr uint32_t IDESC = instr_desc_e4m3(128, 16);
+    constexpr uint32_t IDESC_PV = IDESC | (1u << 16);   // P' is N-major: a token's 16 bytes (the N index) are contiguous
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -173,7 +174,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     const uint32_t v_ring = smem_u32(at);
     const uint8_t *v_ring_ptr = at;                    at += NST * V_STAGE;
     const uint32_t p_sm = smem_u32(at);
-    uint8_t *p_sm_ptr = at;                            at += 2 * P_BYTES;
+                                                       at += 2 * P_BYTES;
     const uint32_t q_sm = smem_u32(at);                at += Q_BYTES;
     TileMeta *meta = reinterpret_cast<TileMeta *>(at); at += 4 * sizeof(TileMeta);
     float *qscale = reinterpret_cast<float *>(at);     at += 2 * 8 * 4;
@@ -203,17 +204,15 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
-    // rows G..7 of both terms of P' stay zero for the whole kernel (their columns of O^T are never read, but
-    // must stay finite); the other rows are rewritten by every tile
-    for (int i = tid; i < 2 * P_BYTES / 16; i += THREADS)
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(p_sm + (uint32_t)(i * 16)), "r"(0u) : "memory");
-    fence_proxy_async();
     const bool late_wait = (p.flags & DECODE_LATE_WAIT) != 0;
     const bool reverse = (p.flags & DECODE_REVERSE) != 0;
     if (!late_wait) pdl_wait();            // anything read below may come from the kernel before this one
     const unsigned long long t_entry = p.trace ? global_timer_ns() : 0ull;
 
-    // sequence lengths and cumulative page counts of the batch (warp 0), visible to all after the barrier
+    // Sequence lengths and cumulative TILE counts of the batch (warp 0), visible to all after the barrier.  The
+    // flattened list that is cut into equal ranges is the list of (sequence, kv head, tile) here, a tile
+    // being pages [8i, 8i+8) of the sequence: equal ranges are then equal numbers of tiles, which is what a
+    // CTA's time goes with.  The merge kernel is told the same counts, so it finds the partials as usual.
     if (warp == 0) {
         int carry = 0;
         for (int i0 = 0; i0 < p.B; i0 += 32) {
@@ -222,7 +221,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
             if (i < p.B) {
                 n = __ldg(p.seq_lens + i);
                 n = n > 0 ? n : 0;
-                v = (n + PAGE - 1) / PAGE;
+                v = (n + TP * PAGE - 1) / (TP * PAGE);       // tiles of the sequence (per kv head)
                 lens[i] = n;
             }
 #pragma unroll
@@ -239,7 +238,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    if (blockIdx.x == 0)       // the merge kernel reads the page counts from global memory
+    if (blockIdx.x == 0)       // the merge kernel reads the counts from global memory
         for (int i = tid; i <= p.B; i += THREADS) p.prefix[i] = prefix[i];
 
     const int64_t W = gridDim.x, w = blockIdx.x;
@@ -265,10 +264,10 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
         bool triggered = false;
         Cursor cur = {0, 0, 0, 1};
         if (n > 0) cur = locate(prefix, p.B, p.Hkv, x_first);
-        int left = n, issued = 0, k = 0, runs = 0;
+        int left = n, k = 0, runs = 0;
         auto give_up = [&]() { if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); *gave_up = 1; } };
         while (left > 0) {
-            if (!triggered && issued >= trigger_at) {
+            if (!triggered && k >= trigger_at) {
                 triggered = true;
                 if (lane == 0) {
                     if (late_wait) pdl_wait();
@@ -277,34 +276,32 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 __syncwarp();
             }
             const int s = k & 1;
-            const int seg_left = reverse ? cur.pg + 1 : cur.pages - cur.pg;
-            int np = seg_left < TP ? seg_left : TP;
-            np = np < left ? np : left;
+            // tile cur.pg of segment (cur.b, cur.h): pages [8 cur.pg, 8 cur.pg + np)
+            const int b = cur.b, h = cur.h, n_b = lens[b], pages = (n_b + PAGE - 1) / PAGE, pg0 = TP * cur.pg;
+            const int np = pages - pg0 < TP ? pages - pg0 : TP;
             const bool first = (k == 0) || (reverse ? cur.pg == cur.pages - 1 : cur.pg == 0);
-            const bool last = (np == seg_left) || (np == left);
-            const int b = cur.b, h = cur.h, pages = cur.pages, n_b = lens[b];
+            const bool last = (left == 1) || (reverse ? cur.pg == 0 : cur.pg == cur.pages - 1);
             // page ids of the tile (lane j < np), fetched before the waits for the stages
             int id = 0;
             if (lane < np) {
-                const int pg = reverse ? cur.pg - lane : cur.pg + lane;
-                id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg);
+                id = __ldg(p.page_table + (int64_t)b * p.pt_stride + pg0 + lane);
                 if (id < 0 || (int64_t)id >= p.max_pages) {
                     atomicOr(p.status, STATUS_BOUNDS);
                     id = 0;
                 }
             }
             const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK;
-            const uint64_t pol = (issued + lane >= keep_from) ? pol_keep : pol_stream;
+            const uint64_t pol = (k >= keep_from) ? pol_keep : pol_stream;
             // K part: its stage comes back as soon as the scores of the tile two before this one are done
             if (k >= 2 && !__all_sync(FULL, wait_bounded(k_empty + 8 * s, (uint32_t)((k / 2 - 1) & 1)))) { give_up(); break; }
             if (lane == 0) {
                 TileMeta m;
                 m.n_pages = np;
-                const int short_valid = n_b - (pages - 1) * PAGE;      // 1..16 tokens in the last page
-                const int last_pg_slot = reverse ? cur.pg - (pages - 1) : (pages - 1) - cur.pg;   // slot of page pages-1
-                m.short_slot = (short_valid < PAGE && last_pg_slot >= 0 && last_pg_slot < np) ? last_pg_slot : -1;
+                const int short_valid = n_b - (pages - 1) * PAGE;      // 1..16 tokens in the sequence's last page
+                const int last_pg_slot = (pages - 1) - pg0;             // its slot, if it is in this tile
+                m.short_slot = (short_valid < PAGE && last_pg_slot < np) ? last_pg_slot : -1;
                 m.short_valid = short_valid;
-                m.flags = (first ? TILE_FIRST : 0) | (last ? TILE_LAST : 0) | (np == left ? TILE_END : 0);
+                m.flags = (first ? TILE_FIRST : 0) | (last ? TILE_LAST : 0) | (left == 1 ? TILE_END : 0);
                 m.b = b;
                 m.h = h;
                 m.qbuf = (first ? runs : runs - 1) & 1;                // which set of query scales
@@ -346,7 +343,12 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 }
                 amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
                 amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
-                const float inv = amax > 0.f ? 256.f / amax : 0.f;
+                // scaled by the power of two that brings the row's maximum into [128, 256): a bf16 number times a
+                // power of two has 8 significant bits, which the two E4M3 terms (4 + 4) hold exactly
+                const uint32_t be = __float_as_uint(amax) >> 23;          // biased exponent (amax >= 0)
+                const bool tiny = be < 8u;                                // zero (or next to it): the row counts as zero
+                const float inv = tiny ? 0.f : __uint_as_float((261u - be) << 23);      // 2^(7 - e)
+                const float back_q = tiny ? 0.f : __uint_as_float((be - 7u) << 23);     // 2^(e - 7)
                 const uint32_t qdst = q_sm + (uint32_t)(g * 16);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {               // 16-dim chunk 2 qd + c
@@ -365,7 +367,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(lead[0]), "r"(lead[1]), "r"(lead[2]), "r"(lead[3]) : "memory");
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a + 1024u), "r"(rem[0]), "r"(rem[1]), "r"(rem[2]), "r"(rem[3]) : "memory");
                 }
-                if (qd == 0) qscale[qset * 8 + g] = amax * (1.f / 256.f) * p.scale_log2;
+                if (qd == 0) qscale[qset * 8 + g] = back_q * p.scale_log2;
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(q_full);
@@ -373,9 +375,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
             }
             ++k;
             tiles_issued = k;
-            issued += np;
-            for (int i = 0; i < np; ++i)
-                if (--left > 0) step(cur, prefix, p.Hkv, reverse);
+            if (--left > 0) step(cur, prefix, p.Hkv, reverse);
         }
         if (!triggered && lane == 0) {
             if (late_wait) pdl_wait();
@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 const int nks = (np_j + 1) >> 1;
                 for (int ks = 0; ks < nks; ++ks)
                     umma_ss_f8(tmem + COL_O, smem_desc(vbase + (uint32_t)(ks * 2 * V_PAGE), V_PAGE, 128),
-                               smem_desc(pbase + (uint32_t)(ks * 512), 256, 128), IDESC, (first_j && ks == 0) ? 0u : 1u);
+                               smem_desc(pbase + (uint32_t)(ks * 512), 128, 128), IDESC_PV, (first_j && ks == 0) ? 0u : 1u);
                 tc_commit(pv_done + 8 * sj);
                 tc_commit(v_empty + 8 * sj);
                 return true;
@@ -451,8 +451,6 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
         float m_ref[GP], l_sum[GP], qs[GP];
 #pragma unroll
         for (int h = 0; h < GP; ++h) { m_ref[h] = -INFINITY; l_sum[h] = 0.f; qs[h] = 0.f; }
-        float cs = 0.f;
-        int runs = 0;
         bool ok = true;
         for (int k = 0; ok; ++k) {
             const int s = k & 1;
@@ -463,15 +461,15 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
             const TileMeta m = load_meta(&meta[k & 3]);
             const bool first = (m.flags & TILE_FIRST) != 0;
             if (first) {
-                wait_bounded(q_full, (uint32_t)(runs & 1));     // already over: the scores used Q'
-                ++runs;
+                // (the query scales were written before Q' was announced, which the issuing thread saw before it
+                // issued these scores; no wait on that barrier here -- it may be two phases on by now, which a
+                // parity wait cannot tell from none)
 #pragma unroll
                 for (int h = 0; h < GP; ++h) {
                     m_ref[h] = -INFINITY;
                     l_sum[h] = 0.f;
                     qs[h] = reinterpret_cast<volatile float *>(qscale)[m.qbuf * 8 + h];
                 }
-                cs = 0.f;
             }
             uint32_t sv[16];
             tmem_ld16(lane_base + (uint32_t)(16 * s), sv);
@@ -483,74 +481,79 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 ksc = *reinterpret_cast<const float *>(vpage + K_PAGE + 4 * tt);
                 vsc = *reinterpret_cast<const float *>(vpage + K_PAGE + 4 * PAGE + 4 * tt);
             }
+            // The reference of head h follows  e = score + log2(vscale), the size of the token's term in the
+            // output, not the score alone: P' = 32 * 2^(e - ref) then stays in E4M3's range whatever the spread
+            // of the V scales (a huge V row with a negligible probability does not push the others out of it).
+            float lv;
+            asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lv) : "f"(vsc));
+            lv = fmaxf(lv, -60.f);         // an all-zero V row (scale 0) counts as a very small one
             float sc[GP];                  // (heads G..GP-1 have zero queries: their scores are 0, their results unused)
 #pragma unroll
             for (int h = 0; h < GP; ++h)
                 sc[h] = valid ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * (ksc * qs[h]) : -INFINITY;
-            // maxima over the tile's 128 tokens: per head, and of the V scales
+            // maxima of e over the tile's 128 tokens, per head
 #pragma unroll
             for (int h = 0; h < GP; ++h) {
-                const int mk = warp_max_s32(float_key(sc[h]));
+                const int mk = warp_max_s32(float_key(sc[h] + lv));
                 if (lane == 0) red[s * 64 + h * 4 + warp] = mk;
-            }
-            {
-                const int mk = warp_max_s32(__float_as_int(vsc));      // scales are >= 0: their bits order them
-                if (lane == 0) red[s * 64 + 8 * 4 + warp] = mk;
             }
             ok = softmax_all(ok);          // the maxima are in place; and has every thread's wait ended normally?
             if (!ok) break;
             bool changed = false;
-            float alpha[GP];               // factor that moves a head's sums to its new reference
+            float m_new[GP];
 #pragma unroll
             for (int h = 0; h < GP; ++h) {
                 const int4 r = *reinterpret_cast<const int4 *>(red + s * 64 + h * 4);      // the four warps' maxima
                 const float mx = key_float(max(max(r.x, r.y), max(r.z, r.w)));           // finite: every tile has a valid token
-                const float m_new = mx > m_ref[h] + RESCALE_STEP ? mx : m_ref[h];
-                alpha[h] = fast_exp2(m_ref[h] - m_new);
-                changed = changed || (m_new != m_ref[h]);
-                m_ref[h] = m_new;
+                m_new[h] = mx > m_ref[h] + RESCALE_STEP ? mx : m_ref[h];
+                changed = changed || (m_new[h] != m_ref[h]);
             }
-            float wp, ca;
+            if (changed) {
+                // the sums (and, unless the run starts here, O^T of the run so far) move to the new references
+                float alpha[GP];
+#pragma unroll
+                for (int h = 0; h < GP; ++h) {
+                    alpha[h] = fast_exp2(m_ref[h] - m_new[h]);
+                    l_sum[h] *= alpha[h];
+                    m_ref[h] = m_new[h];
+                }
+                if (!first) {
+                    // the values of the tile before this one must be done (that barrier's phase before that one is over
+                    // because this tile's scores were issued after it, and its next phase needs the probabilities
+                    // written below)
+                    ok = wait_bounded(pv_done + 8 * ((k - 1) & 1), (uint32_t)(((k - 1) >> 1) & 1));
+                    ok = softmax_all(ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    uint32_t ov[16];
+                    tmem_ld16(lane_base + COL_O, ov);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c)
+                        if ((c & 7) < GP) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha[(c & 7) % GP]);
+                    tmem_st16(lane_base + COL_O, ov);
+                    tmem_wait_st();
+                }
+            }
+            // probabilities, split into two E4M3 terms: the token's 16 bytes [leading terms of heads 0..7 |
+            // remainders of heads 0..7] (heads >= GP zero) are one row of the N-major P' operand
             {
-                const int4 r = *reinterpret_cast<const int4 *>(red + s * 64 + 8 * 4);
-                const float svmax = __int_as_float(max(max(r.x, r.y), max(r.z, r.w)));
-                const float up = __uint_as_float((__float_as_uint(svmax) + 0x007FFFFFu) & 0x7F800000u);   // power of two >= svmax
-                const float cs_new = fmaxf(cs, up);
-                const float inv_cs = cs_new > 0.f ? __uint_as_float(0x7F000000u - __float_as_uint(cs_new)) : 0.f;   // 1 / 2^e
-                ca = cs * inv_cs;                                             // 1 unless the reference grew
-                changed = changed || (cs_new != cs);
-                cs = cs_new;
-                wp = P_SCALE * inv_cs;
-            }
-            if (changed && !first) {
-                // O^T of the run so far moves to the new references: the values of the tile before this one must be
-                // done (that barrier's phase before that one is over because this tile's scores were issued after
-                // it, and its next phase needs the probabilities written below)
-                ok = wait_bounded(pv_done + 8 * ((k - 1) & 1), (uint32_t)(((k - 1) >> 1) & 1));
-                ok = softmax_all(ok);
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t ov[16];
-                tmem_ld16(lane_base + COL_O, ov);
-                tmem_wait_ld();
+                float lead[8], rem[8];
 #pragma unroll
-                for (int c = 0; c < 16; ++c)
-                    if ((c & 7) < GP) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * (alpha[(c & 7) % GP] * ca));
-                tmem_st16(lane_base + COL_O, ov);
-                tmem_wait_st();
-            }
-            // probabilities, split into two E4M3 terms; bytes of token (j, tt): [j][term][head][tt]
-            uint8_t *parea = p_sm_ptr + s * P_BYTES + j * 256 + tt;
+                for (int h = 0; h < 8; ++h) { lead[h] = 0.f; rem[h] = 0.f; }
 #pragma unroll
-            for (int h = 0; h < GP; ++h) {
-                const float pr = fast_exp2(sc[h] - m_ref[h]);       // 0 for a token that is not in use
-                const float pp = pr * (vsc * wp);
-                const float lead = __uint_as_float(__float_as_uint(pp) & 0xFFF00000u);   // E4M3's three mantissa bits
-                const float rem = (pp - lead) * REM_SCALE;                                 // < 8 * 32 at the top binade
-                const uint32_t codes = pack_e4m3x2(lead, rem);       // low byte: leading term, high byte: remainder
-                parea[h * 16] = (uint8_t)(codes & 0xFFu);
-                parea[128 + h * 16] = (uint8_t)(codes >> 8);
-                l_sum[h] = l_sum[h] * alpha[h] + pr;
+                for (int h = 0; h < GP; ++h) {
+                    const float pr = fast_exp2(sc[h] - m_ref[h]);       // 0 for a token that is not in use; its share of the sum
+                    const float pp = pr * (vsc * P_SCALE);               // = 32 * 2^(e - ref) <= 362
+                    lead[h] = __uint_as_float((__float_as_uint(pp) + 0x00080000u) & 0xFFF00000u);   // rounded to E4M3's three mantissa bits
+                    rem[h] = (pp - lead[h]) * REM_SCALE;                              // |.| <= 16 * 16 at the top binade
+                    l_sum[h] += pr;
+                }
+                const uint32_t w0 = pack_e4m3x2(lead[0], lead[1]) | (pack_e4m3x2(lead[2], lead[3]) << 16);
+                const uint32_t w1 = GP > 4 ? pack_e4m3x2(lead[4], lead[5]) | (pack_e4m3x2(lead[6], lead[7]) << 16) : 0u;
+                const uint32_t w2 = pack_e4m3x2(rem[0], rem[1]) | (pack_e4m3x2(rem[2], rem[3]) << 16);
+                const uint32_t w3 = GP > 4 ? pack_e4m3x2(rem[4], rem[5]) | (pack_e4m3x2(rem[6], rem[7]) << 16) : 0u;
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(p_sm + (uint32_t)(s * P_BYTES + tid * 16)), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
             }
             // V codes the tensor core will read but that belong to no token in use must be finite too: the
             // unused slots of the sequence's last page may hold anything, and an odd tile reads one page
@@ -593,7 +596,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
                 softmax_sync();
                 const int64_t seg = (int64_t)m.b * p.Hkv + m.h;
                 const int64_t slot = partial_slot(T, W, w, x0, seg);
-                const float back = cs * (1.f / P_SCALE);
+                const float back = 1.f / P_SCALE;
 #pragma unroll
                 for (int h = 0; h < GP; ++h)
                     if (h < G)

@@ -102,6 +102,30 @@ def test_rows_of_very_different_magnitude():
     assert bool((err <= ATOL + RTOL * row_max).all()), f"max abs err {err.max().item()} at |ref| up to {ref.abs().max().item()}"
 
 
+def test_many_short_sequences():
+    """Hundreds of sequences of at most one tile (128 tokens), more (sequence, kv head) segments than workers: every
+    worker of the tcgen05 kernel goes through several one-tile runs back to back, the case in which its roles are
+    furthest apart (queries of the run after next being prepared while the softmax is still on this one)."""
+    g = torch.Generator().manual_seed(5)
+    lens = torch.randint(1, 129, (320,), generator=g, dtype=torch.int32)
+    lens[::7] = 128
+    lens[3::11] = 0
+    w = W.Workload("fp8_short", 2, 8, 4, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=107)
+    harness, dw = _setup(w, lens)
+    o, _, _, _ = _oracle(dw, range(2))
+    Q = harness.step_inputs(dw, 1)["Q"]
+    ref = o.decode_attn(1, Q.cpu(), dw.lens_cpu)
+    for overlap in (1, 0):
+        dw.retune(overlap=overlap)
+        for rep in range(5):
+            out = torch.full((dw.batch, 8, 128), float("nan"), dtype=torch.bfloat16, device=dw.device)
+            dw.cache.skv_decode_attn(1, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+            torch.cuda.synchronize()
+            assert dw.cache.skv_get_status() == 0
+            err = (out.cpu().double() - ref).abs()
+            assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"overlap {overlap} rep {rep}: {err.max().item()}"
+
+
 def test_whole_step_and_unsupported_calls():
     from paper_2604_22782_b200 import harness
     from paper_2604_22782_b200.binding import SKV_ERR_UNSUPPORTED, SkvError
