@@ -125,9 +125,13 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
  * attention sees  code value x scale.  Cache bytes per token become
  * 2 x |owners| x kv_heads x (head_dim + 4).  skv_decode_attn, skv_decode_step and
  * skv_decode_step_host work on such a cache as on a bf16 one (any q_heads /
- * kv_heads <= 8, tensor cores in f16, scales applied outside the contractions);
- * skv_gather and the pre-fill calls return SKV_ERR_UNSUPPORTED.  Same
- * arguments and errors as skv_cache_pool_bytes / skv_cache_create. */
+ * kv_heads <= 8; the scales are applied outside the contractions).  At
+ * head_dim 128 both contractions run as FP8 tensor-core instructions (tcgen05,
+ * kind f8f6f4) on the stored codes, with the queries and the probabilities each
+ * split into two E4M3 terms; at head_dim 64, or with skv_set_decode_variant(2),
+ * the codes are converted to f16 on the way into mma.sync.  skv_gather and the
+ * pre-fill calls return SKV_ERR_UNSUPPORTED.  Same arguments and errors as
+ * skv_cache_pool_bytes / skv_cache_create. */
 int skv_cache_pool_bytes_fp8(int n_layers, const int32_t *r, int kv_heads, int head_dim,
                              int page_size, int64_t max_pages, size_t *out_bytes);
 int skv_cache_create_fp8(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,
@@ -348,7 +352,10 @@ int skv_get_status(skv_cache *cache, void *stream, int *device_status);
 
 /* Split-K kernel variant: 0 = automatic (CUDA-core kernel when
  * q_heads == kv_heads, tensor-core (mma) kernel otherwise), 1 = CUDA-core
- * kernel (only q_heads == kv_heads), 2 = tensor-core kernel. */
+ * kernel (only q_heads == kv_heads), 2 = tensor-core kernel.  On an FP8 cache:
+ * 0 or 1 = the tcgen05 kernel where it applies (head_dim 128; its worker count
+ * and launch shape are fixed, skv_set_decode_tuning does not apply to it),
+ * 2 = the mma.sync kernel. */
 int skv_set_decode_variant(skv_cache *cache, int variant);
 
 /* Launch shape of the split-K kernel (default: 8 warps per SM with two 8 KB
