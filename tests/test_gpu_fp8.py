@@ -126,6 +126,33 @@ def test_many_short_sequences():
             assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"overlap {overlap} rep {rep}: {err.max().item()}"
 
 
+@pytest.mark.parametrize("trial", range(6))
+def test_random_shapes_whole_steps(trial):
+    """Seeded random batch, lengths and group size through whole decode steps (three layers reading layer 0: forward
+    and backward walks, chained launches) against the oracle."""
+    g = torch.Generator().manual_seed(200 + trial)
+    Hkv = (1, 2, 4, 8, 2, 4)[trial]
+    G = (8, 4, 3, 1, 2, 4)[trial]
+    B = int(torch.randint(1, 14, (1,), generator=g))
+    lens = torch.randint(0, (130, 700, 300, 140, 1200, 260)[trial], (B,), generator=g).to(torch.int32)
+    lens[0] = max(int(lens[0]), 1)
+    w = W.Workload("fp8_rand", 3, G * Hkv, Hkv, 128, 16, B, 0, 0, "explicit", explicit_r=(0, 0, 0), seed=300 + trial)
+    from paper_2604_22782_b200 import harness
+    dw = harness.setup(w, lens=lens, fp8=True)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    o, _, _, _ = _oracle(dw, range(3))
+    for rep in range(2):
+        t["out"].fill_(float("nan"))
+        dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
+        torch.cuda.synchronize()
+        assert dw.cache.skv_get_status() == 0
+        for l in range(3):
+            ref = o.decode_attn(l, t["Q"][l].cpu(), dw.lens_cpu)
+            err = (t["out"][l].cpu().double() - ref).abs()
+            assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"rep {rep} layer {l}: {err.max().item()}"
+
+
 def test_whole_step_and_unsupported_calls():
     from paper_2604_22782_b200 import harness
     from paper_2604_22782_b200.binding import SKV_ERR_UNSUPPORTED, SkvError
