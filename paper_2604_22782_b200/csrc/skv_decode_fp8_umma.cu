@@ -2,33 +2,39 @@
 // tensor cores: both contractions are tcgen05 instructions of kind f8f6f4 that read the stored E4M3
 // codes straight from shared memory, so no code is ever converted.  Same split-K scheme and the same
 // partial format as skv_decode.cu (the merge kernel is shared); here a worker is a CTA and the unit
-// of work is a TILE of up to 8 consecutive pages (128 tokens) of one (sequence, kv head) segment.
+// of work is a TILE: pages [8i, 8i+8) (128 tokens) of one (sequence, kv head) segment.  The list
+// that is cut into equal contiguous ranges is the list of tiles.
 //
 // Per tile, with the tokens as the M dimension (TMEM lanes):
 //   S^T[128 tokens x 16]  = Kc[128 x D] . Q'^T[D x 16]          4 instructions (K = 32 dims each)
 //   O^T[D dims x 16]     += Vc^T[D x 32 tokens] . P'^T[32 x 16]  1 instruction per 2 pages
-// The other operand must be E4M3 too, so Q' = 256 Q / qmax and P' = 256 p vscale / c are split into a
-// leading E4M3 term and an E4M3 remainder (together about as precise as bf16), and the two terms take
-// the 16 columns: column h = leading term of head h, column 8 + h = remainder of head h (h < G <= 8);
-// the softmax adds the two columns.  The per-token scales stay outside the contractions:
-//   score_t = (qmax / 256) kscale_t (S_h + S_{8+h}),     O = (O_h + O_{8+h}) c / 256,
-// with c a power of two >= every vscale of the run so far.
+// The other operand must be E4M3 too, so it is split into a leading E4M3 term and an E4M3 remainder,
+// and the two terms take the 16 columns: column h = leading term of head h, column 8 + h =
+// remainder of head h (h < G <= 8); the softmax adds the two columns.
+//   Q' = Q 2^k, the power of two that brings the row's maximum into [128, 256): a bf16 number times
+//        a power of two has 8 significant bits, which 4 + 4 hold exactly (but for the smallest elements);
+//   P' = 32 p vscale / 2^ref, leading term rounded to 4 significant bits, remainder times 16.
+// The per-token scales stay outside the contractions:  score_t = 2^-k kscale_t (S_h + S_{8+h}).
+// The reference of head h follows  e_t = score_t + log2(vscale_t), the size of the token's term in
+// the output, and only moves when the maximum of e has grown by more than 2^3.5: P' <= 362 fits E4M3
+// whatever the spread of the V scales, O^T is rescaled (through registers) rarely, and the partial
+// (reference, sum of 2^(score - reference), O^T / 32) is in the merge kernel's usual form.
 //
 // Six warps:
 //   warps 0-3  softmax: thread t owns token t of the tile (TMEM lane t); at the end of a run thread
 //              d owns dim d of O^T
 //   warp 4     lane 0 issues the tensor-core instructions
-//   warp 5     walks the worker's block range, prepares Q' of every new segment, issues the copies
-// Shared memory per stage (2 stages): the K parts of the tile's pages side by side (page j at
-// j * 2048: [8-token group][16-dim chunk][8 tokens][16 B], the K-major core-matrix layout the pages
-// are stored in, so the 128 tokens form ONE A operand with a uniform group stride), and the
-// V-and-scales parts side by side (page j at j * 2176: [dim][16 tokens] = K-major core matrices of
-// V^T, then the K and V scales).  P' of a tile overwrites the first 2 KB of the tile's K area, which
-// the tensor core has finished with by then.  Tensor memory (64 columns): two S^T buffers, O^T.
-// The reference maximum of a head only moves when the true maximum has grown by more than 2^8, so O^T
-// is rescaled (through registers) rarely; the partial carries the reference, so the merged result
-// is the exact softmax.  Every wait is bounded; after a timeout the roles leave through the common
-// exit, where copies in flight get their (bounded) wait and the tensor memory is freed.
+//   warp 5     walks the worker's tiles, prepares Q' of every new segment, issues the copies
+// Shared memory: a K ring and a V ring of two stages each.  A K stage holds the K parts of the
+// tile's pages side by side (page j at j * 2048: [8-token group][16-dim chunk][8 tokens][16 B], the
+// K-major core-matrix layout the pages are stored in, so the 128 tokens form ONE A operand with a
+// uniform group stride) and is given back by the tile's score instructions; a V stage holds the
+// V-and-scales parts (page j at j * 2176: [dim][16 tokens] = K-major core matrices of V^T, then the
+// K and V scales) and is given back by the tile's value instructions.  Two P' operands (N-major:
+// a token's 16 bytes are one row), one Q' operand.  Tensor memory (64 columns): two S^T buffers, O^T.
+// Waiting threads are suspended (try_wait with a time hint), not polling.  Every wait is bounded;
+// after a timeout the roles leave through the common exit, where copies in flight get their
+// (bounded) wait and the tensor memory is freed.
 #include "skv_common.cuh"
 #include "skv_tcgen05.cuh"
 #include "skv_walk.cuh"
