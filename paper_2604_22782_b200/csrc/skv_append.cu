@@ -78,9 +78,33 @@ __global__ void __launch_bounds__(COPY_THREADS) gather_kernel(GatherParams p)
 }
 
 // ---- FP8 pages -----------------------------------------------------------------------------
-// One warp per (token, kv head); grid.y picks K or V, grid.z the owner layer.  The row's D values
-// are spread over the lanes (D/32 each); amax by shuffles; scale = amax / 448, codes =
-// E4M3(x * (448 / amax)) round-to-nearest-even, saturating; every step a single fp32 operation.
+// One row (token, kv head) by one warp: the D values are spread over the lanes (PER = D/32 each,
+// dims lane*PER ..); amax by shuffles; scale = amax / 448, codes = E4M3(x * (448 / amax))
+// round-to-nearest-even, saturating; every step a single fp32 operation.  Returns the lane's codes
+// (c01: dims 0,1 of the lane, c23: dims 2,3) and the row's amax.
+__device__ __forceinline__ void quantize_row(const uint16_t *row, int PER, int lane, uint32_t &c01, uint32_t &c23, float &amax)
+{
+    float x[4] = {0.f, 0.f, 0.f, 0.f};
+    if (PER == 4) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2 *>(row + lane * 4));
+        x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    } else {
+        const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(row + lane * 2));
+        x[0] = bf16_lo(w); x[1] = bf16_hi(w);
+    }
+    amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+    const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+    c01 = pack_e4m3x2(__fmul_rn(x[0], inv), __fmul_rn(x[1], inv));
+    c23 = pack_e4m3x2(__fmul_rn(x[2], inv), __fmul_rn(x[3], inv));
+}
+
+// One warp per (token, kv head); grid.y picks K or V, grid.z the owner layer.  A token at a time
+// costs scattered small stores (V is dim-major: one byte in each of D rows; K: D/16 pieces of 4
+// bytes per lane).  When the 16 tokens of a whole page arrive together and in order (a prompt being
+// appended), the warp of the page's first token quantises all 16 rows and writes 16 bytes per
+// store, and the warps of the other 15 tokens have nothing to do.
 __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
 {
     const int lane = threadIdx.x & 31;
@@ -99,22 +123,71 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Param
     const int which = blockIdx.y;
     const int64_t layer = blockIdx.z;
     const int D = p.D, PER = D / 32;                  // 4 values per lane at D = 128, 2 at D = 64
-    const uint16_t *src = (which ? p.V : p.K) + ((layer * p.n_tokens + tok) * p.Hkv + h) * D + lane * PER;
-    float x[4] = {0.f, 0.f, 0.f, 0.f};
-    if (PER == 4) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2 *>(src));
-        x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
-    } else {
-        const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(src));
-        x[0] = bf16_lo(w); x[1] = bf16_hi(w);
-    }
-    float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
-    const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
-    const uint32_t c01 = pack_e4m3x2(__fmul_rn(x[0], inv), __fmul_rn(x[1], inv));
-    const uint32_t c23 = pack_e4m3x2(__fmul_rn(x[2], inv), __fmul_rn(x[3], inv));
+    const uint16_t *rows = (which ? p.V : p.K) + (layer * p.n_tokens * p.Hkv + h) * D;      // row of token t: + t * Hkv * D
     uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
+    // do tokens tok-off .. tok-off+15 of this call carry the page's 16 slots in order?
+    const int64_t t0 = tok - off;
+    bool whole_page = t0 >= 0 && t0 + PAGE <= p.n_tokens;
+    if (whole_page) {
+        const int64_t s_l = lane < PAGE ? p.slot_map[t0 + lane] : 0;
+        whole_page = __all_sync(0xFFFFFFFFu, lane >= PAGE || s_l == page * PAGE + lane);
+    }
+    if (whole_page) {
+        if (off != 0) return;
+        if (which == 0) {
+            // K: lane = (token q of this round, 16-dim chunk c); a chunk of a token is one 16-byte piece of the page
+            const int CH = D / 16, TPI = 32 / CH;          // 8 chunks x 4 tokens per round at D = 128
+            const int c = lane % CH, q = lane / CH;
+            for (int t = q; t < PAGE; t += TPI) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(rows + (t0 + t) * p.Hkv * D + 16 * c);
+                const uint4 a = __ldg(src), b = __ldg(src + 1);
+                const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                float x[16];
+                float amax = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    x[2 * i] = bf16_lo(w[i]);
+                    x[2 * i + 1] = bf16_hi(w[i]);
+                    amax = fmaxf(amax, fmaxf(fabsf(x[2 * i]), fabsf(x[2 * i + 1])));
+                }
+                for (int d = 1; d < CH; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+                const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    o[i] = pack_e4m3x2(__fmul_rn(x[4 * i], inv), __fmul_rn(x[4 * i + 1], inv)) |
+                           (pack_e4m3x2(__fmul_rn(x[4 * i + 2], inv), __fmul_rn(x[4 * i + 3], inv)) << 16);
+                *reinterpret_cast<uint4 *>(blk + fp8_k_pos(D, t, 16 * c)) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (c == 0) *reinterpret_cast<float *>(blk + fp8_ks_off(D) + 4 * t) = __fdiv_rn(amax, 448.f);
+            }
+            return;
+        }
+        {
+            uint32_t v[4][4] = {};                 // [dim of the lane][4 tokens per word]
+            float my_scale = 0.f;
+#pragma unroll
+            for (int t = 0; t < PAGE; ++t) {
+                uint32_t c01, c23;
+                float amax;
+                quantize_row(rows + (t0 + t) * p.Hkv * D, PER, lane, c01, c23, amax);
+                const int sh = 8 * (t & 3);
+                v[0][t >> 2] |= (c01 & 0xFFu) << sh;
+                v[1][t >> 2] |= (c01 >> 8) << sh;
+                v[2][t >> 2] |= (c23 & 0xFFu) << sh;
+                v[3][t >> 2] |= (c23 >> 8) << sh;
+                if (lane == t) my_scale = __fdiv_rn(amax, 448.f);
+            }
+            uint4 *dst = reinterpret_cast<uint4 *>(blk + fp8_v_off(D) + (lane * PER) * PAGE);
+#pragma unroll
+            for (int d = 0; d < 4; ++d)
+                if (d < PER) dst[d] = make_uint4(v[d][0], v[d][1], v[d][2], v[d][3]);
+            if (lane < PAGE) *reinterpret_cast<float *>(blk + fp8_vs_off(D) + 4 * lane) = my_scale;
+            return;
+        }
+    }
+    uint32_t c01, c23;
+    float amax;
+    quantize_row(rows + tok * p.Hkv * D, PER, lane, c01, c23, amax);
     if (which == 0) {                                  // K: a lane's dims are neighbours inside one 16-byte piece
         uint8_t *dst = blk + fp8_k_pos(D, off, lane * PER);
         if (PER == 4) *reinterpret_cast<uint32_t *>(dst) = c01 | (c23 << 16);
