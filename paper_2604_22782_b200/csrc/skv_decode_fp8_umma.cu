@@ -64,7 +64,7 @@ struct alignas(16) TileMeta {
     int short_valid;    // tokens in use in that page
     int flags;          // TILE_FIRST / TILE_LAST of a run inside a segment, TILE_END of the worker
     int b, h;           // the segment
-    int qbuf;           // which Q' buffer holds the segment's queries
+    int qbuf;           // which of the two sets of query scales belongs to the segment
     int pad;
 };
 
