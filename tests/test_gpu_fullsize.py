@@ -6,7 +6,9 @@ whole step through skv_decode_step).  The oracle cannot hold these whole, so:
     |out - ref| <= 1e-2 + 1e-2 |ref|, for a sample of sequences (shortest, longest, seeded picks;
     full length, all heads) on a sample of layers (first owner, its first reader, last owner, last layer);
   - every other output row must be finite and lie inside the convex-combination bound
-    |out| <= max |V| of the generator's value table."""
+    |out| <= max |V| of the generator's value table.
+The Llama-3-8B and Qwen3-8B workloads also run on FP8 pages (codes and scales of the sampled sequences bit for
+bit against the oracle's quantiser, their outputs within the same tolerance)."""
 import pytest
 import torch
 
@@ -121,6 +123,64 @@ def test_llama2_7b_32k_full_size():
 def test_sharing_sweep_full_size(group):
     """Config 5: Llama-3-8B shape, batch 128, lengths U[512,2048], owner fraction 1/group."""
     _check_workload(W.sweep_workload(group), n_seqs=4)
+
+
+def _check_workload_fp8(w, n_seqs):
+    """The same whole step on FP8 pages (library defaults: the tcgen05 kernel at head_dim 128): codes and
+    scales of every token of the sampled sequences on the sampled source layers bit for bit against the oracle's
+    quantiser, their attention outputs element by element, every other row finite and inside the bound."""
+    from oracle import Oracle
+    from paper_2604_22782_b200 import harness
+    dw = harness.setup(w, fp8=True)
+    harness.prefill(dw, upto_offset=-1)
+    t = harness.step_tensors(dw)
+    t["out"].fill_(float("nan"))
+    dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    stats = dw.cache.skv_cache_stats()
+    assert stats["bytes_per_token"] == 2 * len(dw.owners) * w.kv_heads * (w.head_dim + 4)
+
+    seqs = _sample_sequences(dw.lens_cpu, n_seqs, w.seed + 7)
+    layers = _sample_layers(dw.r)
+    sub_lens = dw.lens_cpu[seqs]
+    o = Oracle(w.n_layers, dw.r, w.q_heads, w.kv_heads, w.head_dim, len(seqs), int(sub_lens.max()))
+    local, lpos = W.token_index(sub_lens)
+    glob = torch.as_tensor(seqs, dtype=torch.int64)[local]
+    slots = W.slot_map_for(dw.page_table_cpu, glob, lpos, w.page_size)
+    chunk = 1 << 15
+    for src in sorted({dw.r[l] for l in layers}):
+        for s in range(0, local.numel(), chunk):
+            e = min(local.numel(), s + chunk)
+            K, V = W.draw_kv(w, src, glob[s:e], lpos[s:e], device=dw.device)
+            okc, ovc, oks, ovs = o.append_fp8(src, K.cpu(), V.cpu(), local[s:e], lpos[s:e])
+            n = e - s
+            kc = torch.zeros((n, w.kv_heads, w.head_dim), dtype=torch.uint8, device=dw.device)
+            vc = torch.zeros_like(kc)
+            ks = torch.zeros((n, w.kv_heads), dtype=torch.float32, device=dw.device)
+            vs = torch.zeros_like(ks)
+            dw.cache.skv_gather_fp8(src, slots[s:e].to(dw.device), kc, vc, ks, vs)
+            assert torch.equal(kc.cpu(), okc) and torch.equal(vc.cpu(), ovc), f"codes of layer {src}, tokens {s}..{e}"
+            assert torch.equal(ks.cpu().view(torch.int32), oks.view(torch.int32)), f"K scales of layer {src}"
+            assert torch.equal(vs.cpu().view(torch.int32), ovs.view(torch.int32)), f"V scales of layer {src}"
+    for l in layers:
+        Q = t["Q"][l].cpu()[seqs]
+        ref = o.decode_attn(l, Q, sub_lens)
+        got = t["out"][l].cpu()[seqs].double()
+        err = (got - ref).abs()
+        assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {l}: max abs err {err.max().item()}"
+    o.close()
+    out = t["out"].float()
+    assert torch.isfinite(out).all()
+    assert out.abs().max().item() <= 5.0 * w.kv_std * 1.07      # E4M3 rounding can lift a value by 1/16
+
+
+def test_llama3_8b_full_size_fp8():
+    _check_workload_fp8(W.get_workload("llama3_8b"), n_seqs=4)
+
+
+def test_qwen3_8b_full_size_fp8():
+    _check_workload_fp8(W.get_workload("qwen3_8b"), n_seqs=3)
 
 
 def test_sharing_sweep_cache_bytes_scale_exactly():
