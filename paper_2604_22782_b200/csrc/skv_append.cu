@@ -105,13 +105,24 @@ __device__ __forceinline__ void quantize_row(const uint16_t *row, int PER, int l
 // bytes per lane).  When the 16 tokens of a whole page arrive together and in order (a prompt being
 // appended), the warp of the page's first token quantises all 16 rows and writes 16 bytes per
 // store, and the warps of the other 15 tokens have nothing to do.
+__device__ __forceinline__ void append_fp8_row(const AppendFp8Params &p, int64_t warp, int lane);
+
 __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * COPY_THREADS + threadIdx.x) >> 5;
-    if (warp >= p.n_tokens * p.Hkv) return;
-    const int64_t tok = warp / p.Hkv;
-    const int h = (int)(warp - tok * p.Hkv);
+    // the warps of a bounded grid go through the (token, kv head) rows: most rows of a prompt are done by
+    // their page's first row and end at once, which a loop iteration does more cheaply than a CTA launch
+    // (rows counted head-major and an odd number of warps in the grid: a warp then meets every position inside
+    // a page in turn, instead of always the pages' first rows or never one)
+    const int64_t n_rows = p.n_tokens * p.Hkv, stride = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); warp < n_rows; warp += stride)
+        append_fp8_row(p, warp, lane);
+}
+
+__device__ __forceinline__ void append_fp8_row(const AppendFp8Params &p, int64_t warp, int lane)
+{
+    const int h = (int)(warp / p.n_tokens);
+    const int64_t tok = warp - (int64_t)h * p.n_tokens;
     const int64_t slot = p.slot_map[tok];
     if (slot < 0) return;
     if (slot >= p.n_slots) {
@@ -268,10 +279,11 @@ namespace skv {
 cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s)
 {
     const int64_t warps = p.n_tokens * p.Hkv;
-    const int64_t blocks = (warps * 32 + 255) / 256;
+    int64_t blocks = (warps + 6) / 7;                  // 7 warps per CTA
     if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7FFFFFFFll || n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
-    append_fp8_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), 256, 0, s>>>(p);
+    if (n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
+    if (blocks > 4095) blocks = 4095;                  // the kernel's warps loop over the rows; 7 x 4095 is odd
+    append_fp8_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), 224, 0, s>>>(p);
     return cudaGetLastError();
 }
 
