@@ -508,27 +508,7 @@ __global__ void decode_splitk_kernel(DecodeParams p, int G, int stages)
     if (!late_wait) pdl_wait();            // anything read below may come from the kernel before this one
 
     // sequence lengths and cumulative page counts of the batch (warp 0), visible to all after the barrier
-    if (warp == 0) {
-        int carry = 0;
-        for (int i0 = 0; i0 < p.B; i0 += 32) {
-            const int i = i0 + lane;
-            int n = 0, v = 0;
-            if (i < p.B) {
-                n = __ldg(p.seq_lens + i);
-                n = n > 0 ? n : 0;
-                v = (n + PAGE - 1) / PAGE;
-                lens[i] = n;
-            }
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int u = __shfl_up_sync(FULL, v, d);
-                if (lane >= d) v += u;
-            }
-            if (i < p.B) prefix[i + 1] = carry + v;
-            carry += __shfl_sync(FULL, v, 31);
-        }
-        if (lane == 0) prefix[0] = 0;
-    }
+    if (warp == 0) scan_lengths(p.seq_lens, p.B, PAGE, prefix, lens, lane);
     __syncthreads();
     if (blockIdx.x == 0)       // the merge kernel reads the page counts from global memory
         for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.prefix[i] = prefix[i];

@@ -219,27 +219,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     // flattened list that is cut into equal ranges is the list of (sequence, kv head, tile) here, a tile
     // being pages [8i, 8i+8) of the sequence: equal ranges are then equal numbers of tiles, which is what a
     // CTA's time goes with.  The merge kernel is told the same counts, so it finds the partials as usual.
-    if (warp == 0) {
-        int carry = 0;
-        for (int i0 = 0; i0 < p.B; i0 += 32) {
-            const int i = i0 + lane;
-            int n = 0, v = 0;
-            if (i < p.B) {
-                n = __ldg(p.seq_lens + i);
-                n = n > 0 ? n : 0;
-                v = (n + TP * PAGE - 1) / (TP * PAGE);       // tiles of the sequence (per kv head)
-                lens[i] = n;
-            }
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int u = __shfl_up_sync(FULL, v, d);
-                if (lane >= d) v += u;
-            }
-            if (i < p.B) prefix[i + 1] = carry + v;
-            carry += __shfl_sync(FULL, v, 31);
-        }
-        if (lane == 0) prefix[0] = 0;
-    }
+    if (warp == 0) scan_lengths(p.seq_lens, p.B, TP * PAGE, prefix, lens, lane);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();

@@ -51,6 +51,33 @@ __device__ __forceinline__ void step(Cursor &c, const int32_t *prefix, int Hkv, 
     }
 }
 
+// By one warp: lens[i] = max(seq_lens[i], 0) and prefix[i] = number of units (pages, or tiles of several
+// pages: `unit_tokens` tokens each, the last one of a sequence possibly short) of the sequences before i,
+// per kv head; prefix[B] = all of them.
+__device__ __forceinline__ void scan_lengths(const int32_t *seq_lens, int B, int unit_tokens, int32_t *prefix, int32_t *lens,
+                                             int lane)
+{
+    int carry = 0;
+    for (int i0 = 0; i0 < B; i0 += 32) {
+        const int i = i0 + lane;
+        int n = 0, v = 0;
+        if (i < B) {
+            n = __ldg(seq_lens + i);
+            n = n > 0 ? n : 0;
+            v = (n + unit_tokens - 1) / unit_tokens;
+            lens[i] = n;
+        }
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int u = __shfl_up_sync(0xFFFFFFFFu, v, d);
+            if (lane >= d) v += u;
+        }
+        if (i < B) prefix[i + 1] = carry + v;
+        carry += __shfl_sync(0xFFFFFFFFu, v, 31);
+    }
+    if (lane == 0) prefix[0] = 0;
+}
+
 // Shared-memory carve-up (dynamic): prefix[B+1] | lens[B] | rings | barriers | CTA arrival word
 __host__ __device__ inline size_t table_bytes(int B) { return (((size_t)(2 * B + 1) * 4) + 127) & ~(size_t)127; }
 
