@@ -315,7 +315,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "e4m3 pages, f16 contractions" if args.fp8 else "bf16", "data": "synthetic",
+        "dtype": "e4m3 pages" if args.fp8 else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "family": w.family, "n_layers": L, "owners": n_own, "batch": dw.batch,
                    "tokens": int(dw.lens_cpu.sum()), "q_heads": w.q_heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size,
@@ -412,13 +412,23 @@ def prefill_leg(args, dev):
                        "frac": res["tcgen05"]["tflops"] / peak}
     if dw.cache.skv_get_status() != 0:
         raise SystemExit("device status after the pre-fill leg")
+    # the same prompts on FP8 pages: quantising append and the mma.sync kernel that converts the codes on the way in
+    del dw
+    torch.cuda.empty_cache()
+    dq = harness.setup(w, device=dev, lens=lens, fp8=True)
+    ms_append8 = timed(lambda: dq.cache.skv_append(0, K, V, slots))
+    ms8 = timed(lambda: dq.cache.skv_prefill_attn(1, inp["Q"], inp["cu_q_lens"], dq.page_table, dq.seq_lens, out, T))
+    res["fp8_pages"] = {"append_ms": ms_append8, "ms_per_call": ms8, "tflops": flops / (ms8 * 1e-3) / 1e12,
+                        "tokens_per_s": B * T / (ms8 * 1e-3)}
+    if dq.cache.skv_get_status() != 0:
+        raise SystemExit("device status after the FP8 pre-fill leg")
     return res
 
 
 def fp8_leg(args, dev):
     """The benchmark's workload with FP8 pages (E4M3 codes + one fp32 scale per token and kv head): whole
-    decode steps, cache bytes per token, and the rate in tokens attended per microsecond next to the bf16
-    cache's (the FP8 kernel converts codes on the way into the tensor cores and is bound by that, not by HBM)."""
+    decode steps (at head_dim 128 the tcgen05 kernel that runs both contractions on the stored codes), cache bytes
+    per token, and the rate in tokens attended per microsecond, to be read next to the bf16 cache's."""
     from paper_2604_22782_b200 import harness
     w = W.get_workload("llama3_8b")
     dw = harness.setup(w, device=dev, fp8=True)

@@ -129,9 +129,11 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
  * head_dim 128 both contractions run as FP8 tensor-core instructions (tcgen05,
  * kind f8f6f4) on the stored codes, with the queries and the probabilities each
  * split into two E4M3 terms; at head_dim 64, or with skv_set_decode_variant(2),
- * the codes are converted to f16 on the way into mma.sync.  skv_gather and the
- * pre-fill calls return SKV_ERR_UNSUPPORTED.  Same arguments and errors as
- * skv_cache_pool_bytes / skv_cache_create. */
+ * the codes are converted to f16 on the way into mma.sync.  The pre-fill calls
+ * run an mma.sync kernel that converts the codes the same way (prefill variant 2,
+ * the tcgen05 kernel, reads bf16 pages only: SKV_ERR_UNSUPPORTED); skv_gather
+ * returns SKV_ERR_UNSUPPORTED (use skv_gather_fp8).  Same arguments and errors
+ * as skv_cache_pool_bytes / skv_cache_create. */
 int skv_cache_pool_bytes_fp8(int n_layers, const int32_t *r, int kv_heads, int head_dim,
                              int page_size, int64_t max_pages, size_t *out_bytes);
 int skv_cache_create_fp8(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, int head_dim,

@@ -743,16 +743,18 @@ int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens,
                  const int32_t *seq_lens, void *out, int batch, int max_q_len, int q_heads, int pt_stride,
                  float scale, void *stream)
 {
-    if (c->fp8) return SKV_ERR_UNSUPPORTED;            // pre-fill reads bf16 pages only
     if (!Q || !cu_q_lens || !page_table || !seq_lens || !out || pt_stride <= 0 || max_q_len <= 0) return SKV_ERR_ARG;
     if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
     if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
     const int G = q_heads / c->kv_heads;
-    const bool can_umma = prefill_umma_supported(c->head_dim, G) && aligned(Q, 16) && aligned(out, 16) &&
+    // FP8 pages: the mma.sync kernel that converts the codes on the way in (the tcgen05 kernel reads bf16 pages)
+    const bool can_umma = !c->fp8 && prefill_umma_supported(c->head_dim, G) && aligned(Q, 16) && aligned(out, 16) &&
                           prefill_umma_smem_bytes(c->head_dim) <= (size_t)c->max_smem_optin;
     if (c->prefill_variant == 2 && !can_umma) return SKV_ERR_UNSUPPORTED;
     const bool umma = c->prefill_variant == 2 || (c->prefill_variant == 0 && can_umma);
-    if (!umma && prefill_smem_bytes(c->head_dim) > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
+    if (!umma && (c->fp8 ? prefill_fp8_smem_bytes(c->head_dim) : prefill_smem_bytes(c->head_dim)) > (size_t)c->max_smem_optin)
+        return SKV_ERR_UNSUPPORTED;
+    if (c->fp8 && !aligned(Q, 8)) return SKV_ERR_ARG;
     PrefillParams p;
     p.layer_base = c->layer_base(c->slot[(size_t)src]);
     p.page_stride = (int64_t)c->page_bytes;
@@ -771,8 +773,10 @@ int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens,
     p.status = c->status_word();
     const int tq = umma ? prefill_umma_tile_tokens(G) : prefill_tile_tokens(G);
     const int q_tiles = (max_q_len + tq - 1) / tq;
-    const cudaError_t le = umma ? launch_prefill_umma(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream))
-                                : launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, static_cast<cudaStream_t>(stream));
+    const cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const cudaError_t le = umma     ? launch_prefill_umma(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st)
+                           : c->fp8 ? launch_prefill_fp8(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st)
+                                    : launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st);
     if (le != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;

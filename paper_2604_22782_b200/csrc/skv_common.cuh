@@ -165,6 +165,8 @@ cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, int kernel
                                  int warps, int stages, bool pdl, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 size_t prefill_smem_bytes(int D);
+size_t prefill_fp8_smem_bytes(int D);
+cudaError_t launch_prefill_fp8(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
 int prefill_tile_tokens(int G);                 // query tokens per CTA tile
 cudaError_t launch_prefill(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
 // the tcgen05 (UMMA / tensor-memory) variant

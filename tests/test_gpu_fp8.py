@@ -175,7 +175,29 @@ def test_whole_step_and_unsupported_calls():
     with pytest.raises(SkvError) as e:
         dw.cache.skv_gather(0, dw.slot_new, t["K"][0], t["V"][0])
     assert e.value.status == SKV_ERR_UNSUPPORTED
+    dw.cache.skv_set_prefill_variant(2)              # the tcgen05 pre-fill kernel reads bf16 pages only
     inp = harness.prefill_inputs(dw, 0, torch.ones(lens.numel(), dtype=torch.int32))
     with pytest.raises(SkvError) as e:
         dw.cache.skv_prefill_attn(0, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, torch.empty_like(inp["Q"]), 1)
     assert e.value.status == SKV_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 128), (8, 1, 128), (6, 2, 64), (6, 2, 128)])
+def test_prefill_on_fp8_pages(Hq, Hkv, D):
+    """Pre-fill attention over FP8 pages (whole prompts, chunks, single rows) against the oracle's rows over the
+    dequantised values; unused slots of the pool hold NaN codes and NaN scales."""
+    lens = torch.tensor([1, 15, 16, 17, 63, 64, 65, 100, 257, 700], dtype=torch.int32)
+    w = W.Workload("fp8_pf", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=109, kv_std=1.3)
+    harness, dw = _setup(w, lens, poison=True)
+    o, _, _, _ = _oracle(dw, range(3))
+    for layer, q_lens in ((0, lens), (1, lens), (2, lens), (1, torch.tensor([1, 7, 16, 1, 40, 0, 65, 3, 200, 129], dtype=torch.int32)),
+                          (2, torch.ones(lens.numel(), dtype=torch.int32))):
+        inp = harness.prefill_inputs(dw, layer, q_lens)
+        out = torch.full_like(inp["Q"], float("nan"))
+        dw.cache.skv_prefill_attn(layer, inp["Q"], inp["cu_q_lens"], dw.page_table, dw.seq_lens, out, max(1, int(q_lens.max())))
+        torch.cuda.synchronize()
+        ref = o.attn_rows(layer, inp["Q"].cpu(), inp["q_seq"], inp["q_pos"])
+        err = (out.cpu().double() - ref).abs()
+        assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {layer}: max abs err {err.max().item()}"
+        assert torch.isfinite(out.float()).all()
+    assert dw.cache.skv_get_status() == 0
