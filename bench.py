@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel,
 # from the ncu capture summarised under profiles/ (None until captured)
-NCU_TRAFFIC_BYTES = {"llama3_8b": 343200000}
+NCU_TRAFFIC_BYTES = {"llama3_8b": 343470000}
 DEFAULT_L2_KEEP = 35     # the library's default share of each block range kept in L2 for the next layer
 
 
