@@ -100,102 +100,70 @@ __device__ __forceinline__ void quantize_row(const uint16_t *row, int PER, int l
     c23 = pack_e4m3x2(__fmul_rn(x[2], inv), __fmul_rn(x[3], inv));
 }
 
-// One warp per (token, kv head); grid.y picks K or V, grid.z the owner layer.  A token at a time
-// costs scattered small stores (V is dim-major: one byte in each of D rows; K: D/16 pieces of 4
-// bytes per lane).  When the 16 tokens of a whole page arrive together and in order (a prompt being
-// appended), the warp of the page's first token quantises all 16 rows and writes 16 bytes per
-// store, and the warps of the other 15 tokens have nothing to do.
-__device__ __forceinline__ void append_fp8_row(const AppendFp8Params &p, int64_t warp, int lane);
-
-__global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
+// The 16 rows of a whole page (tokens t0 .. t0+15 of the call, in slot order) by one warp, 16 bytes per store.
+__device__ __forceinline__ void append_fp8_page(const AppendFp8Params &p, int64_t t0, int64_t page, int h, int which,
+                                                int64_t layer, int lane)
 {
-    const int lane = threadIdx.x & 31;
-    // the warps of a bounded grid go through the (token, kv head) rows: most rows of a prompt are done by
-    // their page's first row and end at once, which a loop iteration does more cheaply than a CTA launch
-    // (rows counted head-major and an odd number of warps in the grid: a warp then meets every position inside
-    // a page in turn, instead of always the pages' first rows or never one)
-    const int64_t n_rows = p.n_tokens * p.Hkv, stride = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); warp < n_rows; warp += stride)
-        append_fp8_row(p, warp, lane);
-}
-
-__device__ __forceinline__ void append_fp8_row(const AppendFp8Params &p, int64_t warp, int lane)
-{
-    const int h = (int)(warp / p.n_tokens);
-    const int64_t tok = warp - (int64_t)h * p.n_tokens;
-    const int64_t slot = p.slot_map[tok];
-    if (slot < 0) return;
-    if (slot >= p.n_slots) {
-        if (h == 0 && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
-        return;
-    }
-    const int64_t page = slot / PAGE;
-    const int off = (int)(slot - page * PAGE);
-    const int which = blockIdx.y;
-    const int64_t layer = blockIdx.z;
-    const int D = p.D, PER = D / 32;                  // 4 values per lane at D = 128, 2 at D = 64
+    const int D = p.D, PER = D / 32;
     const uint16_t *rows = (which ? p.V : p.K) + (layer * p.n_tokens * p.Hkv + h) * D;      // row of token t: + t * Hkv * D
     uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
-    // do tokens tok-off .. tok-off+15 of this call carry the page's 16 slots in order?
-    const int64_t t0 = tok - off;
-    bool whole_page = t0 >= 0 && t0 + PAGE <= p.n_tokens;
-    if (whole_page) {
-        const int64_t s_l = lane < PAGE ? p.slot_map[t0 + lane] : 0;
-        whole_page = __all_sync(0xFFFFFFFFu, lane >= PAGE || s_l == page * PAGE + lane);
-    }
-    if (whole_page) {
-        if (off != 0) return;
-        if (which == 0) {
-            // K: lane = (token q of this round, 16-dim chunk c); a chunk of a token is one 16-byte piece of the page
-            const int CH = D / 16, TPI = 32 / CH;          // 8 chunks x 4 tokens per round at D = 128
-            const int c = lane % CH, q = lane / CH;
-            for (int t = q; t < PAGE; t += TPI) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(rows + (t0 + t) * p.Hkv * D + 16 * c);
-                const uint4 a = __ldg(src), b = __ldg(src + 1);
-                const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-                float x[16];
-                float amax = 0.f;
+    if (which == 0) {
+        // K: lane = (token q of this round, 16-dim chunk c); a chunk of a token is one 16-byte piece of the page
+        const int CH = D / 16, TPI = 32 / CH;          // 8 chunks x 4 tokens per round at D = 128
+        const int c = lane % CH, q = lane / CH;
+        for (int t = q; t < PAGE; t += TPI) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(rows + (t0 + t) * p.Hkv * D + 16 * c);
+            const uint4 a = __ldg(src), b = __ldg(src + 1);
+            const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            float x[16];
+            float amax = 0.f;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    x[2 * i] = bf16_lo(w[i]);
-                    x[2 * i + 1] = bf16_hi(w[i]);
-                    amax = fmaxf(amax, fmaxf(fabsf(x[2 * i]), fabsf(x[2 * i + 1])));
-                }
-                for (int d = 1; d < CH; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
-                const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
-                uint32_t o[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    o[i] = pack_e4m3x2(__fmul_rn(x[4 * i], inv), __fmul_rn(x[4 * i + 1], inv)) |
-                           (pack_e4m3x2(__fmul_rn(x[4 * i + 2], inv), __fmul_rn(x[4 * i + 3], inv)) << 16);
-                *reinterpret_cast<uint4 *>(blk + fp8_k_pos(D, t, 16 * c)) = make_uint4(o[0], o[1], o[2], o[3]);
-                if (c == 0) *reinterpret_cast<float *>(blk + fp8_ks_off(D) + 4 * t) = __fdiv_rn(amax, 448.f);
+            for (int i = 0; i < 8; ++i) {
+                x[2 * i] = bf16_lo(w[i]);
+                x[2 * i + 1] = bf16_hi(w[i]);
+                amax = fmaxf(amax, fmaxf(fabsf(x[2 * i]), fabsf(x[2 * i + 1])));
             }
-            return;
-        }
-        {
-            uint32_t v[4][4] = {};                 // [dim of the lane][4 tokens per word]
-            float my_scale = 0.f;
+            for (int d = 1; d < CH; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+            const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+            uint32_t o[4];
 #pragma unroll
-            for (int t = 0; t < PAGE; ++t) {
-                uint32_t c01, c23;
-                float amax;
-                quantize_row(rows + (t0 + t) * p.Hkv * D, PER, lane, c01, c23, amax);
-                const int sh = 8 * (t & 3);
-                v[0][t >> 2] |= (c01 & 0xFFu) << sh;
-                v[1][t >> 2] |= (c01 >> 8) << sh;
-                v[2][t >> 2] |= (c23 & 0xFFu) << sh;
-                v[3][t >> 2] |= (c23 >> 8) << sh;
-                if (lane == t) my_scale = __fdiv_rn(amax, 448.f);
-            }
-            uint4 *dst = reinterpret_cast<uint4 *>(blk + fp8_v_off(D) + (lane * PER) * PAGE);
-#pragma unroll
-            for (int d = 0; d < 4; ++d)
-                if (d < PER) dst[d] = make_uint4(v[d][0], v[d][1], v[d][2], v[d][3]);
-            if (lane < PAGE) *reinterpret_cast<float *>(blk + fp8_vs_off(D) + 4 * lane) = my_scale;
-            return;
+            for (int i = 0; i < 4; ++i)
+                o[i] = pack_e4m3x2(__fmul_rn(x[4 * i], inv), __fmul_rn(x[4 * i + 1], inv)) |
+                       (pack_e4m3x2(__fmul_rn(x[4 * i + 2], inv), __fmul_rn(x[4 * i + 3], inv)) << 16);
+            *reinterpret_cast<uint4 *>(blk + fp8_k_pos(D, t, 16 * c)) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (c == 0) *reinterpret_cast<float *>(blk + fp8_ks_off(D) + 4 * t) = __fdiv_rn(amax, 448.f);
         }
+        return;
     }
+    uint32_t v[4][4] = {};                 // [dim of the lane][4 tokens per word]
+    float my_scale = 0.f;
+#pragma unroll
+    for (int t = 0; t < PAGE; ++t) {
+        uint32_t c01, c23;
+        float amax;
+        quantize_row(rows + (t0 + t) * p.Hkv * D, PER, lane, c01, c23, amax);
+        const int sh = 8 * (t & 3);
+        v[0][t >> 2] |= (c01 & 0xFFu) << sh;
+        v[1][t >> 2] |= (c01 >> 8) << sh;
+        v[2][t >> 2] |= (c23 & 0xFFu) << sh;
+        v[3][t >> 2] |= (c23 >> 8) << sh;
+        if (lane == t) my_scale = __fdiv_rn(amax, 448.f);
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(blk + fp8_v_off(D) + (lane * PER) * PAGE);
+#pragma unroll
+    for (int d = 0; d < 4; ++d)
+        if (d < PER) dst[d] = make_uint4(v[d][0], v[d][1], v[d][2], v[d][3]);
+    if (lane < PAGE) *reinterpret_cast<float *>(blk + fp8_vs_off(D) + 4 * lane) = my_scale;
+}
+
+// One row (token tok at offset off of its page) by one warp: scattered small stores (V is dim-major: one byte
+// in each of D rows; K: 4 bytes per lane).
+__device__ __forceinline__ void append_fp8_token(const AppendFp8Params &p, int64_t tok, int64_t page, int off, int h,
+                                                 int which, int64_t layer, int lane)
+{
+    const int D = p.D, PER = D / 32;                  // 4 values per lane at D = 128, 2 at D = 64
+    const uint16_t *rows = (which ? p.V : p.K) + (layer * p.n_tokens * p.Hkv + h) * D;
+    uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
     uint32_t c01, c23;
     float amax;
     quantize_row(rows + tok * p.Hkv * D, PER, lane, c01, c23, amax);
@@ -214,6 +182,83 @@ __device__ __forceinline__ void append_fp8_row(const AppendFp8Params &p, int64_t
     }
     if (lane == 0)
         *reinterpret_cast<float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * off) = __fdiv_rn(amax, 448.f);
+}
+
+// Small calls (a decode step: one token per sequence): one warp per (token, kv head) row, the warps of a
+// bounded grid looping over the rows; grid.y picks K or V, grid.z the owner layer.  When the 16 tokens of a
+// whole page do arrive together and in order, the warp of the page's first row does the page and the other
+// 15 rows have nothing to do.
+__global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
+{
+    const int lane = threadIdx.x & 31;
+    // (rows counted head-major and an odd number of warps in the grid: a warp then meets every position inside
+    // a page in turn, instead of always the pages' first rows or never one)
+    const int64_t n_rows = p.n_tokens * p.Hkv, stride = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); warp < n_rows; warp += stride) {
+        const int h = (int)(warp / p.n_tokens);
+        const int64_t tok = warp - (int64_t)h * p.n_tokens;
+        const int64_t slot = p.slot_map[tok];
+        if (slot < 0) continue;
+        if (slot >= p.n_slots) {
+            if (h == 0 && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
+            continue;
+        }
+        const int64_t page = slot / PAGE;
+        const int off = (int)(slot - page * PAGE);
+        // do tokens tok-off .. tok-off+15 of this call carry the page's 16 slots in order?
+        const int64_t t0 = tok - off;
+        bool whole_page = t0 >= 0 && t0 + PAGE <= p.n_tokens;
+        if (whole_page) {
+            const int64_t s_l = lane < PAGE ? p.slot_map[t0 + lane] : 0;
+            whole_page = __all_sync(0xFFFFFFFFu, lane >= PAGE || s_l == page * PAGE + lane);
+        }
+        if (!whole_page) append_fp8_token(p, tok, page, off, h, (int)blockIdx.y, blockIdx.z, lane);
+        else if (off == 0) append_fp8_page(p, t0, page, h, (int)blockIdx.y, blockIdx.z, lane);
+    }
+}
+
+// Large calls (a prompt): one warp per (group of 16 consecutive tokens of the call, kv head).  The warp looks at
+// the slots of its tokens and of the 15 tokens on either side, finds the whole page that starts inside its group
+// (at most one: its 16 tokens arrive together and in slot order), does that page 16 bytes per store, and does
+// its tokens that belong to no whole page one row at a time.  Same result as the kernel above for any slot map.
+__global__ void __launch_bounds__(COPY_THREADS) append_fp8_groups_kernel(AppendFp8Params p)
+{
+    constexpr unsigned ALL = 0xFFFFFFFFu;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_groups = (p.n_tokens + PAGE - 1) / PAGE, n_items = n_groups * p.Hkv;
+    const int64_t stride = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t item = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); item < n_items; item += stride) {
+        const int h = (int)(item / n_groups);
+        const int64_t i0 = (item - (int64_t)h * n_groups) * PAGE;
+        // slots of tokens i0-15 .. i0+30: window index x = -15 .. 16 in w0 (lane x+15), 17 .. 30 in w1 (lane x-17)
+        auto slot_of = [&](int64_t i) -> long long { return (i >= 0 && i < p.n_tokens) ? (long long)p.slot_map[i] : -1ll; };
+        const long long w0 = slot_of(i0 - 15 + lane), w1 = lane < 14 ? slot_of(i0 + 17 + lane) : -1ll;
+        auto at = [&](int x) -> long long {               // every lane calls it (with its own x)
+            const long long a = __shfl_sync(ALL, w0, (x + 15) & 31), b = __shfl_sync(ALL, w1, (x - 17) & 31);
+            return x <= 16 ? a : b;
+        };
+        const int l = lane & 15;                          // lanes 16..31 repeat lanes 0..15
+        const long long mine = at(l);
+        const bool valid = i0 + l < p.n_tokens && mine >= 0 && mine < p.n_slots;
+        if (lane < PAGE && i0 + l < p.n_tokens && mine >= p.n_slots && h == 0 && blockIdx.y == 0) atomicOr(p.status, STATUS_BOUNDS);
+        const int off = (int)(mine & (PAGE - 1));
+        const int c = l - off;                            // where the token's page would start in the window (>= -15)
+        bool covered = valid;
+#pragma unroll
+        for (int k = 0; k < PAGE; ++k) covered = (at(c + k) == mine - off + k) && covered;
+        const unsigned starts = __ballot_sync(ALL, lane < PAGE && covered && off == 0);
+        const unsigned loose = __ballot_sync(ALL, lane < PAGE && valid && !covered);
+        if (starts) {
+            const int ls = __ffs(starts) - 1;
+            const long long s0 = __shfl_sync(ALL, mine, ls);
+            append_fp8_page(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane);
+        }
+        for (unsigned m = loose; m; m &= m - 1) {
+            const int lt = __ffs(m) - 1;
+            const long long st = __shfl_sync(ALL, mine, lt);
+            append_fp8_token(p, i0 + lt, st / PAGE, (int)(st & (PAGE - 1)), h, (int)blockIdx.y, blockIdx.z, lane);
+        }
+    }
 }
 
 // read-back: codes as [n][Hkv][D] for both K and V, scales as [n][Hkv]
@@ -278,12 +323,16 @@ namespace skv {
 
 cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s)
 {
-    const int64_t warps = p.n_tokens * p.Hkv;
-    int64_t blocks = (warps + 6) / 7;                  // 7 warps per CTA
-    if (blocks == 0) return cudaSuccess;
+    if (p.n_tokens == 0) return cudaSuccess;
     if (n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
-    if (blocks > 4095) blocks = 4095;                  // the kernel's warps loop over the rows; 7 x 4095 is odd
-    append_fp8_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), 224, 0, s>>>(p);
+    // 7 warps per CTA and at most 4095 CTAs: the kernels' warps loop over their items, and 7 x 4095 is odd
+    const bool groups = p.n_tokens >= 512;
+    const int64_t items = groups ? ((p.n_tokens + PAGE - 1) / PAGE) * p.Hkv : p.n_tokens * p.Hkv;
+    int64_t blocks = (items + 6) / 7;
+    if (blocks > 4095) blocks = 4095;
+    const dim3 grid((unsigned)blocks, 2, (unsigned)n_layers);
+    if (groups) append_fp8_groups_kernel<<<grid, 224, 0, s>>>(p);
+    else append_fp8_kernel<<<grid, 224, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -102,6 +102,54 @@ def test_rows_of_very_different_magnitude():
     assert bool((err <= ATOL + RTOL * row_max).all()), f"max abs err {err.max().item()} at |ref| up to {ref.abs().max().item()}"
 
 
+@pytest.mark.parametrize("n_extra", [0, 700])     # below and above the size at which the page-granular update kernel takes over
+def test_update_with_arbitrary_slot_maps(n_extra):
+    """skv_append on FP8 pages with slot maps that mix whole pages at odd positions of the call, pages in reverse
+    order, pages with a skipped token, scattered single slots and runs of whole pages: every written slot reads
+    back as the oracle quantiser's codes and scales, for both update kernels."""
+    from oracle import quantize_e4m3
+    from paper_2604_22782_b200 import harness
+    Hkv, D = 2, 128
+    n_pages = 120
+    lens = torch.tensor([n_pages * 16], dtype=torch.int32)
+    w = W.Workload("fp8_slots", 1, 4, Hkv, D, 16, 1, 0, 0, "explicit", explicit_r=(0,), seed=113)
+    dw = harness.setup(w, lens=lens, fp8=True)
+    g = torch.Generator().manual_seed(17)
+    pages = torch.randperm(n_pages, generator=g).tolist()
+    page = lambda: pages.pop() * 16
+    parts = [torch.tensor([page() + 3, page() + 9, page()])]                       # three loose tokens first: pages start at odd positions
+    parts.append(page() + torch.arange(16))                                        # a whole page in order
+    parts.append(page() + torch.arange(15, -1, -1))                                # a page in reverse order
+    hole = page() + torch.arange(16); hole[5] = -1; parts.append(hole)             # a page with a skipped token
+    parts.append(torch.cat([page() + torch.arange(16) for _ in range(12)]))        # a run of whole pages
+    parts.append(torch.tensor([page() + i for i in (1, 15, 7)]))                   # loose tokens of one page
+    parts.append(page() + torch.arange(8))                                         # half a page
+    parts.append(torch.cat([page() + torch.arange(16) for _ in range(3)]))
+    if n_extra:
+        rest = torch.cat([page() + torch.arange(16) for _ in range(n_extra // 16)])
+        parts.append(rest[torch.randperm(rest.numel(), generator=g)][: n_extra // 2])    # scattered
+        parts.append(torch.cat([page() + torch.arange(16) for _ in range(20)]))
+    slots = torch.cat(parts).to(torch.int64)
+    n = slots.numel()
+    K = (torch.randn((n, Hkv, D), generator=g) * 1.5).to(torch.bfloat16)
+    V = (torch.randn((n, Hkv, D), generator=g) * torch.exp2(torch.randint(-6, 7, (n, 1, 1), generator=g).float())).to(torch.bfloat16)
+    dw.cache.skv_append(0, K.to(dw.device), V.to(dw.device), slots.to(dw.device))
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    keep = slots >= 0
+    kc = torch.zeros((int(keep.sum()), Hkv, D), dtype=torch.uint8, device=dw.device)
+    vc = torch.zeros_like(kc)
+    ks = torch.zeros((kc.shape[0], Hkv), dtype=torch.float32, device=dw.device)
+    vs = torch.zeros_like(ks)
+    dw.cache.skv_gather_fp8(0, slots[keep].to(dw.device), kc, vc, ks, vs)
+    torch.cuda.synchronize()
+    okc, oks = quantize_e4m3(K[keep])
+    ovc, ovs = quantize_e4m3(V[keep])
+    assert torch.equal(kc.cpu(), okc) and torch.equal(vc.cpu(), ovc)
+    assert torch.equal(ks.cpu().view(torch.int32), oks.view(torch.int32))
+    assert torch.equal(vs.cpu().view(torch.int32), ovs.view(torch.int32))
+
+
 def test_many_short_sequences():
     """Hundreds of sequences of at most one tile (128 tokens), more (sequence, kv head) segments than workers: every
     worker of the tcgen05 kernel goes through several one-tile runs back to back, the case in which its roles are
