@@ -17,7 +17,8 @@
  *     query head h reads KV head floor(h / (q_heads / kv_heads)).
  *   - Cache memory is allocated for owners only, so its size is
  *     2 x |owners| x kv_heads x head_dim x 2 bytes per token (Section 1
- *     footnote with #layers -> |S|; Section 4.3: "scales as 1/g").
+ *     footnote with #layers -> |S|; Section 4.3: with groups of g layers the
+ *     cache shrinks by the factor g).
  *
  * Conventions
  *   - Every function returns an int status: SKV_OK (0) or a negative
@@ -188,7 +189,8 @@ int skv_gather_fp8(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t
 /* ---- Algorithm 2 "Load + Attn": decode attention -------------------------- */
 
 /* Bytes of device workspace skv_decode_attn needs for this batch / head count
- * under the CURRENT launch shape (ask again after skv_set_decode_tuning).
+ * under the CURRENT launch shape (ask again after skv_set_decode_tuning or
+ * skv_set_decode_variant).
  * Independent of sequence lengths.  It holds, twice (two calls of a chain may
  * overlap), the split partials and a page-count prefix. */
 int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, size_t *out_bytes);
@@ -201,16 +203,24 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
  *   page_table  device int32 [batch][pt_stride]; entries past a sequence's
  *               last page are never read
  *   seq_lens    device int32 [batch]; tokens to attend, including the one just
- *               appended; 0 gives an all-zero output row
+ *               appended; 0 gives an all-zero output row.  A length that needs
+ *               more than pt_stride pages is cut to pt_stride * page_size tokens
+ *               on the device and raises SKV_ERR_BOUNDS in the device status
+ *               (no page id is read past the end of a page_table row)
  *   out         device bf16 [batch][q_heads][head_dim]
  *   scale       <= 0 selects 1/sqrt(head_dim)
  *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes; needs
  *               no initialisation and may be shared by calls on one stream.
- * Two launches.  Split-K (flash-decoding): every warp streams an equal share
- * of the (sequence, kv head, page) blocks and writes, for each (sequence, kv
- * head) its share touches, an fp32 partial (max, sum, output).  Merge: one warp
- * per (sequence, kv head) combines its partials by log-sum-exp and writes the
- * bf16 rows.  Slots past seq_lens[b] in the last page contribute nothing
+ * Two launches.  Split-K (flash-decoding): the (sequence, kv head, page) blocks
+ * of the call form one list that is cut into equal contiguous ranges, one per
+ * worker, whatever the mix of lengths; a worker streams its range through
+ * shared memory and leaves, for each (sequence, kv head) its range touches, an
+ * fp32 partial (max, sum, output).  Merge: one warp per (sequence, kv head)
+ * combines its partials by log-sum-exp and writes the bf16 rows.  The worker is
+ * a CTA per SM whose warps share one ring of stages and combine their states in
+ * shared memory -- it then finishes every (sequence, kv head) that lies inside
+ * its range itself and the merge launch has only the others left -- or a single
+ * warp (skv_set_decode_worker).  Slots past seq_lens[b] in the last page contribute nothing
  * whatever they contain.  No host synchronisation; sequence lengths are read
  * on the device.  The split-K launch waits for the work before it in the
  * stream before it reads anything; with skv_set_decode_overlap on, the merge
@@ -284,9 +294,9 @@ int skv_decode_merge(skv_cache *cache, void *out, int batch, int q_heads, void *
  * One launch, no workspace: a CTA owns 64 or 128 query rows (that many /
  * (q_heads/kv_heads) tokens x the query heads of one kv head) and streams the
  * pages they see (skv_set_prefill_variant).
- * Errors as skv_decode_attn; a sequence with q_len_b > seq_lens[b] or
- * q_len_b > max_q_len raises SKV_ERR_BOUNDS in the device status and its rows
- * are left untouched. */
+ * Errors as skv_decode_attn; a sequence with q_len_b > seq_lens[b],
+ * q_len_b > max_q_len or seq_lens[b] > pt_stride * page_size raises
+ * SKV_ERR_BOUNDS in the device status and its rows are left untouched. */
 int skv_prefill_attn(skv_cache *cache, int layer, const void *Q, const int32_t *cu_q_lens,
                      const int32_t *page_table, const int32_t *seq_lens, void *out, int batch,
                      int max_q_len, int q_heads, int pt_stride, float scale, void *stream);
@@ -363,7 +373,7 @@ int skv_set_decode_variant(skv_cache *cache, int variant);
 /* Launch shape of the split-K kernel (default: 8 warps per SM with two 8 KB
  * stages each, as 2 warps x 4 CTAs per SM for the tensor-core kernel and
  * 1 warp x 8 CTAs per SM for the CUDA-core kernel): warps per CTA (1..16), pipeline stages
- * per warp (2..8) and CTAs per SM (1..8); 0 keeps the current value.
+ * per warp (1..8) and CTAs per SM (1..8); 0 keeps the current value (other values: SKV_ERR_ARG).
  * SKV_ERR_UNSUPPORTED if the combination does not fit in shared memory. */
 int skv_set_decode_tuning(skv_cache *cache, int warps_per_cta, int stages, int ctas_per_sm);
 
@@ -381,6 +391,37 @@ int skv_set_prefill_variant(skv_cache *cache, int variant);
  * launches, and skv_decode_step goes layer by layer through skv_append /
  * skv_decode_attn. */
 int skv_set_decode_overlap(skv_cache *cache, int enabled);
+
+/* Which worker the split-K pass of a stand-alone attention call uses
+ * (skv_decode_attn, skv_decode_attn_static; the two-call form skv_decode_splitk +
+ * skv_decode_merge and the chained launches of skv_decode_step always use warps).
+ *   mode 0 (default) or 2: a CTA per SM -- `consumers` warps (1..12, default 8; 0
+ *        keeps the current value) share one ring of `stages` 8 KB stages (2..26;
+ *        0, the default: as many as shared memory allows, at most 20) filled by a
+ *        producer warp, take its blocks in turn and combine their running states
+ *        in shared memory at the end of every (sequence, kv head);
+ *   mode 1: a warp per range, launch shape from skv_set_decode_tuning.
+ * FP8 pages at head_dim 128 keep their tcgen05 kernel either way.  Results agree
+ * to rounding (the order of the sums differs). */
+int skv_set_decode_worker(skv_cache *cache, int mode, int consumers, int stages);
+
+/* Early fetch for stand-alone attention calls (skv_decode_attn, skv_decode_attn_static,
+ * skv_decode_splitk; needs skv_set_decode_overlap on).  0 (default): a split-K
+ * launch waits for the kernel before it in the stream before it reads anything.
+ * 1: it reads seq_lens and page_table, and starts copying pages, while that
+ * kernel is still running, and waits for it only before it reads Q and before it
+ * copies the LAST page of any sequence.  In a decoder this is what the data flow
+ * allows (Algorithm 2: Q of layer l is computed from the output of layer l-1, and
+ * the Update of layer l adds one token, which lands in the sequence's last page;
+ * everything else the call reads is older), and it takes the launch, the length
+ * scan and the first page copies off the critical path: skv_append lets the
+ * launch after it start at once, so on an owner layer they run beside the update.
+ * The caller's promise when switching it on: the kernel directly before each such
+ * call in its stream writes neither seq_lens nor page_table nor any cached token
+ * other than tokens in the last page of a sequence (skv_append of the step's new
+ * token is such a kernel; so is any kernel that only produces Q).  Results are
+ * identical. */
+int skv_set_decode_early_fetch(skv_cache *cache, int enabled);
 
 /* L2 reuse between consecutive layers that read the same owner (the paper's
  * depth-wise sharing makes them stream identical pages): with keep_percent > 0
@@ -400,8 +441,9 @@ int skv_set_host_step(skv_cache *cache, int groups, int ramp);
 /* Tracing: while a device buffer of at least 32 * skv_decode_worker_count bytes
  * is set, every split-K launch records four uint64 per worker (warp): SM id,
  * kernel-entry time, time its first page arrived, exit time (global timer, ns).
- * NULL switches tracing off.  skv_decode_worker_count = SMs * CTAs per SM *
- * warps per CTA under the current tuning. */
+ * NULL switches tracing off.  skv_decode_worker_count = the larger of SMs *
+ * CTAs per SM * warps per CTA under the current tuning and SMs * consumer warps
+ * of the CTA-per-SM kernel (which records one entry per consumer warp). */
 int skv_set_trace_buffer(skv_cache *cache, void *device_buffer, size_t bytes);
 int skv_decode_worker_count(const skv_cache *cache);
 

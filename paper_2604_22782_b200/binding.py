@@ -76,6 +76,8 @@ lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
 lib.skv_set_prefill_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
+lib.skv_set_decode_early_fetch.argtypes = [_vp, _int]
+lib.skv_set_decode_worker.argtypes = [_vp, _int, _int, _int]
 lib.skv_set_host_step.argtypes = [_vp, _int, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
 lib.skv_decode_worker_count.argtypes = [_vp]
@@ -359,6 +361,12 @@ class SkvCache:
 
     def skv_set_decode_overlap(self, enabled: int) -> None:
         _check(lib.skv_set_decode_overlap(self._h, enabled), "skv_set_decode_overlap")
+
+    def skv_set_decode_worker(self, mode: int, consumers: int = 0, stages: int = 0) -> None:
+        _check(lib.skv_set_decode_worker(self._h, mode, consumers, stages), "skv_set_decode_worker")
+
+    def skv_set_decode_early_fetch(self, enabled: int) -> None:
+        _check(lib.skv_set_decode_early_fetch(self._h, enabled), "skv_set_decode_early_fetch")
 
     def skv_set_decode_l2_reuse(self, keep_percent: int) -> None:
         _check(lib.skv_set_decode_l2_reuse(self._h, keep_percent), "skv_set_decode_l2_reuse")

@@ -9,7 +9,37 @@
 #include <string.h>
 #include <vector>
 
+#include <mutex>
+
 using namespace skv;
+
+namespace skv {
+cudaError_t ensure_dynamic_smem_fn(const void *kernel, size_t smem)
+{
+    struct Granted { const void *kernel; int dev; int smem; };
+    static Granted table[128];
+    static int used = 0;
+    static std::mutex lock;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> hold(lock);
+    Granted *g = nullptr;
+    for (int i = 0; i < used && !g; ++i)
+        if (table[i].kernel == kernel && table[i].dev == dev) g = &table[i];
+    if (g && (int)smem <= g->smem) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (!g && used < 128) {
+        g = &table[used++];
+        g->kernel = kernel;
+        g->dev = dev;
+        g->smem = 0;
+    }
+    if (g) g->smem = (int)smem;
+    return cudaSuccess;
+}
+}  // namespace skv
 
 struct skv_cache {
     int n_layers = 0, kv_heads = 0, head_dim = 0, page_size = 0, n_owners = 0;
@@ -22,11 +52,18 @@ struct skv_cache {
     size_t page_bytes = 0;           // one page of one owner layer
     int sm_count = 0;
     int max_smem_optin = 0;
+    int l2_bytes = 0;
     DecodeTuning tune{0, 2, 2, 4, 1};
     bool fp8 = false;                // pages hold E4M3 codes + per-row scales instead of bf16
     int prefill_variant = 0;         // 0 auto (tcgen05 where supported), 1 mma.sync kernel, 2 tcgen05 kernel
     bool shape_is_default = true;    // until skv_set_decode_tuning is called: the CUDA-core kernel runs as 1 x 2 x 8
     int l2_keep_pct = 35;            // > 0: consecutive layers that read one owner walk it in opposite directions
+    bool early_fetch = false;        // stand-alone attention calls fill their rings before waiting for the kernel before them
+    int worker_mode = 0;             // 0 auto (CTA per range for stand-alone calls, warp per range inside chains),
+                                     // 1 warp per range always, 2 CTA per range wherever it applies
+    int cta_consumers = 8;           // consumer warps per CTA of the CTA-per-range kernel
+    int cta_stages = 0;              // its ring depth; 0 = as deep as shared memory allows, up to 20
+    bool cta_in_turn = true;         // its consumers take the blocks in turn (reproducible) instead of first come first served
     std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
     std::vector<uint8_t> walk_keep;      // per layer: the next layer reads the same owner
     int64_t launches = 0;
@@ -103,10 +140,34 @@ WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int
 // FP8 pages go to the tcgen05 kernel (a worker is a CTA there) unless the mma.sync variant is asked for
 bool fp8_on_umma(const skv_cache *c) { return c->fp8 && c->tune.variant != 2 && decode_fp8_umma_supported(c->head_dim, 1); }
 
+// Workers of a warp-per-range (or tcgen05) split-K launch under the current variant and launch shape.  A
+// handle without device memory (accounting only) has no device to ask and counts a B200's 148 SMs.
 int n_workers_of(const skv_cache *c)
 {
-    if (fp8_on_umma(c)) return c->sm_count * decode_fp8_umma_ctas_per_sm();
-    return c->sm_count * c->tune.ctas_per_sm * c->tune.warps;
+    const int sm = c->sm_count > 0 ? c->sm_count : 148;
+    if (fp8_on_umma(c)) return sm * decode_fp8_umma_ctas_per_sm();
+    return sm * c->tune.ctas_per_sm * c->tune.warps;
+}
+
+// Workers of a CTA-per-range launch: one CTA per SM.
+int n_cta_workers_of(const skv_cache *c) { return c->sm_count > 0 ? c->sm_count : 148; }
+
+// The workspace is sized for whichever kernel leaves more partials (a call may run either).
+int n_workers_max(const skv_cache *c)
+{
+    const int a = n_workers_of(c), b = n_cta_workers_of(c);
+    return a > b ? a : b;
+}
+
+// Ring depth of the CTA-per-range kernel for this shape: the handle's setting, else as many stages as fit
+// (at most 20); 0 if not even two fit.
+int cta_stages_for(const skv_cache *c, int batch, int G)
+{
+    int S = c->cta_stages > 0 ? c->cta_stages : 20;
+    while (S >= 2 && decode_cta_smem_bytes(c->head_dim, batch, G, c->cta_consumers, S, c->fp8) > (size_t)c->max_smem_optin) --S;
+    // by default a whole number of rounds of the consumers (a stage then always serves the same consumer)
+    if (c->cta_stages == 0 && S >= 2 * c->cta_consumers) S -= S % c->cta_consumers;
+    return S >= 2 ? S : 0;
 }
 
 // Walk directions for L2 reuse: a layer that reads the same owner as the layer before it walks every
@@ -265,6 +326,7 @@ int create_impl(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, i
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&c->l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess ||
             cudaMemsetAsync(device_pool, 0, need, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
             (void)cudaGetLastError();
             delete c;
@@ -444,40 +506,52 @@ int skv_decode_workspace_bytes(const skv_cache *c, int batch, int q_heads, size_
 {
     if (!c || !out_bytes || batch <= 0 || q_heads <= 0) return SKV_ERR_ARG;
     if (q_heads % c->kv_heads != 0 || q_heads / c->kv_heads > 8) return SKV_ERR_UNSUPPORTED;
-    const int sm = c->sm_count > 0 ? c->sm_count : 148;
-    const int W = sm * c->tune.ctas_per_sm * c->tune.warps;
-    *out_bytes = workspace_layout(c, batch, q_heads, W).total;
+    *out_bytes = workspace_layout(c, batch, q_heads, n_workers_max(c)).total;
     return SKV_OK;
 }
 
 namespace {
+// What a split-K launch tells the merge launch that follows it.
+struct SplitkPlan {
+    int n_workers = 0;       // ranges the block list was cut into
+    int unit_tokens = PAGE;  // tokens per unit of the list
+    int finished_single = 0; // segments inside one range were finished by the split-K launch itself
+};
+
 // Launches the split-K kernel on buffer `buf` (0 or 1) of the workspace.  `chained` = the call follows
 // another attention call of the same step whose inputs were all ready before that call was launched, so
-// it need not wait for it before reading.
+// it need not wait for it before reading.  `out` (may be null) = where the call's result rows go: given
+// it, the CTA-per-range kernel may run, which finishes the segments that lie inside one range.
 int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
                   int batch, int q_heads, int pt_stride, float scale, void *workspace, size_t workspace_bytes,
-                  void *stream, int buf = 0, bool chained = false)
+                  void *stream, SplitkPlan *plan, void *out = nullptr, int buf = 0, bool chained = false)
 {
     int rc = check_decode_args(c, layer, batch, q_heads);
     if (rc) return rc;
     if (!Q || !page_table || !seq_lens || !workspace || pt_stride <= 0) return SKV_ERR_ARG;
     if (!aligned(Q, 16) || !aligned(workspace, 256)) return SKV_ERR_ARG;
+    if (out && !aligned(out, 8)) return SKV_ERR_ARG;
     const int G = q_heads / c->kv_heads;
-    const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, n_workers_max(c));
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
     const bool tensor_core = c->fp8 || c->tune.variant == 2 || (c->tune.variant == 0 && G > 1);
-    // Default launch shapes (8 warps per SM, two 8 KB stages each, many small CTAs so that the CTAs of the
-    // next launch can move in one by one): 2 warps x 4 CTAs per SM for the tensor-core kernel, 1 warp x 8
-    // CTAs per SM for the CUDA-core kernel (measured best for each on B200).  Same worker count either way.
+    const bool umma = fp8_on_umma(c) && decode_fp8_umma_supported(c->head_dim, G);
+    // CTA per range: stand-alone calls whose result buffer is known (not the links of a chain, which overlap
+    // by having many small CTAs; not the tcgen05 FP8 kernel, which has its own CTA-wide design)
+    const int cta_S = cta_stages_for(c, batch, G);
+    const bool cta = !umma && !chained && out && c->worker_mode != 1 && cta_S > 0;
+    // Default launch shapes of the warp-per-range kernel (8 warps per SM, two 8 KB stages each, many small
+    // CTAs so that the CTAs of the next launch can move in one by one): 2 warps x 4 CTAs per SM for the
+    // tensor-core kernel, 1 warp x 8 CTAs per SM for the CUDA-core kernel (measured best for each on B200).
     int warps = c->tune.warps, ctas = c->tune.ctas_per_sm;
     if (c->shape_is_default && !tensor_core) {
         warps = 1;
         ctas = 8;
     }
-    const bool umma = fp8_on_umma(c) && decode_fp8_umma_supported(c->head_dim, G);
-    const size_t smem = umma ? decode_fp8_umma_smem_bytes(c->head_dim, batch)
-                             : decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages, c->fp8);
+    const int W = cta ? n_cta_workers_of(c) : n_workers_of(c);
+    const size_t smem = umma  ? decode_fp8_umma_smem_bytes(c->head_dim, batch)
+                        : cta ? decode_cta_smem_bytes(c->head_dim, batch, G, c->cta_consumers, cta_S, c->fp8)
+                              : decode_smem_bytes(c->head_dim, batch, warps, c->tune.stages, c->fp8);
     if (smem == 0 || smem > (size_t)c->max_smem_optin) return SKV_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
@@ -488,6 +562,7 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.Q = static_cast<const uint16_t *>(Q);
     p.page_table = page_table;
     p.seq_lens = seq_lens;
+    p.out = static_cast<uint16_t *>(out);
     p.part_o = reinterpret_cast<float *>(ws + wl.o_off);
     p.part_ml = reinterpret_cast<float *>(ws + wl.ml_off);
     p.prefix = reinterpret_cast<int32_t *>(ws + wl.prefix_off);
@@ -497,25 +572,35 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.pt_stride = pt_stride;
     const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)c->head_dim);
     p.scale_log2 = sc * 1.4426950408889634f;
-    p.flags = chained ? DECODE_LATE_WAIT : 0;
+    p.flags = chained ? DECODE_LATE_WAIT : (c->early_fetch && c->tune.pdl) ? DECODE_EARLY_FETCH : 0;
+    if (cta && c->cta_in_turn) p.flags |= DECODE_CLAIM_IN_TURN;
     p.keep_pct = 0;
+    // what one call streams fits in L2 beside everything else when it is under about a third of it
+    p.l2_fit_blocks = (int64_t)(c->l2_bytes / 3) / (int64_t)(c->fp8 ? fp8_block_bytes(c->head_dim) : block_bytes(c->head_dim));
     if (c->l2_keep_pct > 0) {
         if (c->walk_reverse[(size_t)layer]) p.flags |= DECODE_REVERSE;
         if (c->walk_keep[(size_t)layer]) p.keep_pct = c->l2_keep_pct;
     }
     p.status = c->status_word();
-    p.trace = (c->trace && c->trace_bytes >= (size_t)W * 32) ? c->trace : nullptr;
-    const int grid = c->sm_count * ctas;
+    const size_t trace_need = (size_t)W * (cta ? c->cta_consumers : 1) * 32;
+    p.trace = (c->trace && c->trace_bytes >= trace_need) ? c->trace : nullptr;
+    const int kernel = c->fp8 ? 2 : tensor_core ? 1 : 0;
     const cudaError_t le =
-        umma ? launch_decode_fp8_umma(p, c->head_dim, G, W, c->tune.pdl != 0, st)
-             : launch_decode_splitk(p, c->head_dim, G, c->fp8 ? 2 : tensor_core ? 1 : 0, grid, warps, c->tune.stages,
-                                    c->tune.pdl != 0, st);
+        umma  ? launch_decode_fp8_umma(p, c->head_dim, G, W, c->tune.pdl != 0, st)
+        : cta ? launch_decode_cta(p, c->head_dim, G, kernel, W, c->cta_consumers, cta_S, c->tune.pdl != 0, st)
+              : launch_decode_splitk(p, c->head_dim, G, kernel, c->sm_count * ctas, warps, c->tune.stages,
+                                     c->tune.pdl != 0, st);
     if (le != cudaSuccess) {
         (void)cudaGetLastError();
         // a launch shape with more warps per CTA than the register file holds for this kernel variant
         return le == cudaErrorLaunchOutOfResources ? SKV_ERR_UNSUPPORTED : SKV_ERR_CUDA;
     }
     c->launches += 1;
+    if (plan) {
+        plan->n_workers = W;
+        plan->unit_tokens = umma ? decode_fp8_umma_tile_tokens() : PAGE;
+        plan->finished_single = cta ? 1 : 0;
+    }
     return SKV_OK;
 }
 }  // namespace
@@ -525,31 +610,37 @@ int skv_decode_splitk(skv_cache *c, int layer, const void *Q, const int32_t *pag
                       size_t workspace_bytes, void *stream)
 {
     return launch_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
-                         workspace_bytes, stream);
+                         workspace_bytes, stream, nullptr);
 }
 
 namespace {
-// the merge kernel on buffer `buf` of the workspace
+// The merge kernel on buffer `buf` of the workspace.  `plan` = what the split-K launch before it did (null:
+// a warp-per-range or tcgen05 launch under the handle's current settings); seq_lens / pt_stride (may be null
+// / 0) let the kernel count the pages itself instead of reading the counts that launch left in the workspace.
 int launch_merge_on(skv_cache *c, void *out, int batch, int q_heads, void *workspace, size_t workspace_bytes,
-                    void *stream, int buf)
+                    void *stream, int buf, const SplitkPlan *plan = nullptr, const int32_t *seq_lens = nullptr,
+                    int pt_stride = 0)
 {
     int rc = check_decode_args(c, 0, batch, q_heads);
     if (rc) return rc;
     if (!out || !workspace || !aligned(out, 8) || !aligned(workspace, 256)) return SKV_ERR_ARG;
-    const int W = n_workers_of(c);
-    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, W);
+    const WorkspaceLayout wl = workspace_layout(c, batch, q_heads, n_workers_max(c));
     if (workspace_bytes < wl.total) return SKV_ERR_NOMEM;
     uint8_t *ws = static_cast<uint8_t *>(workspace) + (size_t)buf * wl.buf_bytes;
     MergeParams m;
     m.part_o = reinterpret_cast<const float *>(ws + wl.o_off);
     m.part_ml = reinterpret_cast<const float *>(ws + wl.ml_off);
     m.prefix = reinterpret_cast<const int32_t *>(ws + wl.prefix_off);
+    m.seq_lens = (seq_lens && pt_stride > 0 && batch <= 4096) ? seq_lens : nullptr;     // the counts go to shared memory
+    m.unit_tokens = plan ? plan->unit_tokens : fp8_on_umma(c) ? decode_fp8_umma_tile_tokens() : PAGE;
+    m.max_tokens = (int64_t)pt_stride * PAGE;
     m.out = static_cast<uint16_t *>(out);
     m.B = batch;
     m.Hq = q_heads;
     m.Hkv = c->kv_heads;
     m.D = c->head_dim;
-    m.n_workers = W;
+    m.n_workers = plan ? plan->n_workers : n_workers_of(c);
+    m.skip_single = plan ? plan->finished_single : 0;
     // with overlappable launches the merge grid must be resident in one wave (see merge_kernel)
     m.max_ctas = c->tune.pdl ? (c->sm_count > 0 ? c->sm_count : 1) : 0x7FFFFFFF;
     if (launch_merge(m, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
@@ -572,28 +663,12 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
                     size_t workspace_bytes, void *stream)
 {
     if (!out) return SKV_ERR_ARG;
+    SplitkPlan plan;
     int rc = launch_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
-                           workspace_bytes, stream);
+                           workspace_bytes, stream, &plan, out);
     if (rc) return rc;
-    return launch_merge_on(c, out, batch, q_heads, workspace, workspace_bytes, stream, 0);
+    return launch_merge_on(c, out, batch, q_heads, workspace, workspace_bytes, stream, 0, &plan, seq_lens, pt_stride);
 }
-
-}  // extern "C"
-
-// Used by skv_decode_attn_static (skv_static.cu): the same two launches as skv_decode_attn on a scratch
-// area the library owns.  Nothing in the area has to be cleared: the merge kernel only reads slots that
-// the split-K launch of the same call has just written.
-namespace skv {
-int decode_attn_on_scratch(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
-                           void *out, int batch, int q_heads, int pt_stride, float scale, void *scratch,
-                           size_t scratch_bytes, void *stream)
-{
-    return skv_decode_attn(c, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, scratch,
-                           scratch_bytes, stream);
-}
-}  // namespace skv
-
-extern "C" {
 
 }  // extern "C"
 
@@ -669,11 +744,14 @@ int step_layers(skv_cache *c, int l0, int l1, const uint8_t *q, const uint8_t *k
             if (rc) return rc;
         }
         const bool chained = c->tune.pdl && updates_done && l > l0;
+        SplitkPlan plan;
         rc = launch_splitk(c, l, q + (size_t)l * q_layer, page_table, seq_lens, batch, q_heads, pt_stride, scale,
-                           workspace, workspace_bytes, stream, l & 1, chained);
+                           workspace, workspace_bytes, stream, &plan, updates_done && c->tune.pdl ? nullptr : o + (size_t)l * q_layer,
+                           l & 1, chained);
         if (rc) return rc;
         // the merge kernel waits for that launch and lets the next split-K launch be scheduled at once
-        rc = launch_merge_on(c, o + (size_t)l * q_layer, batch, q_heads, workspace, workspace_bytes, stream, l & 1);
+        rc = launch_merge_on(c, o + (size_t)l * q_layer, batch, q_heads, workspace, workspace_bytes, stream, l & 1, &plan,
+                             seq_lens, pt_stride);
         if (rc) return rc;
     }
     return SKV_OK;
@@ -967,7 +1045,7 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     if (warps_per_cta) t.warps = warps_per_cta;
     if (stages) t.stages = stages;
     if (ctas_per_sm) t.ctas_per_sm = ctas_per_sm;
-    if (t.warps < 1 || t.warps > 16 || t.stages < 1 || t.stages > 8 || t.ctas_per_sm < 1 || t.ctas_per_sm > 16)
+    if (t.warps < 1 || t.warps > 16 || t.stages < 1 || t.stages > 8 || t.ctas_per_sm < 1 || t.ctas_per_sm > 8)
         return SKV_ERR_ARG;
     if (c->pool) {
         const size_t smem = decode_smem_bytes(c->head_dim, 1, t.warps, t.stages, c->fp8);
@@ -992,6 +1070,24 @@ int skv_set_decode_overlap(skv_cache *c, int enabled)
     return SKV_OK;
 }
 
+int skv_set_decode_early_fetch(skv_cache *c, int enabled)
+{
+    if (!c || enabled < 0 || enabled > 1) return SKV_ERR_ARG;
+    c->early_fetch = enabled != 0;
+    return SKV_OK;
+}
+
+int skv_set_decode_worker(skv_cache *c, int mode, int consumers, int stages)
+{
+    if (!c || mode < 0 || mode > 3 || consumers < 0 || consumers > 12 || stages < 0 || stages == 1 || stages > 26)
+        return SKV_ERR_ARG;
+    c->cta_in_turn = mode != 3;
+    c->worker_mode = mode == 3 ? 2 : mode;
+    if (consumers) c->cta_consumers = consumers;
+    c->cta_stages = stages;
+    return SKV_OK;
+}
+
 int skv_set_decode_l2_reuse(skv_cache *c, int keep_percent)
 {
     if (!c || keep_percent < 0 || keep_percent > 100) return SKV_ERR_ARG;
@@ -1010,7 +1106,8 @@ int skv_set_trace_buffer(skv_cache *c, void *device_buffer, size_t bytes)
 int skv_decode_worker_count(const skv_cache *c)
 {
     if (!c || !c->pool) return SKV_ERR_ARG;
-    return n_workers_of(c);
+    const int warp_ranges = n_workers_of(c), cta_warps = n_cta_workers_of(c) * c->cta_consumers;
+    return warp_ranges > cta_warps ? warp_ranges : cta_warps;
 }
 
 int skv_launch_count(const skv_cache *c, int64_t *out_count)

@@ -37,6 +37,7 @@ __device__ __forceinline__ CopyCoord coord_of(int64_t n_tok, int Hkv, int CH)
 
 __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
 {
+    pdl_trigger();      // an attention launch right after this one may set itself up while the rows are copied
     const int CH = p.D / CHUNK_ELEMS;
     const CopyCoord k = coord_of(p.n_tokens, p.Hkv, CH);
     if (!k.in_range) return;
@@ -190,6 +191,7 @@ __device__ __forceinline__ void append_fp8_token(const AppendFp8Params &p, int64
 // 15 rows have nothing to do.
 __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
 {
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     // (rows counted head-major and an odd number of warps in the grid: a warp then meets every position inside
     // a page in turn, instead of always the pages' first rows or never one)
@@ -223,6 +225,7 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Param
 // its tokens that belong to no whole page one row at a time.  Same result as the kernel above for any slot map.
 __global__ void __launch_bounds__(COPY_THREADS) append_fp8_groups_kernel(AppendFp8Params p)
 {
+    pdl_trigger();
     constexpr unsigned ALL = 0xFFFFFFFFu;
     const int lane = threadIdx.x & 31;
     const int64_t n_groups = (p.n_tokens + PAGE - 1) / PAGE, n_items = n_groups * p.Hkv;

@@ -97,6 +97,13 @@ constexpr int DECODE_REVERSE = 1;     // every worker walks its block range from
 constexpr int DECODE_LATE_WAIT = 2;   // inputs are known to be ready: the wait on the previous kernel in the
                                       // stream is taken half-way through the range instead of before the first read
 
+constexpr int DECODE_EARLY_FETCH = 4;  // the lengths, the page table and all cached tokens except each sequence's
+                                      // newest one were complete before the kernel before this one started: the
+                                      // ring is filled before the wait on that kernel, the queries are read after it
+
+constexpr int DECODE_CLAIM_IN_TURN = 8; // CTA-per-range kernel: block j of a range goes to consumer j mod C instead
+                                      // of to whichever consumer is free first
+
 struct DecodeParams {
     const uint8_t *layer_base;  // first page of the owner layer that is read
     int64_t page_stride;
@@ -104,6 +111,7 @@ struct DecodeParams {
     const uint16_t *Q;          // [B][Hq][D] bf16 bits
     const int32_t *page_table;  // [B][pt_stride]
     const int32_t *seq_lens;    // [B]
+    uint16_t *out;              // [B][Hq][D] bf16 bits (CTA-per-range kernel only: segments inside one range are finished there)
     float *part_o;              // [n_slots][G][D]
     float *part_ml;             // [n_slots][G][2]  (running max in log2 units, sum)
     int32_t *prefix;            // [B+1] cumulative page counts (written by CTA 0 for the merge kernel)
@@ -112,6 +120,8 @@ struct DecodeParams {
     int flags;
     int keep_pct;               // share of each worker's range, at the END of its walk, that is loaded with
                                 // normal L2 priority; the rest is loaded evict-first
+    int64_t l2_fit_blocks;      // a call with at most this many blocks in all is small enough to stay in L2 for
+                                // the next layer that reads the same owner: all of it is loaded with normal priority
     int *status;
     unsigned long long *trace;  // optional [n_workers][4]: sm id, entry ns, first-page ns, exit ns
 };
@@ -119,11 +129,16 @@ struct DecodeParams {
 struct MergeParams {
     const float *part_o;
     const float *part_ml;
-    const int32_t *prefix;      // [B+1]
+    const int32_t *prefix;      // [B+1] page (or tile) counts as the split-K launch left them
+    const int32_t *seq_lens;    // [B], or null.  Not null: the kernel counts the pages itself, before it waits
+                                // for the split-K launch (the lengths are an input of the call, older than that launch)
+    int unit_tokens;            // tokens per unit of the flattened list (a page, or a tile of several pages)
+    int64_t max_tokens;         // pt_stride * PAGE: longer sequences were cut to this by the split-K launch
     uint16_t *out;              // [B][Hq][D] bf16 bits
     int B, Hq, Hkv, D;
     int n_workers;
     int max_ctas;               // grid limit (one CTA per SM)
+    int skip_single;            // 1: segments with a single partial were finished by the split-K launch itself
 };
 
 struct PrefillParams {
@@ -154,6 +169,7 @@ cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
 // decode attention over FP8 pages on tcgen05 (skv_decode_fp8_umma.cu): a worker is a CTA, grid = worker count
 bool decode_fp8_umma_supported(int D, int G);
 int decode_fp8_umma_ctas_per_sm();
+int decode_fp8_umma_tile_tokens();           // tokens per unit of its flattened list
 size_t decode_fp8_umma_smem_bytes(int D, int B);
 cudaError_t launch_decode_fp8_umma(const DecodeParams &p, int D, int G, int grid, bool pdl, cudaStream_t s);
 cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s);
@@ -164,6 +180,10 @@ size_t decode_smem_bytes(int D, int B, int warps, int stages, bool fp8);
 cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, int kernel, int grid,
                                  int warps, int stages, bool pdl, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
+// the CTA-per-range split-K kernel (skv_decode_cta.cu): grid = worker count, consumers + 1 warps per CTA
+size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, bool fp8);
+cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,
+                              bool pdl, cudaStream_t s);
 size_t prefill_smem_bytes(int D);
 size_t prefill_fp8_smem_bytes(int D);
 cudaError_t launch_prefill_fp8(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
@@ -174,6 +194,16 @@ size_t prefill_umma_smem_bytes(int D);
 bool prefill_umma_supported(int D, int G);
 int prefill_umma_tile_tokens(int G);
 cudaError_t launch_prefill_umma(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
+
+// Raise a kernel's dynamic shared-memory limit to `smem` bytes (skv_api.cu).  The limit only ever has to
+// grow, and asking the runtime on every launch costs more than the launch itself, so what has been granted
+// is remembered per kernel and device.
+cudaError_t ensure_dynamic_smem_fn(const void *kernel, size_t smem);
+template <class Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kern, size_t smem)
+{
+    return ensure_dynamic_smem_fn(reinterpret_cast<const void *>(kern), smem);
+}
 
 // ---- worker <-> work-range arithmetic (shared by split-K and merge) --------
 // The flattened work space orders (sequence b, kv head h, page pg) b-major:

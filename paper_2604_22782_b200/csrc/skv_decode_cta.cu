@@ -1,0 +1,387 @@
+// "Load + Attn" of Algorithm 2 for one new token per sequence (Eq. (3.1)), the form used for stand-alone
+// attention calls: the worker of the split-K pass is a whole CTA (one per SM) instead of a warp.
+//
+// The flattened (sequence, kv head, page) block list of the call is cut into one contiguous range per CTA.
+// One producer warp streams the CTA's blocks, in order, through ONE shared ring of 8 KB stages (a linear
+// bulk copy per block, completion on the stage's mbarrier); the consumer warps claim the blocks of the ring
+// one by one, in order (a shared counter: whoever is free takes the next block), each keeping a running
+// (max, sum, out) of its own for the (sequence, kv head) segment the blocks belong to.  At the end of every run of the range inside one
+// segment the consumers put their states side by side in shared memory and combine them:
+//   - a segment that lies wholly inside the CTA's range is finished on the spot: normalised, rounded to
+//     bf16 and written to `out`;
+//   - a segment that continues in a neighbouring CTA leaves one fp32 partial at slot  cta + segment  for the
+//     merge kernel, which only has those segments left to do.
+// Compared with a warp per range this evens out the consumers of an SM block by block (a warp with two
+// copies of its own in flight advances at the pace of its own latencies, and the slowest of 1184 sets the
+// end of the launch), leaves a fifth of the partials, and keeps more bytes in flight per SM.
+#include "skv_common.cuh"
+#include "skv_decode_states.cuh"
+#include "skv_walk.cuh"
+
+namespace skv {
+
+namespace {
+
+constexpr int MAX_CONSUMERS = 12;
+
+// floats of one consumer's state in the scratch: out [G][D], then (max, sum) [G][2], rounded up to 16 bytes
+// (the states are written with 16-byte stores)
+__host__ __device__ constexpr int cta_part_floats(int G, int D) { return G * D + ((2 * G + 3) & ~3); }
+
+// try_wait loop with a time limit that also gives up as soon as another warp of the CTA has
+__device__ __forceinline__ bool wait_or_quit(uint32_t bar, uint32_t parity, volatile int *gave_up)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*gave_up) return false;
+        if (global_timer_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+// try_wait until an absolute time (for the exit path, where one limit covers every copy still in flight)
+__device__ __forceinline__ bool wait_until(uint32_t bar, uint32_t parity, uint64_t deadline_ns)
+{
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() > deadline_ns) return false;
+    }
+}
+
+// Block index a stage's barrier has last been armed for: written by the producer right after arming (and
+// before the copy goes out), read by the consumer that claimed the block before it waits on the barrier.  A
+// parity wait only means "the copy of block k has landed" to a waiter who knows that the barrier is in
+// block k's phase; a consumer that visits the stages in no fixed order does not know, so it is told.
+// Plain volatile accesses: shared-memory operations of one thread reach the SM's memory in program order,
+// and a fence here would make the producer wait for its copies.
+__device__ __forceinline__ void publish_issued(uint32_t addr, int k)
+{
+    asm volatile("st.volatile.shared::cta.s32 [%0], %1;" ::"r"(addr), "r"(k) : "memory");
+}
+
+__device__ __forceinline__ bool wait_issued(uint32_t addr, int k, volatile int *gave_up, int lane)
+{
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i) {
+            int v = 0;
+            if (lane == 0) asm volatile("ld.volatile.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+            if (__shfl_sync(0xFFFFFFFFu, v, 0) == k) return true;
+            __nanosleep(32);
+        }
+        if (*gave_up) return false;
+        if (global_timer_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared memory: tables (prefix, lens) | ring [S][BLOCK] | scratch [2][C] x ([G][D] fp32 out + [G][2] (max, sum))
+//                | full[S], empty[S], run_done[2] mbarriers | gave_up word, claim counter | issued[S]
+// The scratch is double-buffered by run parity: a consumer writes buffer r&1 at the end of run r, and it can
+// only get to the end of run r+2 after every consumer has arrived at the barrier of run r+1, i.e. after
+// every consumer has finished reading buffer r&1.
+template <int D, class State>
+__global__ void decode_cta_kernel(DecodeParams p, int G, int S)
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    constexpr int BLOCK = State::BLOCK;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int C = (int)(blockDim.x >> 5) - 1;          // consumer warps; warp C is the producer
+    const uint64_t t_entry = p.trace ? global_timer_ns() : 0;
+
+    const uint32_t base = smem_u32(smem_raw);
+    const uint32_t pad = (128u - (base & 127u)) & 127u;
+    int32_t *prefix = reinterpret_cast<int32_t *>(smem_raw + pad);
+    int32_t *lens = prefix + p.B + 1;
+    const size_t ring_off = pad + table_bytes(p.B);
+    const uint32_t ring = base + (uint32_t)ring_off;
+    const size_t scratch_off = ring_off + (size_t)S * BLOCK;
+    const int part_floats = cta_part_floats(G, D);     // one consumer's state: out [G][D], then (max, sum) [G][2]
+    float *scratch = reinterpret_cast<float *>(smem_raw + scratch_off);
+    const size_t bars_off = scratch_off + (((size_t)2 * C * part_floats * 4 + 15) & ~(size_t)15);
+    const uint32_t full = base + (uint32_t)bars_off, empty = full + 8u * S, run_done = empty + 8u * S;
+    volatile int *gave_up = reinterpret_cast<volatile int *>(smem_raw + bars_off + 16 * (size_t)S + 16);
+    int *next_claim = const_cast<int *>(gave_up) + 1;
+    const uint32_t issued_at = run_done + 16 + 8;       // int [S]
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full + 8 * s, 1);
+            mbar_init(empty + 8 * s, 1);
+        }
+        mbar_init(run_done, C);
+        mbar_init(run_done + 8, C);
+        gave_up[0] = 0;
+        *next_claim = 0;
+        for (int s = 0; s < S; ++s) publish_issued(issued_at + 4 * s, -1);
+        fence_barrier_init();
+    }
+    const bool early_fetch = (p.flags & DECODE_EARLY_FETCH) != 0;
+    const bool reverse = (p.flags & DECODE_REVERSE) != 0;
+    if (!early_fetch) pdl_wait();                      // anything read below may come from the kernel before this one
+    if (warp == 0) scan_lengths(p.seq_lens, p.B, PAGE, (int64_t)p.pt_stride * PAGE, p.status, prefix, lens, lane);
+    __syncthreads();
+
+    const int64_t W = gridDim.x, w = blockIdx.x;
+    const int64_t T = (int64_t)prefix[p.B] * p.Hkv;
+    int64_t x0 = 0;
+    int n = 0;
+    if (T > 0) {
+        x0 = worker_begin(w, T, W);
+        n = (int)(worker_begin(w + 1, T, W) - x0);
+    }
+    const int64_t x_first = reverse ? x0 + n - 1 : x0;
+
+    if (warp == C) {
+        // ================= producer =================
+        // The range is walked in groups of 32 blocks, lane L of the warp owning block 32g + L: it finds the
+        // block's place in the list and reads its page id one group AHEAD of the copies (the id is a trip to
+        // L2 that must not sit between two batches of copies), then issues the block's copy itself.  Within
+        // a group the copies go out PB lanes at a time, in order (one thread alone cannot issue bulk copies
+        // fast enough for an SM's share of the bandwidth; and never two blocks of one batch in one stage).
+        const int PB = S < 8 ? S : 8;
+        const uint64_t pol_stream = make_policy_evict_first(), pol_keep = make_policy_evict_normal();
+        const int keep_from = (p.keep_pct > 0 && T <= p.l2_fit_blocks) ? 0 : n - (int)(((int64_t)n * p.keep_pct) / 100);
+        bool waited = !early_fetch, triggered = false, quit = false;
+        // This lane's block of a group: kv head, raw page id (checked and turned into an address only when the
+        // group's copies go out, so that the load stays in flight meanwhile; -1 past the end of the range),
+        // and whether the block is the last page of its sequence.
+        auto look_up = [&](int kk, int &id, int &h, bool &last_page) {
+            id = -1;
+            h = 0;
+            last_page = false;
+            if (kk >= n) return;
+            const Cursor cur = locate(prefix, p.B, p.Hkv, reverse ? x_first - kk : x_first + kk);
+            id = __ldg(p.page_table + (int64_t)cur.b * p.pt_stride + cur.pg);
+            h = cur.h;
+            last_page = cur.pg + 1 == cur.pages;
+        };
+        int id = -1, h = 0, id_next = -1, h_next = 0;
+        bool last_page = false, last_next = false;
+        look_up(lane, id, h, last_page);
+        int k = 0;                                      // first block of the current group
+        for (; k < n && !quit; k += 32) {
+            const int kk = k + lane;
+            if (kk < n && (id < 0 || (int64_t)id >= p.max_pages)) {
+                atomicOr(p.status, STATUS_BOUNDS);
+                id = 0;
+            }
+            const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK;
+            look_up(k + 32 + lane, id_next, h_next, last_next);
+            for (int j0 = 0; j0 < 32 && k + j0 < n && !quit; j0 += PB) {
+                const bool active = lane >= j0 && lane < j0 + PB && kk < n;
+                // With early fetch the ring is filled before the wait on the kernel before this one, but
+                // never with a sequence's last page (its newest token may be on its way), and the wait is
+                // taken at the latest when the ring has been filled once.
+                if (!waited && (k + j0 + PB > S || __any_sync(FULL, active && last_page))) {
+                    pdl_wait();
+                    waited = true;
+                }
+                if (!triggered && k + j0 >= n / 2) {   // the merge kernel may move in from here on
+                    triggered = true;
+                    if (!waited) { pdl_wait(); waited = true; }
+                    pdl_trigger();
+                }
+                bool ok = true;
+                if (active) {
+                    const int s = kk % S;
+                    if (kk >= S) ok = wait_or_quit(empty + 8 * s, (uint32_t)((kk / S - 1) & 1), gave_up);
+                    if (ok) {
+                        mbar_expect_tx(full + 8 * s, BLOCK);
+                        publish_issued(issued_at + 4 * s, kk);
+                        bulk_copy_g2s_hint(ring + (uint32_t)(s * BLOCK), src, BLOCK, full + 8 * s, kk >= keep_from ? pol_keep : pol_stream);
+                    }
+                }
+                if (!__all_sync(FULL, ok)) {
+                    if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+                    quit = true;
+                }
+            }
+            id = id_next;
+            h = h_next;
+            last_page = last_next;
+        }
+        if (!waited) pdl_wait();
+        if (!triggered) pdl_trigger();
+        // Leave only when every copy that was issued has landed: the ring must not be written after the CTA
+        // is gone.  (Normally the consumers have seen them all long ago; after a failure they may not have.)
+        // (after a failure some lanes of the last batch may not have issued: those stages' phases were
+        // completed by earlier copies or never armed, and the waits below return at once or at the limit)
+        const int issued = k < n ? k : n;
+        const uint64_t deadline = global_timer_ns() + 2000000000ull;
+        for (int j = issued > S ? issued - S : 0; j < issued; ++j)
+            if (!wait_until(full + 8 * (j % S), (uint32_t)((j / S) & 1), deadline)) break;
+        return;
+    }
+
+    // ================= consumers =================
+    // The page counts go to global memory for the merge kernel (after the wait on the kernel before this
+    // one: the merge of an earlier call may still be reading this buffer).
+    if (early_fetch) pdl_wait();
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i <= p.B; i += C * 32) p.prefix[i] = prefix[i];
+
+    Cursor cons = {0, 0, 0, 1};
+    if (n > 0) cons = locate(prefix, p.B, p.Hkv, x_first);
+    uint64_t t_first = 0;
+    int k = 0, run = 0;
+    int held = -1;                                     // a block of the range this consumer has claimed and not done yet
+    // Dynamic: whoever is free takes the next block (the consumers of an SM end together, but which blocks a
+    // consumer sums, and with that the last bits of the result, vary from run to run).  In turn: block j
+    // goes to consumer j mod C (reproducible bit for bit).
+    const bool in_turn = (p.flags & DECODE_CLAIM_IN_TURN) != 0;
+    // With blocks taken in turn and the ring a whole number of rounds deep, a stage always serves the same
+    // consumer, who then sees every phase of its barrier in order and needs no telling.
+    const bool ask_issued = !in_turn || S % C != 0;
+    int my_next = warp;
+    auto claim = [&]() -> int {
+        if (in_turn) {
+            const int j = my_next;
+            my_next += C;
+            return j;
+        }
+        int j = 0;
+        if (lane == 0) j = atomicAdd(next_claim, 1);
+        return __shfl_sync(FULL, j, 0);
+    };
+    bool failed = false;
+    while (k < n && !failed) {
+        // one run: blocks [k, k + len) of the range, all of segment (b, h)
+        const int b = cons.b, h = cons.h, pages = cons.pages, n_b = lens[b];
+        const int to_edge = reverse ? cons.pg + 1 : pages - cons.pg;           // blocks left in this segment
+        const int len = to_edge < n - k ? to_edge : n - k;
+        const bool whole = len == pages;                                       // the segment lies inside this range
+        float *mine = scratch + ((size_t)(run & 1) * C + warp) * part_floats;
+        if (held < 0) held = claim();
+        if (held < k + len) {
+            State st;
+            st.begin(p, b, h, G, lane);
+            do {
+                const int j = held, s = j % S;
+                if ((ask_issued && !wait_issued(issued_at + 4 * s, j, gave_up, lane)) ||
+                    !wait_or_quit(full + 8 * s, (uint32_t)((j / S) & 1), gave_up)) {
+                    if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+                    failed = true;
+                    break;
+                }
+                if (p.trace && t_first == 0) t_first = global_timer_ns();
+                const int pg = reverse ? cons.pg - (j - k) : cons.pg + (j - k);
+                const int left = n_b - pg * PAGE;
+                st.page(ring + (uint32_t)(s * BLOCK), left < PAGE ? left : PAGE, p.scale_log2, lane);
+                __syncwarp();                           // every lane is done reading this stage
+                if (lane == 0) mbar_arrive(empty + 8 * s);
+                held = claim();
+            } while (held < k + len);
+            if (!failed) st.finish(mine, mine + G * D, 0, G, lane);
+        } else if (lane < G) {
+            mine[G * D + 2 * lane] = -INFINITY;         // no block of this run: nothing to contribute
+        }
+        // all consumers' states of this run are in shared memory
+        __syncwarp();
+        if (lane == 0) mbar_arrive(run_done + 8 * (run & 1));
+        if (failed || !wait_or_quit(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1), gave_up)) {
+            if (lane == 0 && !failed) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+            failed = true;
+            break;
+        }
+        // combine: thread t takes output pairs e2 = t, t + 32C, ... of the G*D/2 pairs
+        {
+            const int slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
+            for (int e2 = (int)threadIdx.x; e2 < G * D / 2; e2 += C * 32) {
+                const int g = (2 * e2) / D;
+                float M = -INFINITY;
+                const float *buf = scratch + (size_t)(run & 1) * C * part_floats;
+                for (int c = 0; c < C; ++c) M = fmaxf(M, buf[c * part_floats + G * D + 2 * g]);
+                float L = 0.f, a0 = 0.f, a1 = 0.f;
+                for (int c = 0; c < C; ++c) {
+                    const float *sc = buf + c * part_floats;
+                    const float m_c = sc[G * D + 2 * g];
+                    if (m_c == -INFINITY) continue;     // this consumer had no block in the run
+                    const float wt = fast_exp2(m_c - M);
+                    L = fmaf(wt, sc[G * D + 2 * g + 1], L);
+                    const float2 v = *reinterpret_cast<const float2 *>(sc + 2 * e2);
+                    a0 = fmaf(wt, v.x, a0);
+                    a1 = fmaf(wt, v.y, a1);
+                }
+                if (whole) {
+                    const float inv = L > 0.f ? 1.f / L : 0.f;
+                    uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)h * G) * D);
+                    dst[e2] = pack_bf16x2(a0 * inv, a1 * inv);
+                } else {
+                    *reinterpret_cast<float2 *>(p.part_o + (int64_t)slot * G * D + 2 * e2) = make_float2(a0, a1);
+                    if ((2 * e2) % D == 0) *reinterpret_cast<float2 *>(p.part_ml + ((int64_t)slot * G + g) * 2) = make_float2(M, L);
+                }
+            }
+        }
+        k += len;
+        ++run;
+        if (k < n) {                                   // first block of the next run
+            cons.pg = reverse ? cons.pg - (len - 1) : cons.pg + (len - 1);
+            step(cons, prefix, p.Hkv, reverse);
+        }
+    }
+    if (p.trace && lane == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        unsigned long long *t = p.trace + 4 * (w * C + warp);
+        t[0] = smid; t[1] = t_entry; t[2] = t_first; t[3] = global_timer_ns();
+    }
+}
+
+template <int D, class State>
+cudaError_t launch_cta_t(const DecodeParams &p, int G, int grid, int consumers, int stages, bool pdl, cudaStream_t s)
+{
+    const size_t smem = decode_cta_smem_bytes(D, p.B, G, consumers, stages, State::BLOCK != block_bytes(D));
+    auto kern = decode_cta_kernel<D, State>;
+    cudaError_t e = ensure_dynamic_smem(kern, smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)((consumers + 1) * 32));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, p, G, stages);
+}
+
+}  // namespace
+
+size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, bool fp8)
+{
+    if (D != 64 && D != 128) return 0;
+    if (consumers < 1 || consumers > MAX_CONSUMERS || stages < 2) return 0;
+    const size_t blk = fp8 ? fp8_block_bytes(D) : block_bytes(D);
+    const size_t scratch = (((size_t)2 * consumers * cta_part_floats(G, D) * 4) + 15) & ~(size_t)15;
+    // 128 bytes of slack for aligning the ring base; barriers: full, empty per stage, two run barriers; two words
+    // ... and the issued-block word of every stage
+    return 128 + table_bytes(B) + (size_t)stages * blk + scratch + 16 * (size_t)stages + 16 + 16 + 4 * (size_t)stages + 16;
+}
+
+cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,
+                              bool pdl, cudaStream_t s)
+{
+    if (D == 128) {
+        if (kernel == 2) return launch_cta_t<128, Fp8State<128>>(p, G, grid, consumers, stages, pdl, s);
+        if (kernel == 1) return launch_cta_t<128, TensorCoreState<128>>(p, G, grid, consumers, stages, pdl, s);
+        return launch_cta_t<128, CudaCoreState<128>>(p, G, grid, consumers, stages, pdl, s);
+    }
+    if (D == 64) {
+        if (kernel == 2) return launch_cta_t<64, Fp8State<64>>(p, G, grid, consumers, stages, pdl, s);
+        if (kernel == 1) return launch_cta_t<64, TensorCoreState<64>>(p, G, grid, consumers, stages, pdl, s);
+        return launch_cta_t<64, CudaCoreState<64>>(p, G, grid, consumers, stages, pdl, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace skv

@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     // flattened list that is cut into equal ranges is the list of (sequence, kv head, tile) here, a tile
     // being pages [8i, 8i+8) of the sequence: equal ranges are then equal numbers of tiles, which is what a
     // CTA's time goes with.  The merge kernel is told the same counts, so it finds the partials as usual.
-    if (warp == 0) scan_lengths(p.seq_lens, p.B, TP * PAGE, prefix, lens, lane);
+    if (warp == 0) scan_lengths(p.seq_lens, p.B, TP * PAGE, (int64_t)p.pt_stride * PAGE, p.status, prefix, lens, lane);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
     if (warp == 5) {
         // ================= producer =================
         const uint64_t pol_stream = make_policy_evict_first(), pol_keep = make_policy_evict_normal();
-        const int keep_from = n - (int)(((int64_t)n * p.keep_pct) / 100);
+        const int keep_from = (p.keep_pct > 0 && T * TP <= p.l2_fit_blocks) ? 0 : n - (int)(((int64_t)n * p.keep_pct) / 100);
         // Where the launch after this one may be scheduled (and, in a chain of calls, where this one waits for
         // the launch before it): at 7/8 of the range, not at the middle as the warp-per-worker kernel does --
         // the CTAs of this kernel are one wave, and CTAs of the next launch that got in early would only sit
@@ -630,6 +630,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM + 1) decode_fp8_umma_kern
 bool decode_fp8_umma_supported(int D, int G) { return D == 128 && G >= 1 && G <= 8; }
 
 int decode_fp8_umma_ctas_per_sm() { return CTAS_PER_SM; }
+int decode_fp8_umma_tile_tokens() { return TP * PAGE; }
 
 size_t decode_fp8_umma_smem_bytes(int D, int B)
 {
@@ -645,7 +646,7 @@ cudaError_t launch_decode_fp8_umma(const DecodeParams &p, int D, int G, int grid
     const size_t smem = decode_fp8_umma_smem_bytes(D, p.B);
     auto kern = G <= 1 ? decode_fp8_umma_kernel<128, 1> : G <= 2 ? decode_fp8_umma_kernel<128, 2>
               : G <= 4 ? decode_fp8_umma_kernel<128, 4> : decode_fp8_umma_kernel<128, 8>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(kern, smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

@@ -40,12 +40,13 @@ __global__ void __launch_bounds__(128, 2) prefill_kernel(PrefillParams p, int G)
     pdl_wait();                                    // inputs may come from the kernel before this one
     const int q_begin = __ldg(p.cu_q + b), q_len = __ldg(p.cu_q + b + 1) - q_begin;
     const int n_b = __ldg(p.seq_lens + b);
+    const bool too_long = (int64_t)n_b > (int64_t)p.pt_stride * PAGE;     // more pages than a page-table row holds
     const int n_tiles = (q_len + TQ - 1) / TQ;
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;      // tiles with the most keys are scheduled first
-    if (blockIdx.x == 0 && threadIdx.x == 0 && (q_len < 0 || q_len > n_b || n_tiles > (int)gridDim.x))
+    if (blockIdx.x == 0 && threadIdx.x == 0 && (q_len < 0 || q_len > n_b || too_long || n_tiles > (int)gridDim.x))
         atomicOr(p.status, STATUS_BOUNDS);         // more queries than cached tokens, or than the caller's bound
     __syncthreads();
-    if (q_len <= 0 || q_len > n_b || qt >= n_tiles) return;
+    if (q_len <= 0 || q_len > n_b || too_long || qt >= n_tiles) return;
     const int q0 = qt * TQ;
     const int q_end = (q0 + TQ < q_len) ? q0 + TQ : q_len;    // tokens [q0, q_end) of the sequence's new ones
     const int pos0 = n_b - q_len;                             // position of the sequence's first new token
@@ -265,12 +266,13 @@ __global__ void __launch_bounds__(128, 2) prefill_fp8_kernel(PrefillParams p, in
     pdl_wait();
     const int q_begin = __ldg(p.cu_q + b), q_len = __ldg(p.cu_q + b + 1) - q_begin;
     const int n_b = __ldg(p.seq_lens + b);
+    const bool too_long = (int64_t)n_b > (int64_t)p.pt_stride * PAGE;     // more pages than a page-table row holds
     const int n_tiles = (q_len + TQ - 1) / TQ;
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
-    if (blockIdx.x == 0 && threadIdx.x == 0 && (q_len < 0 || q_len > n_b || n_tiles > (int)gridDim.x))
+    if (blockIdx.x == 0 && threadIdx.x == 0 && (q_len < 0 || q_len > n_b || too_long || n_tiles > (int)gridDim.x))
         atomicOr(p.status, STATUS_BOUNDS);
     __syncthreads();
-    if (q_len <= 0 || q_len > n_b || qt >= n_tiles) return;
+    if (q_len <= 0 || q_len > n_b || too_long || qt >= n_tiles) return;
     const int q0 = qt * TQ;
     const int q_end = (q0 + TQ < q_len) ? q0 + TQ : q_len;
     const int pos0 = n_b - q_len;
@@ -534,7 +536,7 @@ cudaError_t launch_prefill_fp8(const PrefillParams &p, int D, int G, int q_tiles
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     auto kern = D == 128 ? prefill_fp8_kernel<128> : prefill_fp8_kernel<64>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(kern, smem);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, kern, p, G);
 }
@@ -554,11 +556,11 @@ cudaError_t launch_prefill(const PrefillParams &p, int D, int G, int q_tiles, bo
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     if (D == 128) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = ensure_dynamic_smem(prefill_kernel<128>, smem);
         if (e != cudaSuccess) return e;
         return cudaLaunchKernelEx(&cfg, prefill_kernel<128>, p, G);
     }
-    cudaError_t e = cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(prefill_kernel<64>, smem);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, prefill_kernel<64>, p, G);
 }

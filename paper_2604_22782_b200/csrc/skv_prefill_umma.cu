@@ -96,11 +96,12 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     pdl_wait();
     const int q_begin = __ldg(p.cu_q + b), q_len = __ldg(p.cu_q + b + 1) - q_begin;
     const int n_b = __ldg(p.seq_lens + b);
+    const bool too_long = (int64_t)n_b > (int64_t)p.pt_stride * PAGE;     // more pages than a page-table row holds
     const int n_tiles = (q_len + TQ - 1) / TQ;
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
-    if (blockIdx.x == 0 && tid == 0 && (q_len < 0 || q_len > n_b || n_tiles > (int)gridDim.x))
+    if (blockIdx.x == 0 && tid == 0 && (q_len < 0 || q_len > n_b || too_long || n_tiles > (int)gridDim.x))
         atomicOr(p.status, STATUS_BOUNDS);
-    if (q_len <= 0 || q_len > n_b || qt >= n_tiles) return;    // uniform over the CTA, before any allocation
+    if (q_len <= 0 || q_len > n_b || too_long || qt >= n_tiles) return;    // uniform over the CTA, before any allocation
     const int q0 = qt * TQ;
     const int q_end = (q0 + TQ < q_len) ? q0 + TQ : q_len;
     const int pos0 = n_b - q_len;
@@ -444,7 +445,7 @@ cudaError_t launch_prefill_umma(const PrefillParams &p, int D, int G, int q_tile
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    cudaError_t e = cudaFuncSetAttribute(prefill_umma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(prefill_umma_kernel<128>, smem);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, prefill_umma_kernel<128>, p, G);
 }

@@ -9,12 +9,6 @@
 // a device address: it must never be passed to a kernel directly.
 static __device__ __align__(256) unsigned char g_static_scratch[SKV_STATIC_SCRATCH_BYTES];
 
-namespace skv {
-int decode_attn_on_scratch(skv_cache *c, int layer, const void *Q, const int32_t *page_table, const int32_t *seq_lens,
-                           void *out, int batch, int q_heads, int pt_stride, float scale, void *scratch,
-                           size_t scratch_bytes, void *stream);
-}
-
 namespace {
 
 constexpr int MAX_DEVICES = 64;
@@ -55,6 +49,11 @@ extern "C" int skv_decode_attn_static(skv_cache *cache, int layer, const void *Q
     if (need > SKV_STATIC_SCRATCH_BYTES) return SKV_ERR_TOO_LARGE;
     void *scratch = scratch_address();
     if (!scratch) return SKV_ERR_CUDA;
-    return skv::decode_attn_on_scratch(cache, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale,
-                                       scratch, SKV_STATIC_SCRATCH_BYTES, stream);
+    // The same two launches as skv_decode_attn, on the library's own area.  Nothing in the area has to be
+    // cleared: the merge kernel only reads slots that the split-K launch of the same call has just
+    // written.  Calls on one stream may follow each other without anything in between because a split-K
+    // launch writes its first partial only after its wait on the kernel before it, i.e. after the merge
+    // of the previous call has read the area.
+    return skv_decode_attn(cache, layer, Q, page_table, seq_lens, out, batch, q_heads, pt_stride, scale, scratch,
+                           SKV_STATIC_SCRATCH_BYTES, stream);
 }

@@ -53,9 +53,11 @@ __device__ __forceinline__ void step(Cursor &c, const int32_t *prefix, int Hkv, 
 
 // By one warp: lens[i] = max(seq_lens[i], 0) and prefix[i] = number of units (pages, or tiles of several
 // pages: `unit_tokens` tokens each, the last one of a sequence possibly short) of the sequences before i,
-// per kv head; prefix[B] = all of them.
-__device__ __forceinline__ void scan_lengths(const int32_t *seq_lens, int B, int unit_tokens, int32_t *prefix, int32_t *lens,
-                                             int lane)
+// per kv head; prefix[B] = all of them.  A length that needs more pages than a page-table row holds
+// (max_tokens = pt_stride * PAGE) is cut to what the row holds and flagged in the status word, so that no
+// page id is ever read past the end of a row.
+__device__ __forceinline__ void scan_lengths(const int32_t *seq_lens, int B, int unit_tokens, int64_t max_tokens,
+                                             int *status, int32_t *prefix, int32_t *lens, int lane)
 {
     int carry = 0;
     for (int i0 = 0; i0 < B; i0 += 32) {
@@ -64,6 +66,10 @@ __device__ __forceinline__ void scan_lengths(const int32_t *seq_lens, int B, int
         if (i < B) {
             n = __ldg(seq_lens + i);
             n = n > 0 ? n : 0;
+            if ((int64_t)n > max_tokens) {
+                n = (int)max_tokens;
+                if (status) atomicOr(status, STATUS_BOUNDS);
+            }
             v = (n + unit_tokens - 1) / unit_tokens;
             lens[i] = n;
         }

@@ -37,8 +37,8 @@ class DeviceWorkload:
     def owners(self) -> List[int]:
         return [l for l in range(self.w.n_layers) if self.r[l] == l]
 
-    def retune(self, variant=None, tuning=None, overlap=None, l2_keep=None) -> None:
-        """Change kernel variant / launch shape / overlap / L2 reuse, then size the workspace again."""
+    def retune(self, variant=None, tuning=None, overlap=None, l2_keep=None, early_fetch=None, worker=None) -> None:
+        """Change kernel variant / launch shape / overlap / L2 reuse / early fetch, then size the workspace again."""
         if variant is not None:
             self.cache.skv_set_decode_variant(variant)
         if tuning is not None:
@@ -47,6 +47,10 @@ class DeviceWorkload:
             self.cache.skv_set_decode_overlap(overlap)
         if l2_keep is not None:
             self.cache.skv_set_decode_l2_reuse(l2_keep)
+        if early_fetch is not None:
+            self.cache.skv_set_decode_early_fetch(early_fetch)
+        if worker is not None:                       # mode, or (mode, consumers, stages)
+            self.cache.skv_set_decode_worker(*((worker,) if isinstance(worker, int) else worker))
         need = self.cache.skv_decode_workspace_bytes(self.batch, self.w.q_heads)
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
@@ -88,8 +92,10 @@ def setup(w: W.Workload, device="cuda", lens: Optional[torch.Tensor] = None, r: 
 
 
 def prefill(dw: DeviceWorkload, upto_offset: int = -1, layers: Optional[List[int]] = None,
-            chunk_tokens: int = 1 << 16) -> None:
-    """Append tokens t < lens[b] + upto_offset of every owner layer (drawn on the device)."""
+            chunk_tokens: int = 1 << 16, draw_on=None) -> None:
+    """Append tokens t < lens[b] + upto_offset of every owner layer.  The rows are drawn on the device
+    unless `draw_on` names another one ("cpu": drawn on the host and copied over, so that the only
+    kernels on the GPU are the library's; the generator gives the same bits on either)."""
     w = dw.w
     seq_idx, pos = W.token_index(dw.lens_cpu, upto_offset)
     slots = W.slot_map_for(dw.page_table_cpu, seq_idx, pos, w.page_size)
@@ -98,8 +104,8 @@ def prefill(dw: DeviceWorkload, upto_offset: int = -1, layers: Optional[List[int
             continue
         for s in range(0, seq_idx.numel(), chunk_tokens):
             e = min(seq_idx.numel(), s + chunk_tokens)
-            K, V = W.draw_kv(w, l, seq_idx[s:e], pos[s:e], device=dw.device)
-            dw.cache.skv_append(l, K, V, slots[s:e].to(dw.device))
+            K, V = W.draw_kv(w, l, seq_idx[s:e], pos[s:e], device=dw.device if draw_on is None else draw_on)
+            dw.cache.skv_append(l, K.to(dw.device), V.to(dw.device), slots[s:e].to(dw.device))
     torch.cuda.synchronize(dw.device)
 
 

@@ -51,13 +51,14 @@ def _decode_layer(dw, layer, Q=None, scale=0.0):
 
 
 def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True,
-                     overlap=None, l2_keep=None):
+                     overlap=None, l2_keep=None, early_fetch=None, worker=None):
     """One decode step of every layer: prefill n-1 tokens, append the last one, attend; compare all."""
     harness, dw = _make(w, lens=lens, r=r, permute=permute)
     if poison:   # every byte of the page area becomes a bf16 NaN pattern (0x7FC1)
         dw.pool_view = dw.cache.pool[256:].view(torch.int16)
         dw.pool_view.fill_(0x7FC1)
-    dw.retune(variant=variant or None, tuning=tuning, overlap=overlap, l2_keep=l2_keep)
+    dw.retune(variant=variant or None, tuning=tuning, overlap=overlap, l2_keep=l2_keep, early_fetch=early_fetch,
+              worker=worker)
     B = dw.batch
     harness.prefill(dw, upto_offset=-1)
     seqs = list(range(B))
@@ -110,6 +111,15 @@ def test_all_short_lengths(Hq, Hkv, D):
     _full_step_check(w, lens=lens)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 4, 128), (8, 2, 128), (8, 2, 64), (3, 1, 128)])
+def test_all_short_lengths_with_early_fetch(Hq, Hkv, D):
+    """The same lengths with the split-K launch filling its rings before it waits for the kernel before it
+    (the append of the step's token, or the kernel that produced Q): same outputs, same cache."""
+    lens = torch.arange(0, 3 * 16 + 1, dtype=torch.int32)
+    w = W.Workload("short", 3, Hq, Hkv, D, 16, lens.numel(), 0, 48, "explicit", explicit_r=(0, 0, 2), seed=11)
+    _full_step_check(w, lens=lens, early_fetch=1)
+
+
 def test_poisoned_pool_never_leaks():
     """Unused slots hold NaN patterns: tokens past seq_len must contribute nothing."""
     lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3], dtype=torch.int32)
@@ -124,17 +134,138 @@ def test_forced_variants_and_launch_shapes(variant, Hq, Hkv):
     lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15], dtype=torch.int32)
     w = W.Workload("variants", 2, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=6)
     for tuning in ((4, 3, 2), (1, 2, 1), (8, 2, 1), (2, 6, 2), (3, 4, 3), (2, 2, 4), (1, 1, 8), (8, 1, 1)):
-        _full_step_check(w, lens=lens, variant=variant, tuning=tuning, check_cache=False)
+        _full_step_check(w, lens=lens, variant=variant, tuning=tuning, check_cache=False, worker=1)
 
 
-@pytest.mark.parametrize("overlap,l2_keep", [(1, 0), (0, 0), (1, 30), (0, 100), (1, 1)])
-def test_overlap_and_walk_directions(overlap, l2_keep):
+@pytest.mark.parametrize("variant,Hq,Hkv,D", [(0, 8, 2, 128), (0, 4, 4, 128), (2, 4, 4, 64), (0, 16, 2, 64), (0, 3, 1, 128)])
+def test_cta_worker_shapes(variant, Hq, Hkv, D):
+    """The CTA-per-range kernel with other numbers of consumer warps and ring depths (ranges that hold many
+    whole segments, segments cut by range ends, consumers without a block in a run), with and without
+    early fetch, against the oracle; and the warp-per-range kernel on the same inputs."""
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15, 0, 4100, 17, 16], dtype=torch.int32)
+    w = W.Workload("cta", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=67)
+    for worker, early in (((2, 8, 0), 0), ((2, 1, 2), 0), ((2, 3, 5), 1), ((2, 5, 7), 0), ((2, 10, 4), 1),
+                          ((2, 8, 20), 1), ((2, 2, 26), 0), ((3, 8, 0), 1), ((3, 3, 2), 0), ((3, 10, 4), 0),
+                          (1, 0), (1, 1)):
+        _full_step_check(w, lens=lens, variant=variant, check_cache=False, worker=worker, early_fetch=early)
+
+
+def test_cta_worker_long_segments_and_reverse_walks():
+    """Segments much longer than a range (every CTA holds a piece of one segment and writes a partial), walked
+    forwards and backwards with part of the stream kept in L2."""
+    lens = torch.tensor([60000, 9000, 5], dtype=torch.int32)
+    for Hq, Hkv in ((8, 2), (2, 2)):
+        w = W.Workload("cta_long", 4, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 0, 3), seed=69)
+        _full_step_check(w, lens=lens, check_cache=False, l2_keep=35, early_fetch=1)
+
+
+@pytest.mark.parametrize("overlap,l2_keep,early", [(1, 0, 0), (0, 0, 0), (1, 30, 0), (0, 100, 0), (1, 1, 0),
+                                                   (1, 0, 1), (1, 35, 1), (0, 0, 1)])
+def test_overlap_and_walk_directions(overlap, l2_keep, early):
     """Plain vs overlappable launches; forward-only walks vs alternating directions with part of each
-    range kept in L2 (layers 0,1,2 read owner 0, layer 3 owns)."""
+    range kept in L2 (layers 0,1,2 read owner 0, layer 3 owns); rings filled before or after the wait
+    on the previous kernel."""
     lens = torch.tensor([5000, 33, 1, 256, 1023, 0, 90, 15, 2048], dtype=torch.int32)
     for Hq, Hkv in ((8, 2), (2, 2)):
         w = W.Workload("walks", 4, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 0, 3), seed=31)
-        _full_step_check(w, lens=lens, check_cache=False, overlap=overlap, l2_keep=l2_keep)
+        _full_step_check(w, lens=lens, check_cache=False, overlap=overlap, l2_keep=l2_keep, early_fetch=early)
+
+
+def test_early_fetch_sees_the_token_appended_just_before():
+    """A decoder's order of events, repeated: a kernel writes Q, the update appends one token per sequence,
+    the attention call follows at once with its rings filled early.  The newest token must be attended
+    (it carries nearly all the weight here) although the launch started before the update finished, and
+    the partials of the previous call must not be disturbed while its merge still reads them."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([16, 17, 1, 33, 4000, 250, 64], dtype=torch.int32)
+    w = W.Workload("early", 2, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=61)
+    dw = harness.setup(w, lens=lens)
+    dw.retune(early_fetch=1)
+    harness.prefill(dw, upto_offset=-1)
+    o = _oracle_for(dw, list(range(dw.batch)), range(w.n_layers), upto_offset=-1)
+    b = torch.arange(dw.batch, dtype=torch.int64)
+    last = dw.lens_cpu.to(torch.int64) - 1
+    shape = (dw.batch, w.q_heads, w.head_dim)
+    outs, refs = [], []
+    for rep in range(4):
+        # the new token's K is a large multiple of the query direction, so it dominates the softmax
+        Q = W.draw_rows(w.seed + rep, W.KIND_Q, 0, b, last, w.q_heads, w.head_dim, 1.0, dw.device)
+        K = (Q[:, ::w.q_heads // w.kv_heads, :].float() * 4.0).to(torch.bfloat16).contiguous()
+        V = W.draw_rows(w.seed + rep, W.KIND_V, 0, b, last, w.kv_heads, w.head_dim, 1.0, dw.device)
+        o.append(0, K.cpu(), V.cpu(), b, last)
+        out0 = torch.full(shape, float("nan"), dtype=torch.bfloat16, device=dw.device)
+        out1 = torch.full(shape, float("nan"), dtype=torch.bfloat16, device=dw.device)
+        Qd = torch.add(Q, out0.nan_to_num(0.0), alpha=0.0)       # Q comes out of a kernel of its own
+        dw.cache.skv_append(0, K, V, dw.slot_new)
+        dw.cache.skv_decode_attn(0, Qd, dw.page_table, dw.seq_lens, out0, dw.workspace)
+        dw.cache.skv_decode_attn(1, Qd, dw.page_table, dw.seq_lens, out1, dw.workspace)   # back to back, same workspace
+        outs.append((out0, out1))
+        refs.append(o.decode_attn(0, Q.cpu(), dw.lens_cpu))
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    for rep, ((out0, out1), ref) in enumerate(zip(outs, refs)):
+        for out in (out0, out1):
+            ok, err = _within_tol(out, ref)
+            assert ok, f"rep {rep}: max abs err {err}"
+
+
+def test_length_beyond_the_page_table_row_is_cut_and_flagged():
+    """seq_lens[b] that needs more pages than a page_table row holds: no id is read past the row; the
+    length is cut to the row and the device status says SKV_ERR_BOUNDS (decode and pre-fill)."""
+    from paper_2604_22782_b200 import harness
+    from paper_2604_22782_b200.binding import SKV_ERR_BOUNDS
+    lens = torch.tensor([40, 64, 7], dtype=torch.int32)
+    for fp8 in (False, True):
+        w = W.Workload("ptrow", 1, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0,), seed=71)
+        dw = harness.setup(w, lens=lens, fp8=fp8)
+        harness.prefill(dw, upto_offset=0)
+        width = dw.page_table.shape[1]
+        assert width == 4
+        Q = harness.step_inputs(dw, 0)["Q"]
+        good = torch.full((dw.batch, w.q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device=dw.device)
+        dw.cache.skv_decode_attn(0, Q, dw.page_table, dw.seq_lens, good, dw.workspace)
+        assert dw.cache.skv_get_status() == 0
+        too_long = dw.seq_lens.clone()
+        too_long[2] = width * 16 + 1            # the LAST row: ids past it would lie outside the tensor
+        out = torch.full_like(good, float("nan"))
+        dw.cache.skv_decode_attn(0, Q, dw.page_table, too_long, out, dw.workspace)
+        assert dw.cache.skv_get_status() == SKV_ERR_BOUNDS
+        ok, err = _within_tol(out[:2], good[:2].cpu().double())                       # the other rows are unaffected
+        assert ok, err
+        assert torch.isfinite(out.float()).all()
+        cu = torch.tensor([0, 1, 2, 3], dtype=torch.int32, device=dw.device)
+        pout = torch.full_like(good, float("nan"))
+        dw.cache.skv_prefill_attn(0, Q, cu, dw.page_table, too_long, pout, 1)
+        assert dw.cache.skv_get_status() == SKV_ERR_BOUNDS
+        assert torch.isnan(pout[2].float()).all()                # rows of the offending sequence are left untouched
+        assert torch.isfinite(pout[:2].float()).all()
+
+
+def test_workspace_query_matches_the_launch_after_retuning():
+    """skv_decode_workspace_bytes is what the launches check against, whatever the variant and launch shape."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([300, 77, 512, 129], dtype=torch.int32)
+    for fp8 in (False, True):
+        w = W.Workload("wsq", 1, 32, 8, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0,), seed=73)
+        dw = harness.setup(w, lens=lens, fp8=fp8)
+        harness.prefill(dw, upto_offset=0)
+        Q = harness.step_inputs(dw, 0)["Q"]
+        first = None
+        for variant, tuning in ((0, None), (2, None), (2, (1, 2, 1)), (2, (4, 2, 3)), (0, (2, 2, 8))):
+            dw.cache.skv_set_decode_variant(variant)
+            if tuning:
+                dw.cache.skv_set_decode_tuning(*tuning)
+            need = dw.cache.skv_decode_workspace_bytes(dw.batch, w.q_heads)
+            ws = torch.empty(need, dtype=torch.uint8, device=dw.device)      # exactly what the query says
+            out = torch.full((dw.batch, w.q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device=dw.device)
+            dw.cache.skv_decode_attn(0, Q, dw.page_table, dw.seq_lens, out, ws)
+            assert dw.cache.skv_get_status() == 0
+            first = out if first is None else first
+            ok, err = _within_tol(out, first.cpu().double())
+            assert ok, (fp8, variant, tuning, err)
+            if need > 256:
+                with pytest.raises(Exception):
+                    dw.cache.skv_decode_attn(0, Q, dw.page_table, dw.seq_lens, out, ws[:need - 256])
 
 
 @pytest.mark.parametrize("overlap,l2_keep", [(1, 0), (1, 40), (0, 0)])

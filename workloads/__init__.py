@@ -183,6 +183,16 @@ for _g in (1, 2, 4, 8):
     WORKLOADS[f"sweep_g{_g}"] = sweep_workload(_g)
 
 
+# Table 4's shape (Section 4.3): the Qwen3-8B architecture with groups of four layers, ONE sequence, 2 048
+# or 8 192 prompt tokens plus the 128 generated ones.  An owner layer's cache is 8.9 / 34.1 MB here,
+# well inside the L2 cache: the three reader layers of a group re-read what the owner layer just
+# streamed.  Four groups (16 layers) are enough to show that.
+for _t in (2048, 8192):
+    WORKLOADS[f"qwen3_8b_b1_{_t // 1024}k"] = Workload(
+        f"qwen3_8b_b1_{_t // 1024}k", 16, 32, 8, 128, 16, 1, _t + 128, _t + 128, "groups", group=4,
+        explicit_lens=(_t + 128,), seed=5, q_std=0.5, family="Qwen3-8B")
+
+
 def get_workload(name: str) -> Workload:
     return WORKLOADS[name]
 
