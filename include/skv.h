@@ -395,15 +395,20 @@ int skv_set_decode_overlap(skv_cache *cache, int enabled);
 /* Which worker the split-K pass of a stand-alone attention call uses
  * (skv_decode_attn, skv_decode_attn_static; the two-call form skv_decode_splitk +
  * skv_decode_merge and the chained launches of skv_decode_step always use warps).
- *   mode 0 (default) or 2: a CTA per SM -- `consumers` warps (1..12, default 8; 0
- *        keeps the current value) share one ring of `stages` 8 KB stages (2..26;
- *        0, the default: as many as shared memory allows, at most 20) filled by a
- *        producer warp, take its blocks in turn and combine their running states
- *        in shared memory at the end of every (sequence, kv head);
+ *   mode 0 (default) or 2: CTAs that own a range each -- `consumers` warps
+ *        (1..12; 0 keeps the current value) share one ring of `stages` stages of
+ *        one (page, kv head) block (2..26; 0, the default: as many as fit, at
+ *        most 20 per SM) filled by a producer warp, take its blocks in turn and
+ *        combine their running states in shared memory at the end of every
+ *        (sequence, kv head).  The grid is `ctas_per_sm` (1..4; 0 keeps the current
+ *        value, default 1) CTAs per SM, all resident at once;
+ *   mode 3: as 2, but a consumer takes the ring's next block whenever it is free
+ *        instead of every consumers-th one (results then vary in their last bits
+ *        from run to run);
  *   mode 1: a warp per range, launch shape from skv_set_decode_tuning.
- * FP8 pages at head_dim 128 keep their tcgen05 kernel either way.  Results agree
- * to rounding (the order of the sums differs). */
-int skv_set_decode_worker(skv_cache *cache, int mode, int consumers, int stages);
+ * FP8 pages at head_dim 128 keep their tcgen05 kernel either way.  Results of
+ * the modes agree to rounding (the order of the sums differs). */
+int skv_set_decode_worker(skv_cache *cache, int mode, int consumers, int stages, int ctas_per_sm);
 
 /* Early fetch for stand-alone attention calls (skv_decode_attn, skv_decode_attn_static,
  * skv_decode_splitk; needs skv_set_decode_overlap on).  0 (default): a split-K

@@ -77,7 +77,7 @@ lib.skv_set_prefill_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
 lib.skv_set_decode_early_fetch.argtypes = [_vp, _int]
-lib.skv_set_decode_worker.argtypes = [_vp, _int, _int, _int]
+lib.skv_set_decode_worker.argtypes = [_vp, _int, _int, _int, _int]
 lib.skv_set_host_step.argtypes = [_vp, _int, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
 lib.skv_decode_worker_count.argtypes = [_vp]
@@ -183,6 +183,30 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     return None if t is None else t.data_ptr()
 
 
+def _arg(name: str, t: Optional[torch.Tensor], dtype, shape=None, min_numel: Optional[int] = None,
+         cuda: Optional[bool] = True) -> Optional[torch.Tensor]:
+    """Checks a tensor argument before its raw pointer goes to the library: dtype, device (cuda=None: either),
+    contiguity, and an exact shape or a minimum number of elements.  The kernels trust the sizes they are
+    given, so a wrong one here would be an out-of-bounds access there."""
+    if t is None:
+        return None
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if cuda is not None and t.is_cuda != cuda:
+        raise ValueError(f"{name}: expected a {'CUDA' if cuda else 'host'} tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    if min_numel is not None and t.numel() < min_numel:
+        raise ValueError(f"{name}: needs at least {min_numel} elements, has {t.numel()}")
+    return t
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
 class SkvCache:
     """Handle of one routed cache.  ``device_pool`` is a torch uint8 CUDA tensor
     of at least ``skv_cache_pool_bytes`` bytes that the caller keeps alive; pass
@@ -248,11 +272,19 @@ class SkvCache:
                    slot_map: Optional[torch.Tensor], n_tokens: Optional[int] = None, stream=None) -> None:
         if n_tokens is None:
             n_tokens = 0 if slot_map is None else slot_map.numel()
+        row = (n_tokens, self.kv_heads, self.head_dim)
+        _arg("K", K, torch.bfloat16, row)
+        _arg("V", V, torch.bfloat16, row)
+        _arg("slot_map", slot_map, torch.int64, min_numel=n_tokens)
         rc = lib.skv_append(self._h, layer, _ptr(K), _ptr(V), _ptr(slot_map), n_tokens, _stream_ptr(stream))
         _check(rc, "skv_append")
 
     def skv_gather(self, layer: int, slot_ids: torch.Tensor, K_out: torch.Tensor, V_out: torch.Tensor,
                    stream=None) -> None:
+        n = slot_ids.numel()
+        _arg("slot_ids", slot_ids, torch.int64)
+        _arg("K_out", K_out, torch.bfloat16, (n, self.kv_heads, self.head_dim))
+        _arg("V_out", V_out, torch.bfloat16, (n, self.kv_heads, self.head_dim))
         rc = lib.skv_gather(self._h, layer, _ptr(slot_ids), slot_ids.numel(), _ptr(K_out), _ptr(V_out),
                             _stream_ptr(stream))
         _check(rc, "skv_gather")
@@ -264,6 +296,21 @@ class SkvCache:
         _check(rc, "skv_gather_fp8")
 
     # -- Load + Attn
+    def _decode_args(self, Q, page_table, seq_lens, out):
+        """Shapes of one decode-attention call: Q, out [batch][q_heads][head_dim] bf16; page_table
+        [batch][width] int32; seq_lens [batch] int32, all on the device."""
+        if Q.dim() != 3 or Q.shape[2] != self.head_dim:
+            raise ValueError(f"Q: expected [batch][q_heads][{self.head_dim}], got {tuple(Q.shape)}")
+        batch, q_heads = Q.shape[0], Q.shape[1]
+        _arg("Q", Q, torch.bfloat16)
+        if out is not None:
+            _arg("out", out, torch.bfloat16, Q.shape)
+        _arg("page_table", page_table, torch.int32)
+        if page_table.dim() != 2 or page_table.shape[0] != batch:
+            raise ValueError(f"page_table: expected [{batch}][width], got {tuple(page_table.shape)}")
+        _arg("seq_lens", seq_lens, torch.int32, (batch,))
+        return batch, q_heads
+
     def skv_decode_workspace_bytes(self, batch: int, q_heads: int) -> int:
         out = _sz(0)
         _check(lib.skv_decode_workspace_bytes(self._h, batch, q_heads, ctypes.byref(out)),
@@ -272,9 +319,10 @@ class SkvCache:
 
     def skv_decode_attn(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
                         out: torch.Tensor, workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:
-        batch, q_heads = Q.shape[0], Q.shape[1]
+        batch, q_heads = self._decode_args(Q, page_table, seq_lens, out)
+        _arg("workspace", workspace, torch.uint8)
         rc = lib.skv_decode_attn(self._h, layer, _ptr(Q), _ptr(page_table), _ptr(seq_lens), _ptr(out), batch,
-                                 q_heads, page_table.shape[1], scale, _ptr(workspace), workspace.numel(),
+                                 q_heads, page_table.shape[1], scale, _ptr(workspace), _nbytes(workspace),
                                  _stream_ptr(stream))
         _check(rc, "skv_decode_attn")
 
@@ -283,15 +331,28 @@ class SkvCache:
         """skv_decode_attn without a workspace argument, for callers that cannot allocate device memory:
         the scratch is a fixed SKV_STATIC_SCRATCH_BYTES area inside the library (shared by all calls on
         the device; calls that overlap on the GPU race on it)."""
-        batch, q_heads = Q.shape[0], Q.shape[1]
+        batch, q_heads = self._decode_args(Q, page_table, seq_lens, out)
         rc = lib.skv_decode_attn_static(self._h, layer, _ptr(Q), _ptr(page_table), _ptr(seq_lens), _ptr(out),
                                         batch, q_heads, page_table.shape[1], scale, _stream_ptr(stream))
         _check(rc, "skv_decode_attn_static")
 
+    def _prefill_args(self, Q, cu_q_lens, page_table, seq_lens, out):
+        if Q.dim() != 3 or Q.shape[2] != self.head_dim:
+            raise ValueError(f"Q: expected [n_q][q_heads][{self.head_dim}], got {tuple(Q.shape)}")
+        batch = seq_lens.shape[0]
+        _arg("Q", Q, torch.bfloat16)
+        _arg("out", out, torch.bfloat16, Q.shape)
+        _arg("cu_q_lens", cu_q_lens, torch.int32, (batch + 1,))
+        _arg("page_table", page_table, torch.int32)
+        if page_table.dim() != 2 or page_table.shape[0] != batch:
+            raise ValueError(f"page_table: expected [{batch}][width], got {tuple(page_table.shape)}")
+        _arg("seq_lens", seq_lens, torch.int32, (batch,))
+        return batch, Q.shape[1]
+
     def skv_prefill_attn(self, layer: int, Q: torch.Tensor, cu_q_lens: torch.Tensor, page_table: torch.Tensor,
                          seq_lens: torch.Tensor, out: torch.Tensor, max_q_len: int, scale: float = 0.0,
                          stream=None) -> None:
-        batch, q_heads = seq_lens.shape[0], Q.shape[1]
+        batch, q_heads = self._prefill_args(Q, cu_q_lens, page_table, seq_lens, out)
         rc = lib.skv_prefill_attn(self._h, layer, _ptr(Q), _ptr(cu_q_lens), _ptr(page_table), _ptr(seq_lens),
                                   _ptr(out), batch, max_q_len, q_heads, page_table.shape[1], scale,
                                   _stream_ptr(stream))
@@ -300,7 +361,7 @@ class SkvCache:
     def skv_prefill_attn_src(self, src_layer: int, Q: torch.Tensor, cu_q_lens: torch.Tensor, page_table: torch.Tensor,
                              seq_lens: torch.Tensor, out: torch.Tensor, max_q_len: int, scale: float = 0.0,
                              stream=None) -> None:
-        batch, q_heads = seq_lens.shape[0], Q.shape[1]
+        batch, q_heads = self._prefill_args(Q, cu_q_lens, page_table, seq_lens, out)
         rc = lib.skv_prefill_attn_src(self._h, src_layer, _ptr(Q), _ptr(cu_q_lens), _ptr(page_table), _ptr(seq_lens),
                                       _ptr(out), batch, max_q_len, q_heads, page_table.shape[1], scale,
                                       _stream_ptr(stream))
@@ -308,26 +369,48 @@ class SkvCache:
 
     def skv_decode_splitk(self, layer: int, Q: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
                           workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:
-        batch, q_heads = Q.shape[0], Q.shape[1]
+        batch, q_heads = self._decode_args(Q, page_table, seq_lens, None)
+        _arg("workspace", workspace, torch.uint8)
         rc = lib.skv_decode_splitk(self._h, layer, _ptr(Q), _ptr(page_table), _ptr(seq_lens), batch, q_heads,
-                                   page_table.shape[1], scale, _ptr(workspace), workspace.numel(),
+                                   page_table.shape[1], scale, _ptr(workspace), _nbytes(workspace),
                                    _stream_ptr(stream))
         _check(rc, "skv_decode_splitk")
 
     def skv_decode_merge(self, out: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
         batch, q_heads = out.shape[0], out.shape[1]
+        _arg("out", out, torch.bfloat16, (batch, q_heads, self.head_dim))
+        _arg("workspace", workspace, torch.uint8)
         rc = lib.skv_decode_merge(self._h, _ptr(out), batch, q_heads, _ptr(workspace),
-                                  workspace.numel(), _stream_ptr(stream))
+                                  _nbytes(workspace), _stream_ptr(stream))
         _check(rc, "skv_decode_merge")
 
     def skv_decode_step(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, slot_map: torch.Tensor,
                         page_table: torch.Tensor, seq_lens: torch.Tensor, out: torch.Tensor,
                         workspace: torch.Tensor, scale: float = 0.0, stream=None) -> None:
         batch, q_heads = Q.shape[1], Q.shape[2]
+        self._step_args(Q, K, V, slot_map, page_table, seq_lens, out, cuda=True)
+        _arg("workspace", workspace, torch.uint8)
         rc = lib.skv_decode_step(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(slot_map), _ptr(page_table),
                                  _ptr(seq_lens), _ptr(out), batch, q_heads, page_table.shape[1], scale,
-                                 _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+                                 _ptr(workspace), _nbytes(workspace), _stream_ptr(stream))
         _check(rc, "skv_decode_step")
+
+    def _step_args(self, Q, K, V, slot_map, page_table, seq_lens, out, cuda):
+        """Shapes of one whole step: Q, out [n_layers][batch][q_heads][head_dim]; K, V
+        [n_owners][batch][kv_heads][head_dim]; slot_map [batch] int64; page_table [batch][width]; seq_lens [batch]."""
+        if Q.dim() != 4 or Q.shape[0] != self.n_layers or Q.shape[3] != self.head_dim:
+            raise ValueError(f"Q: expected [{self.n_layers}][batch][q_heads][{self.head_dim}], got {tuple(Q.shape)}")
+        batch = Q.shape[1]
+        n_owners = sum(1 for l, s in enumerate(self.r) if s == l)
+        _arg("Q", Q, torch.bfloat16, cuda=cuda)
+        _arg("out", out, torch.bfloat16, Q.shape, cuda=cuda)
+        _arg("K", K, torch.bfloat16, (n_owners, batch, self.kv_heads, self.head_dim), cuda=cuda)
+        _arg("V", V, torch.bfloat16, (n_owners, batch, self.kv_heads, self.head_dim), cuda=cuda)
+        _arg("slot_map", slot_map, torch.int64, (batch,), cuda=cuda)
+        _arg("page_table", page_table, torch.int32, cuda=cuda)
+        if page_table.dim() != 2 or page_table.shape[0] != batch:
+            raise ValueError(f"page_table: expected [{batch}][width], got {tuple(page_table.shape)}")
+        _arg("seq_lens", seq_lens, torch.int32, (batch,), cuda=cuda)
 
     def skv_decode_step_staging_bytes(self, batch: int, q_heads: int, pt_stride: int) -> int:
         out = _sz(0)
@@ -339,9 +422,11 @@ class SkvCache:
                              h_page_table: torch.Tensor, h_seq_lens: torch.Tensor, h_out: torch.Tensor,
                              staging: torch.Tensor, scale: float = 0.0, stream=None) -> None:
         batch, q_heads = hQ.shape[1], hQ.shape[2]
+        self._step_args(hQ, hK, hV, h_slot_map, h_page_table, h_seq_lens, h_out, cuda=False)
+        _arg("staging", staging, torch.uint8)
         rc = lib.skv_decode_step_host(self._h, _ptr(hQ), _ptr(hK), _ptr(hV), _ptr(h_slot_map), _ptr(h_page_table),
                                       _ptr(h_seq_lens), _ptr(h_out), batch, q_heads, h_page_table.shape[1], scale,
-                                      _ptr(staging), staging.numel(), _stream_ptr(stream))
+                                      _ptr(staging), _nbytes(staging), _stream_ptr(stream))
         _check(rc, "skv_decode_step_host")
 
     # -- status, tuning, counters
@@ -362,8 +447,8 @@ class SkvCache:
     def skv_set_decode_overlap(self, enabled: int) -> None:
         _check(lib.skv_set_decode_overlap(self._h, enabled), "skv_set_decode_overlap")
 
-    def skv_set_decode_worker(self, mode: int, consumers: int = 0, stages: int = 0) -> None:
-        _check(lib.skv_set_decode_worker(self._h, mode, consumers, stages), "skv_set_decode_worker")
+    def skv_set_decode_worker(self, mode: int, consumers: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
+        _check(lib.skv_set_decode_worker(self._h, mode, consumers, stages, ctas_per_sm), "skv_set_decode_worker")
 
     def skv_set_decode_early_fetch(self, enabled: int) -> None:
         _check(lib.skv_set_decode_early_fetch(self._h, enabled), "skv_set_decode_early_fetch")

@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libskv.so")
+LIB_TEST_HOOKS = os.path.join(_HERE, "libskv_testhooks.so")      # the library plus include/skv_test_hooks.h's entry points
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC",
@@ -25,7 +26,7 @@ def sources():
 
 
 def _headers():
-    return glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(_HERE, "..", "include", "skv.h")]
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(_HERE, "..", "include", "*.h"))
 
 
 def _newest_source_mtime() -> float:
@@ -67,5 +68,12 @@ def build(force: bool = False, verbose: bool = False, lib: str = LIB, defines=()
     return lib
 
 
+def build_test_hooks(force: bool = False) -> str:
+    """The same sources with -DSKV_TEST_HOOKS, as a second library for the test suite."""
+    return build(force=force, lib=LIB_TEST_HOOKS, defines=["SKV_TEST_HOOKS"])
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--test-hooks" in sys.argv:
+        print(build_test_hooks(force="--force" in sys.argv))

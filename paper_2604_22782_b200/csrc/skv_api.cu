@@ -62,7 +62,8 @@ struct skv_cache {
     int worker_mode = 0;             // 0 auto (CTA per range for stand-alone calls, warp per range inside chains),
                                      // 1 warp per range always, 2 CTA per range wherever it applies
     int cta_consumers = 8;           // consumer warps per CTA of the CTA-per-range kernel
-    int cta_stages = 0;              // its ring depth; 0 = as deep as shared memory allows, up to 20
+    int cta_stages = 0;              // its ring depth; 0 = as deep as shared memory allows, up to 20 per SM
+    int cta_per_sm = 1;              // its CTAs resident per SM
     bool cta_in_turn = true;         // its consumers take the blocks in turn (reproducible) instead of first come first served
     std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
     std::vector<uint8_t> walk_keep;      // per layer: the next layer reads the same owner
@@ -149,8 +150,8 @@ int n_workers_of(const skv_cache *c)
     return sm * c->tune.ctas_per_sm * c->tune.warps;
 }
 
-// Workers of a CTA-per-range launch: one CTA per SM.
-int n_cta_workers_of(const skv_cache *c) { return c->sm_count > 0 ? c->sm_count : 148; }
+// Workers of a CTA-per-range launch: the CTAs that are resident at once.
+int n_cta_workers_of(const skv_cache *c) { return (c->sm_count > 0 ? c->sm_count : 148) * c->cta_per_sm; }
 
 // The workspace is sized for whichever kernel leaves more partials (a call may run either).
 int n_workers_max(const skv_cache *c)
@@ -163,8 +164,10 @@ int n_workers_max(const skv_cache *c)
 // (at most 20); 0 if not even two fit.
 int cta_stages_for(const skv_cache *c, int batch, int G)
 {
-    int S = c->cta_stages > 0 ? c->cta_stages : 20;
-    while (S >= 2 && decode_cta_smem_bytes(c->head_dim, batch, G, c->cta_consumers, S, c->fp8) > (size_t)c->max_smem_optin) --S;
+    int S = c->cta_stages > 0 ? c->cta_stages : 20 / c->cta_per_sm;
+    // (what one CTA may take when cta_per_sm of them share an SM: the SM's shared memory less 1 KB per CTA the system keeps)
+    const size_t room = ((size_t)c->max_smem_optin + 1024) / c->cta_per_sm - 1024;
+    while (S >= 2 && decode_cta_smem_bytes(c->head_dim, batch, G, c->cta_consumers, S, c->fp8) > room) --S;
     // by default a whole number of rounds of the consumers (a stage then always serves the same consumer)
     if (c->cta_stages == 0 && S >= 2 * c->cta_consumers) S -= S % c->cta_consumers;
     return S >= 2 ? S : 0;
@@ -1077,14 +1080,16 @@ int skv_set_decode_early_fetch(skv_cache *c, int enabled)
     return SKV_OK;
 }
 
-int skv_set_decode_worker(skv_cache *c, int mode, int consumers, int stages)
+int skv_set_decode_worker(skv_cache *c, int mode, int consumers, int stages, int ctas_per_sm)
 {
-    if (!c || mode < 0 || mode > 3 || consumers < 0 || consumers > 12 || stages < 0 || stages == 1 || stages > 26)
+    if (!c || mode < 0 || mode > 3 || consumers < 0 || consumers > 12 || stages < 0 || stages == 1 || stages > 26 ||
+        ctas_per_sm < 0 || ctas_per_sm > 4)
         return SKV_ERR_ARG;
     c->cta_in_turn = mode != 3;
     c->worker_mode = mode == 3 ? 2 : mode;
     if (consumers) c->cta_consumers = consumers;
     c->cta_stages = stages;
+    if (ctas_per_sm) c->cta_per_sm = ctas_per_sm;
     return SKV_OK;
 }
 

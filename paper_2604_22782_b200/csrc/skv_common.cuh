@@ -257,16 +257,22 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     return t;
 }
 
-// Bounded wait: gives up after about two seconds and returns false.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Bounded wait: gives up after limit_ns nanoseconds and returns false.
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > 2000000000ull) return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
     }
+}
+
+// The kernels' limit: about two seconds.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    return mbar_wait_limited(bar, parity, 2000000000ull);
 }
 
 // linear bulk copy global -> this CTA's shared memory, completion on an mbarrier

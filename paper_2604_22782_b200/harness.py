@@ -49,7 +49,7 @@ class DeviceWorkload:
             self.cache.skv_set_decode_l2_reuse(l2_keep)
         if early_fetch is not None:
             self.cache.skv_set_decode_early_fetch(early_fetch)
-        if worker is not None:                       # mode, or (mode, consumers, stages)
+        if worker is not None:                       # mode, or (mode, consumers, stages, CTAs per SM)
             self.cache.skv_set_decode_worker(*((worker,) if isinstance(worker, int) else worker))
         need = self.cache.skv_decode_workspace_bytes(self.batch, self.w.q_heads)
         if need > self.workspace.numel():

@@ -1,5 +1,7 @@
-"""The five full-size workloads, in the launch configuration the benchmark times (library defaults,
-whole step through skv_decode_step).  The oracle cannot hold these whole, so:
+"""The five full-size workloads, in the launch configurations the benchmark times: the step layer by layer
+through skv_append / skv_decode_attn with early fetch on (each layer's query written by a kernel that reads
+the previous layer's output), and the whole step through skv_decode_step.  The Llama-3-8B workload is
+compared with the oracle in full (every sequence, every layer).  The oracle cannot hold the others whole, so:
   - cache contents are compared bit for bit for EVERY token of EVERY owner layer, on the device,
     against the rows the generator draws (the update is a pure copy);
   - attention outputs are compared with the oracle, element by element within
@@ -38,7 +40,7 @@ def _sample_layers(r):
     return sorted({0, first_reader, owners[-1], L - 1})
 
 
-def _check_workload(w, n_seqs):
+def _check_workload(w, n_seqs, all_layers=False):
     from oracle import Oracle
     from paper_2604_22782_b200 import harness
     dw = harness.setup(w)
@@ -48,6 +50,22 @@ def _check_workload(w, n_seqs):
     dw.cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
     torch.cuda.synchronize()
     assert dw.cache.skv_get_status() == 0
+    # the same step as a decoder issues it: per layer a kernel that makes the query from the previous layer's
+    # output, the update (owners), the attention call with early fetch on (the benchmark's headline leg)
+    dw.retune(early_fetch=1)
+    loop_out = torch.full_like(t["out"], float("nan"))
+    q_dep = torch.empty_like(t["Q"][0])
+    for l in range(w.n_layers):
+        torch.add(t["Q"][l], t["out"][l - 1], alpha=0.0, out=q_dep)
+        if dw.r[l] == l:
+            i = dw.owners.index(l)
+            dw.cache.skv_append(l, t["K"][i], t["V"][i], dw.slot_new)
+        dw.cache.skv_decode_attn(l, q_dep, dw.page_table, dw.seq_lens, loop_out[l], dw.workspace)
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    dw.retune(early_fetch=0)
+    a, b = loop_out.float(), t["out"].float()
+    assert bool(((a - b).abs() <= 2 * ATOL + RTOL * b.abs()).all()), "per-layer loop and whole-step call disagree"
 
     # byte accounting scales exactly with the owner count
     stats = dw.cache.skv_cache_stats()
@@ -70,7 +88,7 @@ def _check_workload(w, n_seqs):
 
     # attention outputs of the sampled sequences on the sampled layers against the oracle
     seqs = _sample_sequences(dw.lens_cpu, n_seqs, w.seed + 7)
-    layers = _sample_layers(dw.r)
+    layers = list(range(w.n_layers)) if all_layers else _sample_layers(dw.r)
     sub_lens = dw.lens_cpu[seqs]
     o = Oracle(w.n_layers, dw.r, w.q_heads, w.kv_heads, w.head_dim, len(seqs), int(sub_lens.max()))
     local, lpos = W.token_index(sub_lens)
@@ -84,23 +102,34 @@ def _check_workload(w, n_seqs):
     for l in layers:
         Q = t["Q"][l].cpu()[seqs]
         ref = o.decode_attn(l, Q, sub_lens)
-        got = t["out"][l].cpu()[seqs].double()
-        err = (got - ref).abs()
-        assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {l}: max abs err {err.max().item()}"
-        worst = max(worst, err.max().item())
+        for name, res in (("skv_decode_step", t["out"]), ("per-layer loop", loop_out)):
+            got = res[l].cpu()[seqs].double()
+            err = (got - ref).abs()
+            assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"{name}, layer {l}: max abs err {err.max().item()}"
+            worst = max(worst, err.max().item())
     o.close()
 
     # every row: finite and inside the convex-combination bound
     vmax = 5.0 * w.kv_std            # the generator's table ends below 4.5 standard deviations
-    out = t["out"].float()
-    assert torch.isfinite(out).all()
-    assert out.abs().max().item() <= vmax
+    for res in (t["out"], loop_out):
+        out = res.float()
+        assert torch.isfinite(out).all()
+        assert out.abs().max().item() <= vmax
     return worst
 
 
 def test_llama3_8b_full_size():
-    """Config 2: 32 layers, 32q/8kv, D=128, 16 owners, batch 32, lengths U[1024,4096]."""
-    _check_workload(W.get_workload("llama3_8b"), n_seqs=6)
+    """Config 2: 32 layers, 32q/8kv, D=128, 16 owners, batch 32, lengths U[1024,4096]: every sequence on
+    every layer against the oracle (16 source stores of 32 x 4096 tokens on the host)."""
+    _check_workload(W.get_workload("llama3_8b"), n_seqs=32, all_layers=True)
+
+
+@pytest.mark.parametrize("name", ["qwen3_8b_b1_2k", "qwen3_8b_b1_8k"])
+def test_table4_shape_one_sequence(name):
+    """Table 4's shape: Qwen3-8B heads, groups of four layers, ONE sequence of 2 048 / 8 192 + 128 tokens (an
+    owner layer's cache fits in L2 and is loaded with normal priority for the group's reader layers): every
+    layer against the oracle."""
+    _check_workload(W.get_workload(name), n_seqs=1, all_layers=True)
 
 
 def test_qwen3_8b_full_size():

@@ -146,6 +146,7 @@ def test_cta_worker_shapes(variant, Hq, Hkv, D):
     w = W.Workload("cta", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=67)
     for worker, early in (((2, 8, 0), 0), ((2, 1, 2), 0), ((2, 3, 5), 1), ((2, 5, 7), 0), ((2, 10, 4), 1),
                           ((2, 8, 20), 1), ((2, 2, 26), 0), ((3, 8, 0), 1), ((3, 3, 2), 0), ((3, 10, 4), 0),
+                          ((2, 4, 0, 2), 1), ((2, 4, 6, 2), 0), ((2, 2, 4, 4), 1), ((2, 8, 0, 1), 0),
                           (1, 0), (1, 1)):
         _full_step_check(w, lens=lens, variant=variant, check_cache=False, worker=worker, early_fetch=early)
 
@@ -157,6 +158,7 @@ def test_cta_worker_long_segments_and_reverse_walks():
     for Hq, Hkv in ((8, 2), (2, 2)):
         w = W.Workload("cta_long", 4, Hq, Hkv, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 0, 3), seed=69)
         _full_step_check(w, lens=lens, check_cache=False, l2_keep=35, early_fetch=1)
+        _full_step_check(w, lens=lens, check_cache=False, l2_keep=35, early_fetch=1, worker=(2, 4, 0, 2))
 
 
 @pytest.mark.parametrize("overlap,l2_keep,early", [(1, 0, 0), (0, 0, 0), (1, 30, 0), (0, 100, 0), (1, 1, 0),
