@@ -58,6 +58,78 @@ __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
     *reinterpret_cast<uint4 *>(dst) = __ldg(src);
 }
 
+// Large calls (a prompt): one warp per (group of 16 consecutive tokens of the call, kv head), grid.y = K or V,
+// grid.z = owner layer.  The warp reads the group's 16 rows of that head as whole rows (two 256-byte rows per
+// load instruction at head_dim 128: full lines, where the kernel above reads 32 bytes per token and
+// instruction).  If the 16 tokens are the 16 slots of one page, in order -- what a prompt's tokens are -- the
+// rows are turned into the page's chunk-major half through shared memory and written as one contiguous run
+// (4 KB at head_dim 128); the shared-memory positions are XOR-swizzled so that neither the row-major writes
+// nor the chunk-major reads conflict.  Any other slot pattern (loose tokens, holes, reversed pages, the
+// ragged end of the call) takes the rows the same way and scatters their 16-byte chunks one by one, as the
+// kernel above does: the same cache for every slot map.
+constexpr int PAGE_WARPS = 8;
+
+__global__ void __launch_bounds__(PAGE_WARPS * 32, 4) append_pages_kernel(AppendParams p)
+{
+    pdl_trigger();
+    __shared__ __align__(16) uint4 stage[PAGE_WARPS][PAGE * 16];
+    constexpr unsigned ALL = 0xFFFFFFFFu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int CH = p.D / CHUNK_ELEMS;                     // 16-byte chunks per row of one head: 16 or 8
+    const int rows_per_load = 32 / CH, loads = PAGE / rows_per_load;
+    const int c = lane % CH, t_in_load = lane / CH;
+    const int64_t n_groups = (p.n_tokens + PAGE - 1) / PAGE, n_items = n_groups * p.Hkv;
+    const int which = blockIdx.y;
+    const int64_t layer = blockIdx.z;
+    const uint4 *rows = (which ? p.V : p.K) + layer * p.n_tokens * p.Hkv * CH;
+    uint8_t *half = p.layer_base + layer * p.layer_stride + (int64_t)which * half_bytes(p.D);
+    for (int64_t item = (int64_t)blockIdx.x * PAGE_WARPS + warp; item < n_items; item += (int64_t)gridDim.x * PAGE_WARPS) {
+        const int64_t g = item / p.Hkv;
+        const int h = (int)(item - g * p.Hkv);
+        const int64_t i0 = g * PAGE;
+        // the rows first (their addresses do not depend on the slots), so that both trips to memory overlap
+        uint4 v[PAGE / 2];                                // at most 8 loads (head_dim 128)
+#pragma unroll
+        for (int i = 0; i < PAGE / 2; ++i) {
+            const int64_t tok = i0 + i * rows_per_load + t_in_load;
+            v[i] = (i < loads && tok < p.n_tokens) ? __ldg(rows + (tok * p.Hkv + h) * CH + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        const int64_t mine = (lane < PAGE && i0 + lane < p.n_tokens) ? p.slot_map[i0 + lane] : -1;
+        const int64_t first = __shfl_sync(ALL, mine, 0);
+        const bool whole = __all_sync(ALL, lane >= PAGE || (first >= 0 && first % PAGE == 0 && first + PAGE <= p.n_slots &&
+                                                             mine == first + lane));
+        if (whole) {
+#pragma unroll
+            for (int i = 0; i < PAGE / 2; ++i)
+                if (i < loads) {
+                    const int t = i * rows_per_load + t_in_load;
+                    stage[warp][c * PAGE + (t ^ (c & (PAGE - 1)))] = v[i];
+                }
+            __syncwarp();
+            uint4 *dst = reinterpret_cast<uint4 *>(half + (first / PAGE) * p.page_stride + (int64_t)h * block_bytes(p.D));
+            for (int u = lane; u < CH * PAGE; u += 32) {
+                const int c2 = u / PAGE, t2 = u % PAGE;
+                dst[u] = stage[warp][c2 * PAGE + (t2 ^ (c2 & (PAGE - 1)))];
+            }
+            __syncwarp();
+        } else {
+#pragma unroll
+            for (int i = 0; i < PAGE / 2; ++i) {
+                const int t = i * rows_per_load + t_in_load;             // (< PAGE also for i >= loads: a lane that exists)
+                const int64_t slot = __shfl_sync(ALL, mine, t & (PAGE - 1));
+                if (i >= loads || i0 + t >= p.n_tokens || slot < 0) continue;
+                if (slot >= p.n_slots) {
+                    if (h == 0 && c == 0 && which == 0) atomicOr(p.status, STATUS_BOUNDS);
+                    continue;
+                }
+                const int64_t page = slot / PAGE;
+                const int off = (int)(slot - page * PAGE);
+                *reinterpret_cast<uint4 *>(half + page * p.page_stride + (int64_t)h * block_bytes(p.D) + ((int64_t)c * PAGE + off) * 16) = v[i];
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(COPY_THREADS) gather_kernel(GatherParams p)
 {
     const int CH = p.D / CHUNK_ELEMS;
@@ -157,6 +229,82 @@ __device__ __forceinline__ void append_fp8_page(const AppendFp8Params &p, int64_
     if (lane < PAGE) *reinterpret_cast<float *>(blk + fp8_vs_off(D) + 4 * lane) = my_scale;
 }
 
+// The same page, all 16 rows at once (the large-call kernel).  The rows come in as whole rows (coalesced)
+// through shared memory; then lane (token t = lane % 16, half hf = lane / 16) owns half a row: its maximum
+// needs ONE shuffle with the other half's (instead of five per row, row after row), and it quantises D/2
+// values.  K codes leave as the 16-byte pieces of the page layout; V codes are turned dim-major through shared
+// memory (a piece = one dim x 16 tokens).  in_rows: PAGE x (2 D + 16) bytes, codes: PAGE x (D + 4) bytes of
+// shared memory of this warp (the paddings keep the column accesses off one bank).
+__device__ __forceinline__ void append_fp8_page_wide(const AppendFp8Params &p, int64_t t0, int64_t page, int h, int which,
+                                                     int64_t layer, int lane, uint8_t *in_rows, uint8_t *codes)
+{
+    const int D = p.D, row_bytes = 2 * D, in_stride = row_bytes + 16, code_stride = D + 4;
+    const uint16_t *rows = (which ? p.V : p.K) + (layer * p.n_tokens * p.Hkv + h) * D;      // row of token t: + t * Hkv * D
+    uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
+    // ---- rows -> shared memory: 32 lanes x 16 bytes per load, PAGE * row_bytes / 512 loads (8 at head_dim 128)
+    const int units = row_bytes / 16, n_loads = PAGE * units / 32;
+    uint4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if (i < n_loads) {
+            const int u = i * 32 + lane, r = u / units, cu = u - r * units;
+            v[i] = __ldg(reinterpret_cast<const uint4 *>(rows + (t0 + r) * p.Hkv * D) + cu);
+        }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if (i < n_loads) {
+            const int u = i * 32 + lane, r = u / units, cu = u - r * units;
+            *reinterpret_cast<uint4 *>(in_rows + r * in_stride + cu * 16) = v[i];
+        }
+    __syncwarp();
+    // ---- half a row per lane: maximum and scale (a first pass over the lane's values in shared memory) ...
+    const int t = lane & 15, hf = lane >> 4, half_vals = D / 2;                    // 64 or 32 values
+    const uint8_t *mine = in_rows + t * in_stride + hf * D;                        // (D bytes = D/2 bf16)
+    float amax = 0.f;
+    for (int i = 0; i < half_vals / 8; ++i) {
+        const uint4 q = *reinterpret_cast<const uint4 *>(mine + 16 * i);
+        amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16_lo(q.x)), fabsf(bf16_hi(q.x))), fmaxf(fabsf(bf16_lo(q.y)), fabsf(bf16_hi(q.y)))));
+        amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16_lo(q.z)), fabsf(bf16_hi(q.z))), fmaxf(fabsf(bf16_lo(q.w)), fabsf(bf16_hi(q.w)))));
+    }
+    amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 16));
+    const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+    if (hf == 0) *reinterpret_cast<float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * t) = __fdiv_rn(amax, 448.f);
+    // ... and the codes (a second pass), 16 values = one 16-byte piece of codes at a time
+    auto piece = [&](int j) -> uint4 {                                             // values 16j .. 16j+15 of the lane's half
+        const uint4 a = *reinterpret_cast<const uint4 *>(mine + 32 * j), b2 = *reinterpret_cast<const uint4 *>(mine + 32 * j + 16);
+        const uint32_t wv[8] = {a.x, a.y, a.z, a.w, b2.x, b2.y, b2.z, b2.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            o[i] = pack_e4m3x2(__fmul_rn(bf16_lo(wv[2 * i]), inv), __fmul_rn(bf16_hi(wv[2 * i]), inv)) |
+                   (pack_e4m3x2(__fmul_rn(bf16_lo(wv[2 * i + 1]), inv), __fmul_rn(bf16_hi(wv[2 * i + 1]), inv)) << 16);
+        return make_uint4(o[0], o[1], o[2], o[3]);
+    };
+    if (which == 0) {
+        // K: 16 dims of a token are one 16-byte piece of the page; the lane has half_vals / 16 of them
+        for (int j = 0; j < half_vals / 16; ++j)
+            *reinterpret_cast<uint4 *>(blk + fp8_k_pos(D, t, hf * half_vals + 16 * j)) = piece(j);
+        __syncwarp();                                                              // (in_rows is free again)
+        return;
+    }
+    // V: token-major codes into shared memory, dim-major pieces out
+    for (int j = 0; j < half_vals / 16; ++j) {
+        const uint4 o = piece(j);
+        uint32_t *dstw = reinterpret_cast<uint32_t *>(codes + t * code_stride + hf * half_vals + 16 * j);   // (4-byte aligned rows)
+        dstw[0] = o.x; dstw[1] = o.y; dstw[2] = o.z; dstw[3] = o.w;
+    }
+    __syncwarp();
+    for (int d = lane; d < D; d += 32) {
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            o[q] = (uint32_t)codes[(4 * q) * code_stride + d] | ((uint32_t)codes[(4 * q + 1) * code_stride + d] << 8) |
+                   ((uint32_t)codes[(4 * q + 2) * code_stride + d] << 16) | ((uint32_t)codes[(4 * q + 3) * code_stride + d] << 24);
+        *reinterpret_cast<uint4 *>(blk + fp8_v_off(D) + d * PAGE) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    __syncwarp();
+}
+
 // One row (token tok at offset off of its page) by one warp: scattered small stores (V is dim-major: one byte
 // in each of D rows; K: 4 bytes per lane).
 __device__ __forceinline__ void append_fp8_token(const AppendFp8Params &p, int64_t tok, int64_t page, int off, int h,
@@ -223,9 +371,14 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Param
 // the slots of its tokens and of the 15 tokens on either side, finds the whole page that starts inside its group
 // (at most one: its 16 tokens arrive together and in slot order), does that page 16 bytes per store, and does
 // its tokens that belong to no whole page one row at a time.  Same result as the kernel above for any slot map.
-__global__ void __launch_bounds__(COPY_THREADS) append_fp8_groups_kernel(AppendFp8Params p)
+constexpr int FP8_GROUP_WARPS = 7;
+constexpr int FP8_IN_BYTES = PAGE * (2 * 128 + 16), FP8_CODE_BYTES = PAGE * (128 + 4);     // per warp, head_dim <= 128
+
+__global__ void __launch_bounds__(FP8_GROUP_WARPS * 32, 3) append_fp8_groups_kernel(AppendFp8Params p)
 {
     pdl_trigger();
+    __shared__ __align__(16) uint8_t wide_in[FP8_GROUP_WARPS][FP8_IN_BYTES];
+    __shared__ __align__(16) uint8_t wide_codes[FP8_GROUP_WARPS][FP8_CODE_BYTES];
     constexpr unsigned ALL = 0xFFFFFFFFu;
     const int lane = threadIdx.x & 31;
     const int64_t n_groups = (p.n_tokens + PAGE - 1) / PAGE, n_items = n_groups * p.Hkv;
@@ -254,7 +407,8 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_groups_kernel(AppendF
         if (starts) {
             const int ls = __ffs(starts) - 1;
             const long long s0 = __shfl_sync(ALL, mine, ls);
-            append_fp8_page(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane);
+            append_fp8_page_wide(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane, wide_in[threadIdx.x >> 5],
+                                 wide_codes[threadIdx.x >> 5]);
         }
         for (unsigned m = loose; m; m &= m - 1) {
             const int lt = __ffs(m) - 1;
@@ -307,6 +461,13 @@ cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s)
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     if (n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
+    if (p.n_tokens >= 256) {                              // a prompt: rows read whole, pages written whole
+        const int64_t items = ((p.n_tokens + PAGE - 1) / PAGE) * p.Hkv;
+        int64_t ctas = (items + PAGE_WARPS - 1) / PAGE_WARPS;
+        if (ctas > 65535 * 4) ctas = 65535 * 4;           // (the warps loop over their items)
+        append_pages_kernel<<<dim3((unsigned)ctas, 2, (unsigned)n_layers), PAGE_WARPS * 32, 0, s>>>(p);
+        return cudaGetLastError();
+    }
     append_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), COPY_THREADS, 0, s>>>(p);
     return cudaGetLastError();
 }

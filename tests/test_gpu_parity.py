@@ -363,6 +363,71 @@ def test_non_owner_append_is_a_noop_and_null_inputs_are_fine():
         dw.cache.skv_append(0, None, None, dw.slot_new)       # an owner needs real K,V
 
 
+@pytest.mark.parametrize("D", [128, 64])
+@pytest.mark.parametrize("n_extra", [0, 700])     # below and above the size at which the page-granular update kernel takes over
+def test_update_with_arbitrary_slot_maps(n_extra, D):
+    """skv_append with slot maps that mix whole pages at odd positions of the call, pages in reverse order,
+    pages with a skipped token, scattered single slots, runs of whole pages and a ragged end: every written
+    slot reads back bit for bit, nothing else is touched, for both update kernels."""
+    from paper_2604_22782_b200 import harness
+    Hkv = 2
+    n_pages = 120
+    lens = torch.tensor([n_pages * 16], dtype=torch.int32)
+    w = W.Workload("slots", 1, 4, Hkv, D, 16, 1, 0, 0, "explicit", explicit_r=(0,), seed=113)
+    dw = harness.setup(w, lens=lens)
+    g = torch.Generator().manual_seed(17)
+    pages = torch.randperm(n_pages, generator=g).tolist()
+    page = lambda: pages.pop() * 16
+    parts = [torch.tensor([page() + 3, page() + 9, page()])]                       # three loose tokens first: pages start at odd positions
+    parts.append(page() + torch.arange(16))                                        # a whole page in order
+    parts.append(page() + torch.arange(15, -1, -1))                                # a page in reverse order
+    hole = page() + torch.arange(16); hole[5] = -1; parts.append(hole)             # a page with a skipped token
+    parts.append(torch.tensor([-1]))                                               # realign: whole pages on group boundaries from here
+    parts.append(torch.cat([page() + torch.arange(16) for _ in range(12)]))        # a run of whole pages
+    parts.append(torch.tensor([page() + i for i in (1, 15, 7)]))                   # loose tokens of one page
+    parts.append(page() + torch.arange(8))                                         # half a page
+    parts.append(torch.cat([page() + torch.arange(16) for _ in range(3)]))
+    if n_extra:
+        rest = torch.cat([page() + torch.arange(16) for _ in range(n_extra // 16)])
+        parts.append(rest[torch.randperm(rest.numel(), generator=g)][: n_extra // 2])    # scattered
+        pad = (-sum(x.numel() for x in parts)) % 16
+        parts.append(torch.full((pad,), -1))
+        parts.append(torch.cat([page() + torch.arange(16) for _ in range(20)]))    # whole pages on group boundaries
+        parts.append(page() + torch.arange(5))                                     # ragged end of the call
+    slots = torch.cat(parts).to(torch.int64)
+    n = slots.numel()
+    K = torch.randn((n, Hkv, D), generator=g).to(torch.bfloat16)
+    V = torch.randn((n, Hkv, D), generator=g).to(torch.bfloat16)
+    before = dw.cache.pool.clone()
+    dw.cache.skv_append(0, K.to(dw.device), V.to(dw.device), slots.to(dw.device))
+    torch.cuda.synchronize()
+    assert dw.cache.skv_get_status() == 0
+    keep = slots >= 0
+    Kg = torch.zeros((int(keep.sum()), Hkv, D), dtype=torch.bfloat16, device=dw.device)
+    Vg = torch.zeros_like(Kg)
+    dw.cache.skv_gather(0, slots[keep].to(dw.device), Kg, Vg)
+    torch.cuda.synchronize()
+    assert torch.equal(Kg.cpu().view(torch.int16), K[keep].view(torch.int16))
+    assert torch.equal(Vg.cpu().view(torch.int16), V[keep].view(torch.int16))
+    # nothing but the named slots changed: every other slot of the layer reads back as before (zeros)
+    others = torch.ones(n_pages * 16, dtype=torch.bool)
+    others[slots[keep]] = False
+    idx = torch.nonzero(others).flatten().to(dw.device)
+    Ko = torch.ones((idx.numel(), Hkv, D), dtype=torch.bfloat16, device=dw.device)
+    Vo = torch.ones_like(Ko)
+    dw.cache.skv_gather(0, idx, Ko, Vo)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(Ko.view(torch.int16)) == 0 and torch.count_nonzero(Vo.view(torch.int16)) == 0
+    assert torch.equal(before[:256], dw.cache.pool[:256])
+    # a slot past the pool in a large call is flagged and skipped
+    if n_extra:
+        from paper_2604_22782_b200.binding import SKV_ERR_BOUNDS
+        bad = slots.clone()
+        bad[40] = n_pages * 16 + 3
+        dw.cache.skv_append(0, K.to(dw.device), V.to(dw.device), bad.to(dw.device))
+        assert dw.cache.skv_get_status() == SKV_ERR_BOUNDS
+
+
 def test_out_of_range_ids_are_flagged_not_followed():
     """Bad slot / page ids raise the device status word; nothing is read or written out of bounds."""
     from paper_2604_22782_b200 import harness
