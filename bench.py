@@ -670,9 +670,19 @@ def prefill_leg(args, dev):
     torch.cuda.empty_cache()
     dq = harness.setup(w, device=dev, lens=lens, fp8=True)
     ms_append8 = timed(lambda: dq.cache.skv_append(0, K, V, slots))
+    st8 = dq.cache.skv_cache_stats()
     ms8 = timed(lambda: dq.cache.skv_prefill_attn(1, inp["Q"], inp["cu_q_lens"], dq.page_table, dq.seq_lens, out, T))
-    res["fp8_pages"] = {"append_ms": ms_append8, "ms_per_call": ms8, "tflops": flops / (ms8 * 1e-3) / 1e12,
-                        "tokens_per_s": B * T / (ms8 * 1e-3)}
+    res["fp8_pages"] = {"append_ms": ms_append8,
+                        "append_gbs": (K.numel() * 2 * 2 + st8["page_bytes"] * dq.total_pages) / (ms_append8 * 1e-3) / 1e9,
+                        "mma_sync": {"ms_per_call": ms8, "tflops": flops / (ms8 * 1e-3) / 1e12, "tokens_per_s": B * T / (ms8 * 1e-3)}}
+    # ... and with a scratch area: the pages turned into bf16 (one more launch, timed with the call), then the tcgen05 kernel
+    area = torch.empty(dq.cache.skv_prefill_scratch_bytes(), dtype=torch.uint8, device=dev)
+    dq.cache.skv_set_prefill_scratch(area)
+    ms8s = timed(lambda: dq.cache.skv_prefill_attn(1, inp["Q"], inp["cu_q_lens"], dq.page_table, dq.seq_lens, out, T))
+    res["fp8_pages"]["tcgen05_via_bf16_scratch"] = {"ms_per_call": ms8s, "tflops": flops / (ms8s * 1e-3) / 1e12,
+                                                    "tokens_per_s": B * T / (ms8s * 1e-3),
+                                                    "frac_of_bf16_tcgen05": res["tcgen05"]["ms_per_call"] / ms8s}
+    dq.cache.skv_set_prefill_scratch(None)
     if dq.cache.skv_get_status() != 0:
         raise SystemExit("device status after the FP8 pre-fill leg")
     return res

@@ -131,8 +131,9 @@ int skv_cache_create(skv_cache **out, int n_layers, const int32_t *r, int kv_hea
  * kind f8f6f4) on the stored codes, with the queries and the probabilities each
  * split into two E4M3 terms; at head_dim 64, or with skv_set_decode_variant(2),
  * the codes are converted to f16 on the way into mma.sync.  The pre-fill calls
- * run an mma.sync kernel that converts the codes the same way (prefill variant 2,
- * the tcgen05 kernel, reads bf16 pages only: SKV_ERR_UNSUPPORTED); skv_gather
+ * run an mma.sync kernel that converts the codes the same way, or, given a
+ * scratch area (skv_set_prefill_scratch), the tcgen05 kernel on a bf16 copy of
+ * the pages they reach (prefill variant 2 without one: SKV_ERR_UNSUPPORTED); skv_gather
  * returns SKV_ERR_UNSUPPORTED (use skv_gather_fp8).  Same arguments and errors
  * as skv_cache_pool_bytes / skv_cache_create. */
 int skv_cache_pool_bytes_fp8(int n_layers, const int32_t *r, int kv_heads, int head_dim,
@@ -310,6 +311,21 @@ int skv_prefill_attn(skv_cache *cache, int layer, const void *Q, const int32_t *
 int skv_prefill_attn_src(skv_cache *cache, int src_layer, const void *Q, const int32_t *cu_q_lens,
                          const int32_t *page_table, const int32_t *seq_lens, void *out, int batch,
                          int max_q_len, int q_heads, int pt_stride, float scale, void *stream);
+
+/* Pre-fill on an FP8 cache through the bf16 tensor-core kernel.  Given a scratch
+ * area of skv_prefill_scratch_bytes (room for the pages of ONE owner layer as
+ * bf16: max_pages * 2 * page_size * kv_heads * head_dim * 2 bytes; device,
+ * 256-byte aligned, the caller's, kept until it is taken back with NULL),
+ * skv_prefill_attn / skv_prefill_attn_src on an FP8 cache first turn the pages
+ * that the call's sequences reach back into bf16 (code value x the row's scale,
+ * rounded to nearest even) in that area -- one more launch, a pass over the
+ * pages that costs a few per cent of a prompt's attention -- and then run the
+ * tcgen05 kernel on it.  Without a scratch area (the default), or where that
+ * kernel does not apply, they run the mma.sync kernel that converts the codes on
+ * the way in.  Calls that use the area must not overlap on the GPU.
+ * skv_prefill_scratch_bytes gives 0 for a bf16 cache. */
+int skv_prefill_scratch_bytes(const skv_cache *cache, size_t *out_bytes);
+int skv_set_prefill_scratch(skv_cache *cache, void *device_scratch, size_t bytes);
 
 /* One whole decode step of Algorithm 2 with inputs already on the device:
  * for l = 0..L-1: append (owners only) then decode attention, on `stream`.

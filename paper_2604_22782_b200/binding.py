@@ -74,6 +74,8 @@ lib.skv_get_status.argtypes = [_vp, _vp, ctypes.POINTER(_int)]
 lib.skv_set_decode_variant.argtypes = [_vp, _int]
 lib.skv_set_decode_tuning.argtypes = [_vp, _int, _int, _int]
 lib.skv_set_prefill_variant.argtypes = [_vp, _int]
+lib.skv_prefill_scratch_bytes.argtypes = [_vp, _szp]
+lib.skv_set_prefill_scratch.argtypes = [_vp, _vp, _sz]
 lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
 lib.skv_set_decode_early_fetch.argtypes = [_vp, _int]
@@ -440,6 +442,19 @@ class SkvCache:
 
     def skv_set_decode_tuning(self, warps_per_cta: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
         _check(lib.skv_set_decode_tuning(self._h, warps_per_cta, stages, ctas_per_sm), "skv_set_decode_tuning")
+
+    def skv_prefill_scratch_bytes(self) -> int:
+        out = _sz(0)
+        _check(lib.skv_prefill_scratch_bytes(self._h, ctypes.byref(out)), "skv_prefill_scratch_bytes")
+        return out.value
+
+    def skv_set_prefill_scratch(self, scratch: Optional[torch.Tensor]) -> None:
+        """Give (or, with None, take back) the area in which pre-fill calls on an FP8 cache keep a bf16 copy of
+        the pages they reach; the tensor must stay alive while it is set."""
+        _arg("scratch", scratch, torch.uint8)
+        self._prefill_scratch = scratch
+        _check(lib.skv_set_prefill_scratch(self._h, _ptr(scratch), 0 if scratch is None else _nbytes(scratch)),
+               "skv_set_prefill_scratch")
 
     def skv_set_prefill_variant(self, variant: int) -> None:
         _check(lib.skv_set_prefill_variant(self._h, variant), "skv_set_prefill_variant")

@@ -56,6 +56,8 @@ struct skv_cache {
     DecodeTuning tune{0, 2, 2, 4, 1};
     bool fp8 = false;                // pages hold E4M3 codes + per-row scales instead of bf16
     int prefill_variant = 0;         // 0 auto (tcgen05 where supported), 1 mma.sync kernel, 2 tcgen05 kernel
+    uint8_t *prefill_scratch = nullptr;   // FP8 cache: room for one owner layer's pages as bf16 (caller's device memory)
+    size_t prefill_scratch_bytes = 0;
     bool shape_is_default = true;    // until skv_set_decode_tuning is called: the CUDA-core kernel runs as 1 x 2 x 8
     int l2_keep_pct = 35;            // > 0: consecutive layers that read one owner walk it in opposite directions
     bool early_fetch = false;        // stand-alone attention calls fill their rings before waiting for the kernel before them
@@ -828,8 +830,12 @@ int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens,
     if (!aligned(Q, 4) || !aligned(out, 4)) return SKV_ERR_ARG;
     if (batch > 65535 || c->kv_heads > 65535) return SKV_ERR_UNSUPPORTED;      // grid.y / grid.z limits
     const int G = q_heads / c->kv_heads;
-    // FP8 pages: the mma.sync kernel that converts the codes on the way in (the tcgen05 kernel reads bf16 pages)
-    const bool can_umma = !c->fp8 && prefill_umma_supported(c->head_dim, G) && aligned(Q, 16) && aligned(out, 16) &&
+    // FP8 pages: with a scratch area for one layer's pages as bf16, the pages the call reaches are converted
+    // there first and the tcgen05 kernel runs on the scratch; without one, the mma.sync kernel that converts
+    // the codes on the way in
+    const size_t bf16_page = page_bytes_of(c->kv_heads, c->head_dim, false);
+    const bool via_scratch = c->fp8 && c->prefill_scratch && c->prefill_scratch_bytes >= (size_t)c->max_pages * bf16_page;
+    const bool can_umma = (!c->fp8 || via_scratch) && prefill_umma_supported(c->head_dim, G) && aligned(Q, 16) && aligned(out, 16) &&
                           prefill_umma_smem_bytes(c->head_dim) <= (size_t)c->max_smem_optin;
     if (c->prefill_variant == 2 && !can_umma) return SKV_ERR_UNSUPPORTED;
     const bool umma = c->prefill_variant == 2 || (c->prefill_variant == 0 && can_umma);
@@ -855,6 +861,26 @@ int prefill_over(skv_cache *c, int src, const void *Q, const int32_t *cu_q_lens,
     const int tq = umma ? prefill_umma_tile_tokens(G) : prefill_tile_tokens(G);
     const int q_tiles = (max_q_len + tq - 1) / tq;
     const cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (umma && c->fp8) {
+        DequantParams dq;
+        dq.fp8_base = p.layer_base;
+        dq.bf16_base = c->prefill_scratch;
+        dq.fp8_page_stride = (int64_t)c->page_bytes;
+        dq.bf16_page_stride = (int64_t)bf16_page;
+        dq.max_pages = c->max_pages;
+        dq.page_table = page_table;
+        dq.seq_lens = seq_lens;
+        dq.B = batch;
+        dq.Hkv = c->kv_heads;
+        dq.pt_stride = pt_stride;
+        if (launch_dequant_pages(dq, c->head_dim, pt_stride, st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SKV_ERR_CUDA;
+        }
+        c->launches += 1;
+        p.layer_base = c->prefill_scratch;
+        p.page_stride = (int64_t)bf16_page;
+    }
     const cudaError_t le = umma     ? launch_prefill_umma(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st)
                            : c->fp8 ? launch_prefill_fp8(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st)
                                     : launch_prefill(p, c->head_dim, G, q_tiles, c->tune.pdl != 0, st);
@@ -1056,6 +1082,21 @@ int skv_set_decode_tuning(skv_cache *c, int warps_per_cta, int stages, int ctas_
     }
     c->tune = t;
     c->shape_is_default = false;
+    return SKV_OK;
+}
+
+int skv_prefill_scratch_bytes(const skv_cache *c, size_t *out_bytes)
+{
+    if (!c || !out_bytes) return SKV_ERR_ARG;
+    *out_bytes = c->fp8 ? (size_t)c->max_pages * page_bytes_of(c->kv_heads, c->head_dim, false) : 0;
+    return SKV_OK;
+}
+
+int skv_set_prefill_scratch(skv_cache *c, void *device_scratch, size_t bytes)
+{
+    if (!c || (device_scratch && !aligned(device_scratch, 256))) return SKV_ERR_ARG;
+    c->prefill_scratch = static_cast<uint8_t *>(device_scratch);
+    c->prefill_scratch_bytes = device_scratch ? bytes : 0;
     return SKV_OK;
 }
 

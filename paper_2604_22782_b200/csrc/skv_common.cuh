@@ -155,6 +155,16 @@ struct PrefillParams {
     int *status;
 };
 
+struct DequantParams {
+    const uint8_t *fp8_base;    // first page of the FP8 owner layer
+    uint8_t *bf16_base;         // scratch: the same pages in the bf16 layout
+    int64_t fp8_page_stride, bf16_page_stride;
+    int64_t max_pages;
+    const int32_t *page_table;  // [B][pt_stride]
+    const int32_t *seq_lens;    // [B]
+    int B, Hkv, pt_stride;
+};
+
 struct DecodeTuning {
     int variant;                // 0 auto, 1 CUDA-core (G=1), 2 tensor-core
     int warps;                  // per CTA
@@ -184,6 +194,8 @@ cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, bool fp8);
 cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,
                               bool pdl, cudaStream_t s);
+// FP8 pages of the sequences' pages -> bf16 pages in a scratch area (skv_dequant.cu); grid covers max_pages_per_seq
+cudaError_t launch_dequant_pages(const DequantParams &p, int D, int max_pages_per_seq, cudaStream_t s);
 size_t prefill_smem_bytes(int D);
 size_t prefill_fp8_smem_bytes(int D);
 cudaError_t launch_prefill_fp8(const PrefillParams &p, int D, int G, int q_tiles, bool pdl, cudaStream_t s);
