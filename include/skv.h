@@ -412,7 +412,7 @@ int skv_set_decode_overlap(skv_cache *cache, int enabled);
  * (skv_decode_attn, skv_decode_attn_static; the two-call form skv_decode_splitk +
  * skv_decode_merge and the chained launches of skv_decode_step always use warps).
  *   mode 0 (default) or 2: CTAs that own a range each -- `consumers` warps
- *        (1..12; 0 keeps the current value) share one ring of `stages` stages of
+ *        (1..8; 0 keeps the current value) share one ring of `stages` stages of
  *        one (page, kv head) block (2..26; 0, the default: as many as fit, at
  *        most 20 per SM) filled by a producer warp, take its blocks in turn and
  *        combine their running states in shared memory at the end of every

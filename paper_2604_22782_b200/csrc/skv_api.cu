@@ -1123,7 +1123,7 @@ int skv_set_decode_early_fetch(skv_cache *c, int enabled)
 
 int skv_set_decode_worker(skv_cache *c, int mode, int consumers, int stages, int ctas_per_sm)
 {
-    if (!c || mode < 0 || mode > 3 || consumers < 0 || consumers > 12 || stages < 0 || stages == 1 || stages > 26 ||
+    if (!c || mode < 0 || mode > 3 || consumers < 0 || consumers > 8 || stages < 0 || stages == 1 || stages > 26 ||
         ctas_per_sm < 0 || ctas_per_sm > 4)
         return SKV_ERR_ARG;
     c->cta_in_turn = mode != 3;

@@ -22,7 +22,7 @@ namespace skv {
 
 namespace {
 
-constexpr int MAX_CONSUMERS = 12;
+constexpr int MAX_CONSUMERS = 8;      // (+ the producer: 288 threads, which the register budget is set for)
 
 // floats of one consumer's state in the scratch: out [G][D], then (max, sum) [G][2], rounded up to 16 bytes
 // (the states are written with 16-byte stores)
@@ -83,12 +83,22 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 }
 
 // Shared memory: tables (prefix, lens) | ring [S][BLOCK] | scratch [2][C] x ([G][D] fp32 out + [G][2] (max, sum))
-//                | full[S], empty[S], run_done[2] mbarriers | gave_up word, claim counter | issued[S]
-// The scratch is double-buffered by run parity: a consumer writes buffer r&1 at the end of run r, and it can
-// only get to the end of run r+2 after every consumer has arrived at the barrier of run r+1, i.e. after
-// every consumer has finished reading buffer r&1.
+//                | query rows [2][G][D] bf16 | full[S], empty[S], run_done[2], q_full[2] mbarriers
+//                | gave_up word, claim counter, q_taken[2] | issued[S]
+// A RUN is the part of the CTA's range inside one (sequence, kv head) segment.  What a run costs beyond its
+// blocks is kept off the consumers' path, because a range holds two to five of them and the slowest CTA sets
+// the end of the launch:
+//   - the run's query rows are brought into shared memory by the producer, ahead of the run's first block
+//     (two buffers by run parity; q_full: the rows have landed; q_taken: how many consumers have taken their
+//     copy of a buffer's rows so far, a plain count that runs on, because the producer lanes that refill the
+//     buffer do not see every phase a barrier would go through);
+//   - at the end of run r a consumer writes its state to scratch buffer r&1 and goes straight on with run
+//     r+1; the states of run r are combined at the end of run r+1, when they have long been complete.
+// Order at the end of run r: wait for run r-1 to be complete and combine it, THEN write the state of run r
+// and arrive for run r.  So a consumer that writes scratch buffer r&1 has passed the barrier of run r-1,
+// which every consumer arrives at only after it has combined run r-2, the last reader of that buffer.
 template <int D, class State>
-__global__ void decode_cta_kernel(DecodeParams p, int G, int S)
+__global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode_cta_kernel(DecodeParams p, int G, int S)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = State::BLOCK;
@@ -105,19 +115,35 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
     const size_t scratch_off = ring_off + (size_t)S * BLOCK;
     const int part_floats = cta_part_floats(G, D);     // one consumer's state: out [G][D], then (max, sum) [G][2]
     float *scratch = reinterpret_cast<float *>(smem_raw + scratch_off);
-    const size_t bars_off = scratch_off + (((size_t)2 * C * part_floats * 4 + 15) & ~(size_t)15);
+    const size_t q_off = scratch_off + (((size_t)2 * C * part_floats * 4 + 15) & ~(size_t)15);
+    const int q_bytes = G * D * 2;                     // the query rows of one kv head: a multiple of 128 bytes
+    const uint16_t *q_rows = reinterpret_cast<const uint16_t *>(smem_raw + q_off);
+    const size_t bars_off = q_off + 2 * (size_t)q_bytes;
     const uint32_t full = base + (uint32_t)bars_off, empty = full + 8u * S, run_done = empty + 8u * S;
-    volatile int *gave_up = reinterpret_cast<volatile int *>(smem_raw + bars_off + 16 * (size_t)S + 16);
+    const uint32_t q_full = run_done + 16;
+    volatile int *gave_up = reinterpret_cast<volatile int *>(smem_raw + bars_off + 16 * (size_t)S + 32);
     int *next_claim = const_cast<int *>(gave_up) + 1;
-    const uint32_t issued_at = run_done + 16 + 8;       // int [S]
+    volatile int *q_taken = gave_up + 2;                // [2]: consumers that have taken their copy of a buffer's rows, ever
+    const uint32_t issued_at = q_full + 16 + 16;        // int [S]
 
+    {   // the layout above must fit the shared memory the launch was given (else: flag it and do nothing)
+        uint32_t given;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(given));
+        if (issued_at - base + 4u * (uint32_t)S > given) {
+            if (threadIdx.x == 0) atomicOr(p.status, STATUS_BOUNDS);
+            return;
+        }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(full + 8 * s, 1);
             mbar_init(empty + 8 * s, 1);
         }
-        mbar_init(run_done, C);
-        mbar_init(run_done + 8, C);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(run_done + 8 * i, C);
+            mbar_init(q_full + 8 * i, 1);
+            q_taken[i] = 0;
+        }
         gave_up[0] = 0;
         *next_claim = 0;
         for (int s = 0; s < S; ++s) publish_issued(issued_at + 4 * s, -1);
@@ -146,51 +172,89 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
         // L2 that must not sit between two batches of copies), then issues the block's copy itself.  Within
         // a group the copies go out PB lanes at a time, in order (one thread alone cannot issue bulk copies
         // fast enough for an SM's share of the bandwidth; and never two blocks of one batch in one stage).
+        // The lane whose block opens a run first sends for the run's query rows.
         const int PB = S < 8 ? S : 8;
         const uint64_t pol_stream = make_policy_evict_first(), pol_keep = make_policy_evict_normal();
         const int keep_from = (p.keep_pct > 0 && T <= p.l2_fit_blocks) ? 0 : n - (int)(((int64_t)n * p.keep_pct) / 100);
         bool waited = !early_fetch, triggered = false, quit = false;
-        // This lane's block of a group: kv head, raw page id (checked and turned into an address only when the
-        // group's copies go out, so that the load stays in flight meanwhile; -1 past the end of the range),
-        // and whether the block is the last page of its sequence.
-        auto look_up = [&](int kk, int &id, int &h, bool &last_page) {
-            id = -1;
-            h = 0;
-            last_page = false;
-            if (kk >= n) return;
+        // This lane's block of a group: sequence and kv head, raw page id (checked and turned into an address
+        // only when the group's copies go out, so that the load stays in flight meanwhile; -1 past the end of
+        // the range), whether the block is the last page of its sequence, whether it opens a run.
+        struct Look { int id, b, h; bool last_page, opens; };
+        auto look_up = [&](int kk) -> Look {
+            Look r = {-1, 0, 0, false, false};
+            if (kk >= n) return r;
             const Cursor cur = locate(prefix, p.B, p.Hkv, reverse ? x_first - kk : x_first + kk);
-            id = __ldg(p.page_table + (int64_t)cur.b * p.pt_stride + cur.pg);
-            h = cur.h;
-            last_page = cur.pg + 1 == cur.pages;
+            r.id = __ldg(p.page_table + (int64_t)cur.b * p.pt_stride + cur.pg);
+            r.b = cur.b;
+            r.h = cur.h;
+            r.last_page = cur.pg + 1 == cur.pages;
+            r.opens = kk == 0 || (reverse ? cur.pg + 1 == cur.pages : cur.pg == 0);
+            return r;
         };
-        int id = -1, h = 0, id_next = -1, h_next = 0;
-        bool last_page = false, last_next = false;
-        look_up(lane, id, h, last_page);
+        // The first run's query rows go out before anything else (unless early fetch holds them back until the
+        // wait): the consumers start on them while this warp is still looking up its first page ids.
+        Look cur = look_up(lane), nxt;                  // (the page ids first: they are the longest chain to the first block)
+        bool first_rows_sent = false;
+        if (n > 0 && waited) {
+            if (lane == 0) {
+                mbar_expect_tx(q_full, (uint32_t)q_bytes);
+                bulk_copy_g2s(base + (uint32_t)q_off, p.Q + ((int64_t)cur.b * p.Hq + (int64_t)cur.h * G) * D, (uint32_t)q_bytes, q_full);
+            }
+            first_rows_sent = true;
+        }
+        int runs_before = 0;                            // runs opened in earlier groups
         int k = 0;                                      // first block of the current group
         for (; k < n && !quit; k += 32) {
             const int kk = k + lane;
+            int id = cur.id;
             if (kk < n && (id < 0 || (int64_t)id >= p.max_pages)) {
                 atomicOr(p.status, STATUS_BOUNDS);
                 id = 0;
             }
-            const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)h * BLOCK;
-            look_up(k + 32 + lane, id_next, h_next, last_next);
+            const uint8_t *src = p.layer_base + (int64_t)id * p.page_stride + (int64_t)cur.h * BLOCK;
+            const unsigned openers = __ballot_sync(FULL, cur.opens);
+            const int my_run = runs_before + __popc(openers & ((2u << lane) - 1u)) - 1;     // (for a lane that opens one)
+            bool q_pending = false;                      // this lane's block opened a run whose query rows are not sent for yet
+            auto send_for_rows = [&]() {
+                // The rows of run r go into buffer r&1 once every consumer has taken its copy of run r-2's (C times
+                // r/2 copies of that buffer taken in all).  All lanes stay in this loop together and each sends
+                // when its turn has come: a lane that left early would stand between a later lane and its turn.
+                if (!__any_sync(FULL, q_pending)) return true;
+                const int qb = my_run & 1, need = C * (my_run / 2);
+                const uint64_t t0 = global_timer_ns();
+                bool ok = true;
+                while (__any_sync(FULL, q_pending)) {
+                    if (q_pending && q_taken[qb] >= need) {
+                        mbar_expect_tx(q_full + 8 * qb, (uint32_t)q_bytes);
+                        bulk_copy_g2s(base + (uint32_t)q_off + (uint32_t)(qb * q_bytes),
+                                      p.Q + ((int64_t)cur.b * p.Hq + (int64_t)cur.h * G) * D, (uint32_t)q_bytes, q_full + 8 * qb);
+                        q_pending = false;
+                    }
+                    if (!__any_sync(FULL, q_pending)) break;
+                    if (gave_up[0] || global_timer_ns() - t0 > 2000000000ull) {
+                        ok = false;
+                        break;
+                    }
+                }
+                return ok;
+            };
             for (int j0 = 0; j0 < 32 && k + j0 < n && !quit; j0 += PB) {
                 const bool active = lane >= j0 && lane < j0 + PB && kk < n;
                 // With early fetch the ring is filled before the wait on the kernel before this one, but
                 // never with a sequence's last page (its newest token may be on its way), and the wait is
-                // taken at the latest when the ring has been filled once.
-                if (!waited && (k + j0 + PB > S || __any_sync(FULL, active && last_page))) {
+                // taken at the latest when the ring has been filled once.  Query rows are sent for after it.
+                bool ok = true;
+                if (!waited && (k + j0 + PB > S || k + j0 >= n / 2 || __any_sync(FULL, active && cur.last_page))) {
                     pdl_wait();
                     waited = true;
+                    ok = send_for_rows();              // the rows held back so far, before any copy below waits for a stage
                 }
                 if (!triggered && k + j0 >= n / 2) {   // the merge kernel may move in from here on
                     triggered = true;
-                    if (!waited) { pdl_wait(); waited = true; }
                     pdl_trigger();
                 }
-                bool ok = true;
-                if (active) {
+                if (ok && active) {
                     const int s = kk % S;
                     if (kk >= S) ok = wait_or_quit(empty + 8 * s, (uint32_t)((kk / S - 1) & 1), gave_up);
                     if (ok) {
@@ -198,26 +262,36 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
                         publish_issued(issued_at + 4 * s, kk);
                         bulk_copy_g2s_hint(ring + (uint32_t)(s * BLOCK), src, BLOCK, full + 8 * s, kk >= keep_from ? pol_keep : pol_stream);
                     }
+                    if (cur.opens && !(kk == 0 && first_rows_sent)) q_pending = true;
                 }
-                if (!__all_sync(FULL, ok)) {
+                if (j0 == 0) nxt = look_up(k + 32 + lane);   // (after the group's first copies have gone out)
+                ok = __all_sync(FULL, ok);
+                if (ok && waited) ok = send_for_rows();  // (all of the group's blocks so far are out: nobody waits for one of them)
+                if (!ok) {
                     if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
                     quit = true;
                 }
             }
-            id = id_next;
-            h = h_next;
-            last_page = last_next;
+            if (!quit && __any_sync(FULL, q_pending)) {   // rows held back by early fetch: the range ends inside the first ring fill
+                if (!waited) { pdl_wait(); waited = true; }
+                if (!send_for_rows()) {
+                    if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+                    quit = true;
+                }
+            }
+            runs_before += __popc(openers);
+            cur = nxt;
         }
         if (!waited) pdl_wait();
         if (!triggered) pdl_trigger();
         // Leave only when every copy that was issued has landed: the ring must not be written after the CTA
         // is gone.  (Normally the consumers have seen them all long ago; after a failure they may not have.)
-        // (after a failure some lanes of the last batch may not have issued: those stages' phases were
-        // completed by earlier copies or never armed, and the waits below return at once or at the limit)
         const int issued = k < n ? k : n;
         const uint64_t deadline = global_timer_ns() + 2000000000ull;
         for (int j = issued > S ? issued - S : 0; j < issued; ++j)
             if (!wait_until(full + 8 * (j % S), (uint32_t)((j / S) & 1), deadline)) break;
+        for (int r = runs_before > 2 ? runs_before - 2 : 0; r < runs_before; ++r)
+            if (!wait_until(q_full + 8 * (r & 1), (uint32_t)((r / 2) & 1), deadline)) break;
         return;
     }
 
@@ -228,11 +302,6 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
     if (blockIdx.x == 0)
         for (int i = threadIdx.x; i <= p.B; i += C * 32) p.prefix[i] = prefix[i];
 
-    Cursor cons = {0, 0, 0, 1};
-    if (n > 0) cons = locate(prefix, p.B, p.Hkv, x_first);
-    uint64_t t_first = 0;
-    int k = 0, run = 0;
-    int held = -1;                                     // a block of the range this consumer has claimed and not done yet
     // Dynamic: whoever is free takes the next block (the consumers of an SM end together, but which blocks a
     // consumer sums, and with that the last bits of the result, vary from run to run).  In turn: block j
     // goes to consumer j mod C (reproducible bit for bit).
@@ -251,24 +320,68 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
         if (lane == 0) j = atomicAdd(next_claim, 1);
         return __shfl_sync(FULL, j, 0);
     };
-    bool failed = false;
+    // the states of run `r` (all consumers', in scratch buffer r&1) -> the segment's rows, or its partial at `slot`
+    auto combine = [&](int r, int b, int h, bool whole, int slot) {
+        const float *buf = scratch + (size_t)(r & 1) * C * part_floats;
+        for (int e2 = (int)threadIdx.x; e2 < G * D / 2; e2 += C * 32) {       // thread t takes output pairs t, t + 32C, ...
+            const int g = (2 * e2) / D;
+            float M = -INFINITY;
+            for (int c = 0; c < C; ++c) M = fmaxf(M, buf[c * part_floats + G * D + 2 * g]);
+            float L = 0.f, a0 = 0.f, a1 = 0.f;
+            for (int c = 0; c < C; ++c) {
+                const float *sc = buf + c * part_floats;
+                const float m_c = sc[G * D + 2 * g];
+                if (m_c == -INFINITY) continue;         // this consumer had no block in the run
+                const float wt = fast_exp2(m_c - M);
+                L = fmaf(wt, sc[G * D + 2 * g + 1], L);
+                const float2 v = *reinterpret_cast<const float2 *>(sc + 2 * e2);
+                a0 = fmaf(wt, v.x, a0);
+                a1 = fmaf(wt, v.y, a1);
+            }
+            if (whole) {
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)h * G) * D);
+                dst[e2] = pack_bf16x2(a0 * inv, a1 * inv);
+            } else {
+                *reinterpret_cast<float2 *>(p.part_o + (int64_t)slot * G * D + 2 * e2) = make_float2(a0, a1);
+                if ((2 * e2) % D == 0) *reinterpret_cast<float2 *>(p.part_ml + ((int64_t)slot * G + g) * 2) = make_float2(M, L);
+            }
+        }
+    };
+
+    Cursor cons = {0, 0, 0, 1};
+    if (n > 0) cons = locate(prefix, p.B, p.Hkv, x_first);
+    uint64_t t_first = 0;
+    int k = 0, run = 0;
+    int held = -1;                                     // a block of the range this consumer has claimed and not done yet
+    int prev_b = 0, prev_h = 0, prev_slot = 0;         // the run before this one, not yet combined
+    bool prev_whole = false, failed = false;
+    auto fail = [&]() {
+        if (lane == 0 && !gave_up[0]) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+        failed = true;
+    };
     while (k < n && !failed) {
         // one run: blocks [k, k + len) of the range, all of segment (b, h)
         const int b = cons.b, h = cons.h, pages = cons.pages, n_b = lens[b];
         const int to_edge = reverse ? cons.pg + 1 : pages - cons.pg;           // blocks left in this segment
         const int len = to_edge < n - k ? to_edge : n - k;
-        const bool whole = len == pages;                                       // the segment lies inside this range
-        float *mine = scratch + ((size_t)(run & 1) * C + warp) * part_floats;
+        const int qb = run & 1;
+        float *mine = scratch + ((size_t)qb * C + warp) * part_floats;
         if (held < 0) held = claim();
-        if (held < k + len) {
+        const bool has_blocks = held < k + len;
+        {
             State st;
-            st.begin(p, b, h, G, lane);
-            do {
+            if (has_blocks) {
+                if (!wait_or_quit(q_full + 8 * qb, (uint32_t)((run >> 1) & 1), gave_up)) { fail(); break; }
+                st.begin_rows(q_rows + (size_t)qb * G * D, G, lane);
+            }
+            __syncwarp();
+            if (lane == 0) atomicAdd(const_cast<int *>(q_taken) + qb, 1);       // (with or without a copy taken)
+            while (has_blocks && held < k + len) {
                 const int j = held, s = j % S;
                 if ((ask_issued && !wait_issued(issued_at + 4 * s, j, gave_up, lane)) ||
                     !wait_or_quit(full + 8 * s, (uint32_t)((j / S) & 1), gave_up)) {
-                    if (lane == 0) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
-                    failed = true;
+                    fail();
                     break;
                 }
                 if (p.trace && t_first == 0) t_first = global_timer_ns();
@@ -278,54 +391,34 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
                 __syncwarp();                           // every lane is done reading this stage
                 if (lane == 0) mbar_arrive(empty + 8 * s);
                 held = claim();
-            } while (held < k + len);
-            if (!failed) st.finish(mine, mine + G * D, 0, G, lane);
-        } else if (lane < G) {
-            mine[G * D + 2 * lane] = -INFINITY;         // no block of this run: nothing to contribute
-        }
-        // all consumers' states of this run are in shared memory
-        __syncwarp();
-        if (lane == 0) mbar_arrive(run_done + 8 * (run & 1));
-        if (failed || !wait_or_quit(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1), gave_up)) {
-            if (lane == 0 && !failed) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
-            failed = true;
-            break;
-        }
-        // combine: thread t takes output pairs e2 = t, t + 32C, ... of the G*D/2 pairs
-        {
-            const int slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
-            for (int e2 = (int)threadIdx.x; e2 < G * D / 2; e2 += C * 32) {
-                const int g = (2 * e2) / D;
-                float M = -INFINITY;
-                const float *buf = scratch + (size_t)(run & 1) * C * part_floats;
-                for (int c = 0; c < C; ++c) M = fmaxf(M, buf[c * part_floats + G * D + 2 * g]);
-                float L = 0.f, a0 = 0.f, a1 = 0.f;
-                for (int c = 0; c < C; ++c) {
-                    const float *sc = buf + c * part_floats;
-                    const float m_c = sc[G * D + 2 * g];
-                    if (m_c == -INFINITY) continue;     // this consumer had no block in the run
-                    const float wt = fast_exp2(m_c - M);
-                    L = fmaf(wt, sc[G * D + 2 * g + 1], L);
-                    const float2 v = *reinterpret_cast<const float2 *>(sc + 2 * e2);
-                    a0 = fmaf(wt, v.x, a0);
-                    a1 = fmaf(wt, v.y, a1);
-                }
-                if (whole) {
-                    const float inv = L > 0.f ? 1.f / L : 0.f;
-                    uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)h * G) * D);
-                    dst[e2] = pack_bf16x2(a0 * inv, a1 * inv);
-                } else {
-                    *reinterpret_cast<float2 *>(p.part_o + (int64_t)slot * G * D + 2 * e2) = make_float2(a0, a1);
-                    if ((2 * e2) % D == 0) *reinterpret_cast<float2 *>(p.part_ml + ((int64_t)slot * G + g) * 2) = make_float2(M, L);
-                }
             }
+            if (failed) break;
+            // the run before this one has long been complete: combine it, then hand in this run's state
+            if (run > 0) {
+                if (!wait_or_quit(run_done + 8 * (qb ^ 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up)) { fail(); break; }
+                combine(run - 1, prev_b, prev_h, prev_whole, prev_slot);
+            }
+            if (has_blocks) st.finish(mine, mine + G * D, 0, G, lane);
+            else if (lane < G) mine[G * D + 2 * lane] = -INFINITY;             // no block of this run: nothing to contribute
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(run_done + 8 * qb);
+        prev_b = b;
+        prev_h = h;
+        prev_whole = len == pages;                                             // the segment lies inside this range
+        prev_slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
         k += len;
         ++run;
         if (k < n) {                                   // first block of the next run
             cons.pg = reverse ? cons.pg - (len - 1) : cons.pg + (len - 1);
             step(cons, prefix, p.Hkv, reverse);
         }
+    }
+    if (!failed && run > 0) {
+        if (wait_or_quit(run_done + 8 * ((run - 1) & 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up))
+            combine(run - 1, prev_b, prev_h, prev_whole, prev_slot);
+        else
+            fail();
     }
     if (p.trace && lane == 0) {
         unsigned smid;
@@ -338,6 +431,7 @@ __global__ void decode_cta_kernel(DecodeParams p, int G, int S)
 template <int D, class State>
 cudaError_t launch_cta_t(const DecodeParams &p, int G, int grid, int consumers, int stages, bool pdl, cudaStream_t s)
 {
+    if (consumers > State::MAX_CTA_CONSUMERS) consumers = State::MAX_CTA_CONSUMERS;      // (what its registers allow)
     const size_t smem = decode_cta_smem_bytes(D, p.B, G, consumers, stages, State::BLOCK != block_bytes(D));
     auto kern = decode_cta_kernel<D, State>;
     cudaError_t e = ensure_dynamic_smem(kern, smem);
@@ -364,8 +458,9 @@ size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, boo
     const size_t blk = fp8 ? fp8_block_bytes(D) : block_bytes(D);
     const size_t scratch = (((size_t)2 * consumers * cta_part_floats(G, D) * 4) + 15) & ~(size_t)15;
     // 128 bytes of slack for aligning the ring base; barriers: full, empty per stage, two run barriers; two words
-    // ... and the issued-block word of every stage
-    return 128 + table_bytes(B) + (size_t)stages * blk + scratch + 16 * (size_t)stages + 16 + 16 + 4 * (size_t)stages + 16;
+    // ... the query rows of two runs, their barriers, and the issued-block word of every stage
+    return 128 + table_bytes(B) + (size_t)stages * blk + scratch + 2 * (size_t)G * D * 2 + 16 * (size_t)stages + 32 + 16 +
+           4 * (size_t)stages + 16;
 }
 
 cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,

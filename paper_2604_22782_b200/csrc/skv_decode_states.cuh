@@ -24,6 +24,7 @@ constexpr int WIN = 128;   // page ids a warp keeps in registers (4 per lane)
 template <int D>
 struct TensorCoreState {
     static constexpr int BLOCK = block_bytes(D);   // bytes of one (page, kv head) block
+    static constexpr int MAX_CTA_CONSUMERS = 8;    // consumer warps of the CTA-per-range kernel that the registers allow
     static constexpr int KS = D / 16;   // k-steps of QK^T, and pairs of 8-dim tiles of PV
     uint32_t qa[KS][2];
     float o[D / 8][4];
@@ -31,12 +32,18 @@ struct TensorCoreState {
 
     __device__ __forceinline__ void begin(const DecodeParams &p, int b, int h, int G, int lane)
     {
+        begin_rows(p.Q + ((int64_t)b * p.Hq + (int64_t)h * G) * D, G, lane);
+    }
+
+    // rows: the G query rows [G][D] of the kv head (global or shared memory)
+    __device__ __forceinline__ void begin_rows(const uint16_t *rows, int G, int lane)
+    {
         const int g = lane >> 2, tig = lane & 3;
-        const uint16_t *q = p.Q + ((int64_t)b * p.Hq + (int64_t)h * G + g) * D + 2 * tig;
+        const uint16_t *q = rows + g * D + 2 * tig;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            qa[ks][0] = (g < G) ? __ldg(reinterpret_cast<const unsigned int *>(q + 16 * ks)) : 0u;
-            qa[ks][1] = (g < G) ? __ldg(reinterpret_cast<const unsigned int *>(q + 16 * ks + 8)) : 0u;
+            qa[ks][0] = (g < G) ? *reinterpret_cast<const unsigned int *>(q + 16 * ks) : 0u;
+            qa[ks][1] = (g < G) ? *reinterpret_cast<const unsigned int *>(q + 16 * ks + 8) : 0u;
         }
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
@@ -127,18 +134,24 @@ struct TensorCoreState {
 template <int D>
 struct CudaCoreState {
     static constexpr int BLOCK = block_bytes(D);
+    static constexpr int MAX_CTA_CONSUMERS = D > 64 ? 7 : 8;   // (64 query and 64 output values per lane at head_dim 128)
     static constexpr int HC = D / 16;   // 16-byte chunks per dim half
     float q[D / 2];
     float o[D / 2];
     float m, l;
 
-    __device__ __forceinline__ void begin(const DecodeParams &p, int b, int h, int /*G*/, int lane)
+    __device__ __forceinline__ void begin(const DecodeParams &p, int b, int h, int G, int lane)
+    {
+        begin_rows(p.Q + ((int64_t)b * p.Hq + h) * D, G, lane);
+    }
+
+    __device__ __forceinline__ void begin_rows(const uint16_t *rows, int /*G*/, int lane)
     {
         const int hf = lane >> 4;
-        const uint16_t *qp = p.Q + ((int64_t)b * p.Hq + h) * D + hf * (D / 2);
+        const uint16_t *qp = rows + hf * (D / 2);
 #pragma unroll
         for (int c = 0; c < HC; ++c) {
-            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(qp) + c);
+            const uint4 w = *(reinterpret_cast<const uint4 *>(qp) + c);
             q[c * 8 + 0] = bf16_lo(w.x); q[c * 8 + 1] = bf16_hi(w.x);
             q[c * 8 + 2] = bf16_lo(w.y); q[c * 8 + 3] = bf16_hi(w.y);
             q[c * 8 + 4] = bf16_lo(w.z); q[c * 8 + 5] = bf16_hi(w.z);
@@ -248,6 +261,7 @@ struct CudaCoreState {
 template <int D>
 struct Fp8State {
     static constexpr int BLOCK = fp8_block_bytes(D);
+    static constexpr int MAX_CTA_CONSUMERS = 8;
     static constexpr int KS = D / 16;
     static constexpr int DT = D / 4;    // dims per thread of a quad
     uint32_t qa[KS][2];                 // f16x2: dims DT*tig + 4ks + {0,1} and + {2,3} of Q / qmax
@@ -256,14 +270,19 @@ struct Fp8State {
 
     __device__ __forceinline__ void begin(const DecodeParams &p, int b, int h, int G, int lane)
     {
+        begin_rows(p.Q + ((int64_t)b * p.Hq + (int64_t)h * G) * D, G, lane);
+    }
+
+    __device__ __forceinline__ void begin_rows(const uint16_t *rows, int G, int lane)
+    {
         const int g = lane >> 2, tig = lane & 3;
         float q[DT];
         float amax = 0.f;
         if (g < G) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + ((int64_t)b * p.Hq + (int64_t)h * G + g) * D + DT * tig);
+            const uint4 *src = reinterpret_cast<const uint4 *>(rows + g * D + DT * tig);
 #pragma unroll
             for (int c = 0; c < DT / 8; ++c) {
-                const uint4 w = __ldg(src + c);
+                const uint4 w = src[c];
                 q[8 * c + 0] = bf16_lo(w.x); q[8 * c + 1] = bf16_hi(w.x);
                 q[8 * c + 2] = bf16_lo(w.y); q[8 * c + 3] = bf16_hi(w.y);
                 q[8 * c + 4] = bf16_lo(w.z); q[8 * c + 5] = bf16_hi(w.z);
