@@ -39,9 +39,10 @@ METRIC = "decode_attn_hbm_gbs"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel,
-# from the ncu capture summarised under profiles/ (None until captured)
-NCU_TRAFFIC_BYTES = {"llama3_8b": 343470000}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel of a stand-alone attention
+# call (decode_cta_kernel), mean of the two launches of the ncu capture summarised in
+# profiles/decode_cta_llama3_8b.md (taken on the two-layer form of the workload, which issues the same call)
+NCU_TRAFFIC_BYTES = {"llama3_8b": 343256000, "llama3_8b_2layers": 343256000}
 DEFAULT_L2_KEEP = 35     # the library's default share of each block range kept in L2 for the next layer
 
 
@@ -415,6 +416,9 @@ def main():
         return {"us_per_call": us, "gbs": g, "frac": g / peak, "frac_of_nominal_8TBs": g / NOMINAL_HBM_GBS,
                 **spread_of(leg, K)}
 
+    worker_mode = int(args.worker.split(",")[0]) if args.worker else 0
+    kernel_name = ("decode_fp8_umma_kernel" if (args.fp8 and w.head_dim == 128 and args.variant != 2)
+                   else "decode_splitk_kernel" if worker_mode == 1 else "decode_cta_kernel")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": leg_main["ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -435,7 +439,7 @@ def main():
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "clocks": all_clocks,
         "gpu_launches": int(launches) * K,
-        "roofline": {"bound": "hbm", "kernel": "decode_splitk_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "us_per_launch": us_per_launch,
                      "bytes_per_launch": attn_bytes,
@@ -443,7 +447,7 @@ def main():
                             "so the query kernel, the updates and the merge launches are charged to it",
                      "us_per_launch_minus_rest": us_per_launch - us_rest,
                      "us_query_kernel_and_update_per_layer": us_rest,
-                     "traffic": None if args.fp8 else NCU_TRAFFIC_BYTES.get(w.name),
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if kernel_name == "decode_cta_kernel" else None,
                      "traffic_from": "committed ncu profile (profiles/), not this run",
                      **spread_of(leg_hbm, K)},
         "per_layer_api": {"early_fetch_on": call_fig(leg_main) if args.early_fetch else None,
@@ -699,34 +703,31 @@ def fp8_leg(args, dev):
     t = harness.step_tensors(dw)
     cache = dw.cache
 
-    def step():
-        cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"], dw.workspace)
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize(dev)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_per_layer, _, step_up_front = make_steps(dw, t)
     n = max(3, args.steps // 2)
-    e0.record()
-    for _ in range(n):
-        step()
-    e1.record()
-    torch.cuda.synchronize(dev)
-    ms = e0.elapsed_time(e1) / n
+    run, how, keep_alive = as_graph(step_per_layer, dev) if args.graph else (step_per_layer, "eager", None)
+    ms_loop = simple_time(run, dev, args.warmup, n)
+    ms = simple_time(step_up_front, dev, args.warmup, n)
+    del run, keep_alive
     if cache.skv_get_status() != 0:
         raise SystemExit("device status after the FP8 leg")
     st = cache.skv_cache_stats()
     tokens = int(dw.lens_cpu.sum())
-    return {"workload": w.name, "kv_bytes_per_token": st["bytes_per_token"], "ms_per_step": ms,
-            "us_per_attn_call": ms * 1e3 / w.n_layers,
-            "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
-            "tokens_attended_per_us": w.n_layers * tokens / (ms * 1e3)}
+    return {"workload": w.name, "kv_bytes_per_token": st["bytes_per_token"],
+            "per_layer_loop": {"ms_per_step": ms_loop, "us_per_attn_call": ms_loop * 1e3 / w.n_layers,
+                               "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms_loop * 1e-3) / 1e9,
+                               "tokens_attended_per_us": w.n_layers * tokens / (ms_loop * 1e3), "launch": how},
+            "inputs_up_front": {"ms_per_step": ms, "us_per_attn_call": ms * 1e3 / w.n_layers,
+                                "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
+                                "tokens_attended_per_us": w.n_layers * tokens / (ms * 1e3)}}
 
 
 def sharing_sweep(args, dev):
     """Llama-3-8B shape, batch 128, lengths U[512,2048]: owner fractions 1, 1/2, 1/4, 1/8 (evenly spaced
     owners).  Per ratio: cache bytes, the largest batch a 120e9-byte KV budget holds, whole decode steps per
-    second (update of the owners + attention of all 32 layers) and the time per attention call."""
+    second (per layer: query kernel that reads the previous layer's output, update on owners, attention -- the
+    loop of make_steps, replayed as a CUDA graph) and the time per attention call; beside it the same step through
+    skv_decode_step, which is given all queries up front."""
     from paper_2604_22782_b200 import harness
     rows = []
     budget = 120e9
@@ -737,21 +738,13 @@ def sharing_sweep(args, dev):
         t = harness.step_tensors(dw)
         cache = dw.cache
 
-        def step():
-            cache.skv_decode_step(t["Q"], t["K"], t["V"], dw.slot_new, dw.page_table, dw.seq_lens, t["out"],
-                                  dw.workspace)
-
-        for _ in range(args.warmup):
-            step()
-        torch.cuda.synchronize(dev)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dw.retune(early_fetch=args.early_fetch)
+        step_per_layer, _, step_up_front = make_steps(dw, t)
         n = max(3, args.steps // 2)
-        e0.record()
-        for _ in range(n):
-            step()
-        e1.record()
-        torch.cuda.synchronize(dev)
-        ms = e0.elapsed_time(e1) / n
+        run, how, keep_alive = as_graph(step_per_layer, dev) if args.graph else (step_per_layer, "eager", None)
+        ms = simple_time(run, dev, args.warmup, n)                  # the step as a decoder runs it (see make_steps)
+        ms_up_front = simple_time(step_up_front, dev, args.warmup, n)
+        del run, keep_alive
         st = cache.skv_cache_stats()
         pages = (dw.lens_cpu.to(torch.int64) + w.page_size - 1) // w.page_size
         per_seq_mean = st["n_owners"] * float(pages.double().mean()) * st["page_bytes"]
@@ -763,11 +756,13 @@ def sharing_sweep(args, dev):
             "max_batch_120e9_mean_len": int(budget // per_seq_mean),
             "max_batch_120e9_max_len": int(budget // per_seq_worst),
             "ms_per_step": ms, "steps_per_s": 1e3 / ms, "us_per_attn_call": ms * 1e3 / w.n_layers,
-            "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
+            "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9, "launch": how,
+            "inputs_up_front": {"ms_per_step": ms_up_front, "steps_per_s": 1e3 / ms_up_front,
+                                "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms_up_front * 1e-3) / 1e9},
         })
         if cache.skv_get_status() != 0:
             raise SystemExit("device status after the sweep")
-        del dw, cache, t
+        del dw, cache, t, step_per_layer, step_up_front
         torch.cuda.empty_cache()
     return rows
 

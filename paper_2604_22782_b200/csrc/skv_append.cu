@@ -305,6 +305,90 @@ __device__ __forceinline__ void append_fp8_page_wide(const AppendFp8Params &p, i
     __syncwarp();
 }
 
+// 4 x 4 bytes transposed: word i of the input holds bytes [i][0..3], word j of the output bytes [0..3][j]
+__device__ __forceinline__ void transpose_4x4_bytes(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                    uint32_t &o0, uint32_t &o1, uint32_t &o2, uint32_t &o3)
+{
+    const uint32_t t0 = __byte_perm(a0, a1, 0x5140), t1 = __byte_perm(a0, a1, 0x7362);
+    const uint32_t t2 = __byte_perm(a2, a3, 0x5140), t3 = __byte_perm(a2, a3, 0x7362);
+    o0 = __byte_perm(t0, t2, 0x5410);
+    o1 = __byte_perm(t0, t2, 0x7632);
+    o2 = __byte_perm(t1, t3, 0x5410);
+    o3 = __byte_perm(t1, t3, 0x7632);
+}
+
+// A whole page at head_dim 128 in registers only.  Lane = (token r of a round of four, 16-dim chunk c):
+// in round k the lane holds dims 16c .. 16c+15 of token 4k + r, read as 32 contiguous bytes (a warp-wide load
+// covers four whole rows).  A row's maximum is three shuffles among the eight lanes of the row.  K: the lane's
+// 16 codes ARE one 16-byte piece of the page.  V (dim-major pages): the four lanes that share a chunk swap
+// words so that lane r ends up with dims 16c+4r .. 16c+4r+3 of all 16 tokens (two exchange steps of a
+// four-way transpose per round, then byte transposes in registers), 64 contiguous bytes of the page.
+__device__ __forceinline__ void append_fp8_page_regs128(const AppendFp8Params &p, int64_t t0, int64_t page, int h, int which,
+                                                        int64_t layer, int lane)
+{
+    constexpr int D = 128;
+    constexpr unsigned ALL = 0xFFFFFFFFu;
+    const uint16_t *rows = (which ? p.V : p.K) + (layer * p.n_tokens * p.Hkv + h) * D;      // row of token t: + t * Hkv * D
+    uint8_t *blk = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)h * fp8_block_bytes(D);
+    const int c = lane & 7, r = lane >> 3;
+    uint4 in[4][2];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(rows + (t0 + 4 * k + r) * p.Hkv * D + 16 * c);
+        in[k][0] = __ldg(src);
+        in[k][1] = __ldg(src + 1);
+    }
+    uint32_t code[4][4];                   // [round][dim quad of the chunk]: four codes per word
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t w[8] = {in[k][0].x, in[k][0].y, in[k][0].z, in[k][0].w, in[k][1].x, in[k][1].y, in[k][1].z, in[k][1].w};
+        float amax = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w[i])), fabsf(bf16_hi(w[i]))));
+        amax = fmaxf(amax, __shfl_xor_sync(ALL, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(ALL, amax, 2));
+        amax = fmaxf(amax, __shfl_xor_sync(ALL, amax, 4));
+        const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            code[k][j] = pack_e4m3x2(__fmul_rn(bf16_lo(w[2 * j]), inv), __fmul_rn(bf16_hi(w[2 * j]), inv)) |
+                         (pack_e4m3x2(__fmul_rn(bf16_lo(w[2 * j + 1]), inv), __fmul_rn(bf16_hi(w[2 * j + 1]), inv)) << 16);
+        if (c == 0)
+            *reinterpret_cast<float *>(blk + (which ? fp8_vs_off(D) : fp8_ks_off(D)) + 4 * (4 * k + r)) = __fdiv_rn(amax, 448.f);
+    }
+    if (which == 0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            *reinterpret_cast<uint4 *>(blk + fp8_k_pos(D, 4 * k + r, 16 * c)) = make_uint4(code[k][0], code[k][1], code[k][2], code[k][3]);
+        return;
+    }
+    // four-way transpose of the dim quads across the lanes r = 0..3 of a chunk: afterwards code[k][q] of lane r is
+    // what lane q held as code[k][r] (token 4k + q, dims 16c + 4r ..)
+#pragma unroll
+    for (int bit = 0; bit < 2; ++bit) {
+        const bool up = (r >> bit) & 1;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (!((j >> bit) & 1)) {
+                    const int jl = j, jh = j | (1 << bit);
+                    const uint32_t give = up ? code[k][jl] : code[k][jh];
+                    const uint32_t got = __shfl_xor_sync(ALL, give, 8 << bit);
+                    if (up) code[k][jl] = got;
+                    else code[k][jh] = got;
+                }
+    }
+    // bytes: round k's four words (tokens 4k .. 4k+3) -> word k of each of the lane's four dims
+    uint32_t piece[4][4];                  // [dim of the lane][tokens 4k .. 4k+3]
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        transpose_4x4_bytes(code[k][0], code[k][1], code[k][2], code[k][3], piece[0][k], piece[1][k], piece[2][k], piece[3][k]);
+    uint4 *dst = reinterpret_cast<uint4 *>(blk + fp8_v_off(D) + (16 * c + 4 * r) * PAGE);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) dst[b] = make_uint4(piece[b][0], piece[b][1], piece[b][2], piece[b][3]);
+}
+
 // One row (token tok at offset off of its page) by one warp: scattered small stores (V is dim-major: one byte
 // in each of D rows; K: 4 bytes per lane).
 __device__ __forceinline__ void append_fp8_token(const AppendFp8Params &p, int64_t tok, int64_t page, int off, int h,
@@ -374,11 +458,13 @@ __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Param
 constexpr int FP8_GROUP_WARPS = 7;
 constexpr int FP8_IN_BYTES = PAGE * (2 * 128 + 16), FP8_CODE_BYTES = PAGE * (128 + 4);     // per warp, head_dim <= 128
 
-__global__ void __launch_bounds__(FP8_GROUP_WARPS * 32, 3) append_fp8_groups_kernel(AppendFp8Params p)
+// REGS128: head_dim 128, whole pages in registers (no shared memory, more warps per SM); otherwise through shared memory.
+template <bool REGS128>
+__global__ void __launch_bounds__(FP8_GROUP_WARPS * 32, REGS128 ? 4 : 3) append_fp8_groups_kernel(AppendFp8Params p)
 {
     pdl_trigger();
-    __shared__ __align__(16) uint8_t wide_in[FP8_GROUP_WARPS][FP8_IN_BYTES];
-    __shared__ __align__(16) uint8_t wide_codes[FP8_GROUP_WARPS][FP8_CODE_BYTES];
+    __shared__ __align__(16) uint8_t wide_in[REGS128 ? 1 : FP8_GROUP_WARPS][REGS128 ? 16 : FP8_IN_BYTES];
+    __shared__ __align__(16) uint8_t wide_codes[REGS128 ? 1 : FP8_GROUP_WARPS][REGS128 ? 16 : FP8_CODE_BYTES];
     constexpr unsigned ALL = 0xFFFFFFFFu;
     const int lane = threadIdx.x & 31;
     const int64_t n_groups = (p.n_tokens + PAGE - 1) / PAGE, n_items = n_groups * p.Hkv;
@@ -386,6 +472,15 @@ __global__ void __launch_bounds__(FP8_GROUP_WARPS * 32, 3) append_fp8_groups_ker
     for (int64_t item = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); item < n_items; item += stride) {
         const int h = (int)(item / n_groups);
         const int64_t i0 = (item - (int64_t)h * n_groups) * PAGE;
+        if (REGS128 && i0 + PAGE <= p.n_tokens) {
+            // the usual case first: the group's 16 tokens are one page, in order, from its first slot on
+            const long long s_l = (long long)p.slot_map[i0 + (lane & 15)];
+            const long long s_0 = __shfl_sync(ALL, s_l, 0);
+            if (s_0 >= 0 && (s_0 & (PAGE - 1)) == 0 && s_0 + PAGE <= p.n_slots && __all_sync(ALL, s_l == s_0 + (lane & 15))) {
+                append_fp8_page_regs128(p, i0, s_0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane);
+                continue;
+            }
+        }
         // slots of tokens i0-15 .. i0+30: window index x = -15 .. 16 in w0 (lane x+15), 17 .. 30 in w1 (lane x-17)
         auto slot_of = [&](int64_t i) -> long long { return (i >= 0 && i < p.n_tokens) ? (long long)p.slot_map[i] : -1ll; };
         const long long w0 = slot_of(i0 - 15 + lane), w1 = lane < 14 ? slot_of(i0 + 17 + lane) : -1ll;
@@ -407,8 +502,9 @@ __global__ void __launch_bounds__(FP8_GROUP_WARPS * 32, 3) append_fp8_groups_ker
         if (starts) {
             const int ls = __ffs(starts) - 1;
             const long long s0 = __shfl_sync(ALL, mine, ls);
-            append_fp8_page_wide(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane, wide_in[threadIdx.x >> 5],
-                                 wide_codes[threadIdx.x >> 5]);
+            if (REGS128) append_fp8_page_regs128(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane);
+            else append_fp8_page_wide(p, i0 + ls, s0 / PAGE, h, (int)blockIdx.y, blockIdx.z, lane, wide_in[threadIdx.x >> 5],
+                                      wide_codes[threadIdx.x >> 5]);
         }
         for (unsigned m = loose; m; m &= m - 1) {
             const int lt = __ffs(m) - 1;
@@ -495,7 +591,8 @@ cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream
     int64_t blocks = (items + 6) / 7;
     if (blocks > 4095) blocks = 4095;
     const dim3 grid((unsigned)blocks, 2, (unsigned)n_layers);
-    if (groups) append_fp8_groups_kernel<<<grid, 224, 0, s>>>(p);
+    if (groups && p.D == 128) append_fp8_groups_kernel<true><<<grid, 224, 0, s>>>(p);
+    else if (groups) append_fp8_groups_kernel<false><<<grid, 224, 0, s>>>(p);
     else append_fp8_kernel<<<grid, 224, 0, s>>>(p);
     return cudaGetLastError();
 }

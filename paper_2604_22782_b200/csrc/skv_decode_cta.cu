@@ -3,10 +3,12 @@
 //
 // The flattened (sequence, kv head, page) block list of the call is cut into one contiguous range per CTA.
 // One producer warp streams the CTA's blocks, in order, through ONE shared ring of 8 KB stages (a linear
-// bulk copy per block, completion on the stage's mbarrier); the consumer warps claim the blocks of the ring
-// one by one, in order (a shared counter: whoever is free takes the next block), each keeping a running
-// (max, sum, out) of its own for the (sequence, kv head) segment the blocks belong to.  At the end of every run of the range inside one
-// segment the consumers put their states side by side in shared memory and combine them:
+// bulk copy per block, completion on the stage's mbarrier); the consumer warps take the blocks of the ring
+// in turn (consumer c takes blocks c, c + C, ...: the same sum order every time, so results repeat bit for
+// bit) or, as an option, claim them from a shared counter (whoever is free takes the next block), each
+// keeping a running (max, sum, out) of its own for the (sequence, kv head) segment the blocks belong to.
+// At the end of every run of the range inside one segment the consumers put their states side by side in
+// shared memory and combine them:
 //   - a segment that lies wholly inside the CTA's range is finished on the spot: normalised, rounded to
 //     bf16 and written to `out`;
 //   - a segment that continues in a neighbouring CTA leaves one fp32 partial at slot  cta + segment  for the
