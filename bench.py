@@ -426,7 +426,10 @@ def main():
         "config": {"workload": w.name, "family": w.family, "n_layers": L, "owners": n_own, "batch": dw.batch,
                    "tokens": int(dw.lens_cpu.sum()), "q_heads": w.q_heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size, "early_fetch": args.early_fetch, "l2_keep": l2_keep,
-                   "l2": "inputs larger than L2: every attention call streams %.0f MB of pages" % (attn_bytes / 1e6),
+                   "l2": ("inputs larger than L2: every attention call streams %.0f MB of pages" % (attn_bytes / 1e6))
+                         if attn_bytes > 126e6 else
+                         ("a call's pages (%.2f MB) fit the L2 cache and are not flushed between calls: a small case, "
+                          "not a bandwidth figure" % (attn_bytes / 1e6)),
                    "step": "per layer: query kernel (reads the previous layer's output), skv_append on owners, "
                            "skv_decode_attn (split-K + merge); one stream, no events inside",
                    "value_is": "algorithmic GB/s (bytes the method must move / time), not DRAM traffic: with L2 reuse "
