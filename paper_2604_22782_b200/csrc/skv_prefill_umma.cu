@@ -3,14 +3,17 @@
 // tensor memory.
 //
 // One CTA (2 per SM) owns 128 query rows: 128/G tokens x the G query heads of one kv head, row
-// r = token r/G, head r%G.  Six warps:
+// r = token r/G, head r%G.  Eight warps:
 //   warps 0-3  softmax: thread r owns row r (= TMEM lane r)
 //   warp 4     lane 0 issues the UMMA instructions
-//   warp 5     copies K and V of the next key blocks into the rings
+//   warps 5, 6 copy K of the even / odd key blocks into the K ring (a warp waits for its own copies to land
+//              before it hands the stage over, so one warp doing every block made the landing time of a
+//              block's K the period of the whole pipeline: 2730 cycles per block with the softmax switched off)
+//   warp 7     copies V into the V ring
 // Shared memory
 //   Q tile   K-major core-matrix layout [D/8 chunks][128 rows][16 B]
 //   K ring   2 stages of 64 keys, [D/8 chunks][64 keys][16 B]: a page's K half is
-//            [chunk][16 keys][16 B]; warp 4 moves it with 16-byte cp.async copies that interleave
+//            [chunk][16 keys][16 B]; a copy warp moves it with 16-byte cp.async copies that interleave
 //            the four pages of a stage by chunk, which makes the 64 keys ONE N=64 operand
 //   V ring   2 stages of 4 pages, each page's V half copied as it is (4 KB): read as the B operand
 //            of P V it is the MN-major core-matrix layout
@@ -56,7 +59,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
            ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-constexpr int THREADS = 192;
+constexpr int THREADS = 256;
 
 template <int D>
 __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams p, int G)
@@ -114,7 +117,7 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
         tmem_relinquish();
     }
 
-    // ---- copies (warp 5, all lanes).  Lane j < KB carries the id of page j of a block. ----
+    // ---- copies (warps 5-7, all lanes).  Lane j < KB carries the id of page j of a block. ----
     auto load_ids = [&](int kb) -> int {
         const int pg = kb * KB + lane;
         int id = 0;
@@ -160,7 +163,7 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_k + 8 * (kb % NSTAGE)) : "memory");
     };
-    int v_copies = 0;                              // V blocks issued (warp 5)
+    int v_copies = 0;                              // V blocks issued (warp 7)
 
     // ---- this thread's row (softmax warps): Q into shared memory in core-matrix layout ----
     const int qi = tid / G, g = tid - qi * G;
@@ -182,55 +185,52 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     tc_fence_after();
     const uint32_t tmem = *slot_ptr;
 
-    if (warp == 5) {
-        // =================== copy warp ===================
+    if (warp == 5 || warp == 6) {
+        // =================== K copy warps: warp 5 the even key blocks (stage 0), warp 6 the odd ones ===================
+        const int par = warp - 5;
+        bool ok = true;
+        if (par < n_kb) {
+            int ids = load_ids(par);
+            copy_k(par, ids);
+            ids = load_ids(par + 2);                           // fetched ahead of its use
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            publish_k(par);
+            for (int kb = par; kb + 2 < n_kb; kb += 2) {
+                // Q K^T(kb) complete (its scores are ready): the stage takes K(kb+2).  The barrier's next completion
+                // needs the very copy issued after this wait, so the warp can never fall a whole phase behind.
+                if (lane == 0) ok = mbar_wait_bounded(s_ready + 8 * par, (uint32_t)((kb / NSTAGE) & 1));
+                ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                copy_k(kb + 2, ids);
+                ids = load_ids(kb + 4);
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                publish_k(kb + 2);
+            }
+        }
+        if (!ok && lane == 0) {
+            atomicOr(p.status, STATUS_TIMEOUT);
+            *gave_up = 1;
+        }
+    } else if (warp == 7) {
+        // =================== V copy warp ===================
         bool ok = true;
         int ids = load_ids(0);
         copy_v(0, ids);
-        copy_k(0, ids);
         v_copies = 1;
         if (n_kb > 1) {
             ids = load_ids(1);
             copy_v(1, ids);
-            copy_k(1, ids);
             v_copies = 2;
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-            publish_k(0);
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            publish_k(1);
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            publish_k(0);
         }
-        // page ids are fetched ahead of their use: ids_prev, ids_cur, ids_next belong to blocks kb+1, kb+2, kb+3
-        int ids_prev = ids, ids_cur = load_ids(2), ids_next = load_ids(3);
-        for (int kb = 0; kb + 1 < n_kb; ++kb) {
-            // Q K^T(kb) complete (its scores are ready): the K stage of block kb takes K(kb+2).
-            // P V of block kb-1 complete: the V stage of block kb-1 takes V(kb+1) (V(1) went out above).
-            // Each wait is on a per-stage barrier whose next completion needs the very copy issued after it,
-            // so this warp can never fall a whole phase behind.
-            const bool more_k = kb + 2 < n_kb;
-            if (more_k) {
-                if (lane == 0) ok = mbar_wait_bounded(s_ready + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
-                ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
-                if (!ok) break;
-                copy_k(kb + 2, ids_cur);
-            }
-            if (kb >= 1) {
-                if (lane == 0) ok = mbar_wait_bounded(pv_done + 8 * ((kb - 1) % NSTAGE), (uint32_t)(((kb - 1) / NSTAGE) & 1));
-                ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
-                if (!ok) break;
-                copy_v(kb + 1, ids_prev);
-                v_copies = kb + 2;
-            }
-            const int ids_new = load_ids(kb + 4);
-            if (more_k) {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                publish_k(kb + 2);
-            }
-            ids_prev = ids_cur;
-            ids_cur = ids_next;
-            ids_next = ids_new;
+        ids = load_ids(2);
+        for (int kb = 0; kb + 2 < n_kb; ++kb) {
+            // P V of block kb complete: its V stage takes V(kb+2)
+            if (lane == 0) ok = mbar_wait_bounded(pv_done + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
+            ok = __shfl_sync(FULL, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            copy_v(kb + 2, ids);
+            v_copies = kb + 3;
+            ids = load_ids(kb + 3);
         }
         if (!ok && lane == 0) {
             atomicOr(p.status, STATUS_TIMEOUT);
@@ -330,13 +330,13 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
                 if (!__all_sync(FULL, ok)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
-                for (int q4 = 0; q4 < D / 32; ++q4) {
-                    uint32_t ov[32];
-                    tmem_ld32(lane_base + COL_O + 32 * q4, ov);
+                for (int q4 = 0; q4 < D / 16; ++q4) {
+                    uint32_t ov[16];
+                    tmem_ld16(lane_base + COL_O + 16 * q4, ov);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-                    tmem_st32(lane_base + COL_O + 32 * q4, ov);
+                    for (int c = 0; c < 16; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                    tmem_st16(lane_base + COL_O + 16 * q4, ov);
                 }
             }
             l_sum *= alpha;
@@ -404,10 +404,10 @@ __global__ void __launch_bounds__(THREADS, 2) prefill_umma_kernel(PrefillParams 
     pdl_trigger();
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 5 || warp == 6) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (warp == 7) {
         // after a timeout the last copies issued may still be in flight: give them their (bounded) wait
         // before the shared memory goes away
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (lane == 0 && *gave_up)
             for (int kb = (v_copies > NSTAGE ? v_copies - NSTAGE : 0); kb < v_copies; ++kb)
                 mbar_wait_bounded(full_v + 8 * (kb % NSTAGE), (uint32_t)((kb / NSTAGE) & 1));
