@@ -30,16 +30,33 @@ constexpr int MAX_CONSUMERS = 8;      // (+ the producer: 288 threads, which the
 // (the states are written with 16-byte stores)
 __host__ __device__ constexpr int cta_part_floats(int G, int D) { return G * D + ((2 * G + 3) & ~3); }
 
-// try_wait loop with a time limit that also gives up as soon as another warp of the CTA has
+// One try with the thread suspended until the phase completes or `ns` nanoseconds have passed (a plain
+// try_wait comes back at once, and a warp that polls in a loop takes issue slots from the warps that work).
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+// wait with a time limit that also gives up soon after another warp of the CTA has
 __device__ __forceinline__ bool wait_or_quit(uint32_t bar, uint32_t parity, volatile int *gave_up)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
+    uint64_t t0 = 0;
     for (;;) {
-        for (int i = 0; i < 128; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait_for(bar, parity, 4000u)) return true;
         if (*gave_up) return false;
-        if (global_timer_ns() - t0 > 2000000000ull) return false;
+        const uint64_t now = global_timer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > 2000000000ull) return false;
     }
 }
 
@@ -86,7 +103,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 
 // Shared memory: tables (prefix, lens) | ring [S][BLOCK] | scratch [2][C] x ([G][D] fp32 out + [G][2] (max, sum))
 //                | query rows [2][G][D] bf16 | full[S], empty[S], run_done[2], q_full[2] mbarriers
-//                | gave_up word, claim counter, q_taken[2] | issued[S]
+//                | gave_up word, claim counter, q_taken[2] | issued[S] | scratch_free[2] mbarriers
 // A RUN is the part of the CTA's range inside one (sequence, kv head) segment.  What a run costs beyond its
 // blocks is kept off the consumers' path, because a range holds two to five of them and the slowest CTA sets
 // the end of the launch:
@@ -95,17 +112,25 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 //     copy of a buffer's rows so far, a plain count that runs on, because the producer lanes that refill the
 //     buffer do not see every phase a barrier would go through);
 //   - at the end of run r a consumer writes its state to scratch buffer r&1 and goes straight on with run
-//     r+1; the states of run r are combined at the end of run r+1, when they have long been complete.
-// Order at the end of run r: wait for run r-1 to be complete and combine it, THEN write the state of run r
-// and arrive for run r.  So a consumer that writes scratch buffer r&1 has passed the barrier of run r-1,
+//     r+1; the states of a run are combined by a warp of their own (warp C + 1), which gives the buffer
+//     back through the scratch_free barrier of its parity (a consumer waits for that of run r-2 before it
+//     writes run r's state).  Combining on the consumers cost 0.45 us per run: they all stop at the same
+//     blocks, and with them the SM's copies.  Only the range's last run is combined by the consumers, all
+//     together, because they have nothing else left to do then and one warp alone would make the CTA end later.
+// Where the registers leave no room for the extra warp (one query head per kv head at head_dim 128) the
+// consumers combine: the states of run r at the end of run r+1, when they have long been complete; order
+// at the end of run r: wait for run r-1 to be complete and combine it, THEN write the state of run r and
+// arrive for run r, so that a consumer that writes scratch buffer r&1 has passed the barrier of run r-1,
 // which every consumer arrives at only after it has combined run r-2, the last reader of that buffer.
 template <int D, class State>
-__global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode_cta_kernel(DecodeParams p, int G, int S)
+__global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + (State::CTA_COMBINER ? 2 : 1)) * 32, 1)
+__maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = State::BLOCK;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int C = (int)(blockDim.x >> 5) - 1;          // consumer warps; warp C is the producer
+    constexpr bool COMBINER = State::CTA_COMBINER;     // warp C + 1 combines the runs' states; else the consumers do
+    const int C = (int)(blockDim.x >> 5) - (COMBINER ? 2 : 1);   // consumer warps; warp C is the producer
     const uint64_t t_entry = p.trace ? global_timer_ns() : 0;
 
     const uint32_t base = smem_u32(smem_raw);
@@ -127,11 +152,12 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
     int *next_claim = const_cast<int *>(gave_up) + 1;
     volatile int *q_taken = gave_up + 2;                // [2]: consumers that have taken their copy of a buffer's rows, ever
     const uint32_t issued_at = q_full + 16 + 16;        // int [S]
+    const uint32_t scratch_free = (issued_at + 4u * (uint32_t)S + 7u) & ~7u;   // two: scratch buffer r&1 has been combined
 
     {   // the layout above must fit the shared memory the launch was given (else: flag it and do nothing)
         uint32_t given;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(given));
-        if (issued_at - base + 4u * (uint32_t)S > given) {
+        if (scratch_free - base + 16u > given) {
             if (threadIdx.x == 0) atomicOr(p.status, STATUS_BOUNDS);
             return;
         }
@@ -144,6 +170,7 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
         for (int i = 0; i < 2; ++i) {
             mbar_init(run_done + 8 * i, C);
             mbar_init(q_full + 8 * i, 1);
+            mbar_init(scratch_free + 8 * i, 1);
             q_taken[i] = 0;
         }
         gave_up[0] = 0;
@@ -301,7 +328,7 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
     // The page counts go to global memory for the merge kernel (after the wait on the kernel before this
     // one: the merge of an earlier call may still be reading this buffer).
     if (early_fetch) pdl_wait();
-    if (blockIdx.x == 0)
+    if (blockIdx.x == 0 && warp < C)
         for (int i = threadIdx.x; i <= p.B; i += C * 32) p.prefix[i] = prefix[i];
 
     // Dynamic: whoever is free takes the next block (the consumers of an SM end together, but which blocks a
@@ -323,22 +350,38 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
         return __shfl_sync(FULL, j, 0);
     };
     // the states of run `r` (all consumers', in scratch buffer r&1) -> the segment's rows, or its partial at `slot`
-    auto combine = [&](int r, int b, int h, bool whole, int slot) {
+    // the states of run `r` (all consumers', in scratch buffer r&1) -> the segment's rows, or its partial at `slot`;
+    // by the threads first, first + step, ... of a group of `step` threads, one pair of outputs at a time
+    auto combine = [&](int r, int b, int h, bool whole, int slot, int first, int step) {
         const float *buf = scratch + (size_t)(r & 1) * C * part_floats;
-        for (int e2 = (int)threadIdx.x; e2 < G * D / 2; e2 += C * 32) {       // thread t takes output pairs t, t + 32C, ...
+        for (int e2 = first; e2 < G * D / 2; e2 += step) {
             const int g = (2 * e2) / D;
+            // every consumer's (max, sum) of the head and its pair of outputs: all loads first
+            float m_c[MAX_CONSUMERS], l_c[MAX_CONSUMERS];
+            float2 v_c[MAX_CONSUMERS];
+#pragma unroll
+            for (int c = 0; c < MAX_CONSUMERS; ++c) {
+                m_c[c] = -INFINITY;
+                l_c[c] = 0.f;
+                v_c[c] = make_float2(0.f, 0.f);
+                if (c < C) {
+                    const float *sc = buf + c * part_floats;
+                    m_c[c] = sc[G * D + 2 * g];
+                    l_c[c] = sc[G * D + 2 * g + 1];
+                    v_c[c] = *reinterpret_cast<const float2 *>(sc + 2 * e2);
+                }
+            }
             float M = -INFINITY;
-            for (int c = 0; c < C; ++c) M = fmaxf(M, buf[c * part_floats + G * D + 2 * g]);
+#pragma unroll
+            for (int c = 0; c < MAX_CONSUMERS; ++c) M = fmaxf(M, m_c[c]);
             float L = 0.f, a0 = 0.f, a1 = 0.f;
-            for (int c = 0; c < C; ++c) {
-                const float *sc = buf + c * part_floats;
-                const float m_c = sc[G * D + 2 * g];
-                if (m_c == -INFINITY) continue;         // this consumer had no block in the run
-                const float wt = fast_exp2(m_c - M);
-                L = fmaf(wt, sc[G * D + 2 * g + 1], L);
-                const float2 v = *reinterpret_cast<const float2 *>(sc + 2 * e2);
-                a0 = fmaf(wt, v.x, a0);
-                a1 = fmaf(wt, v.y, a1);
+#pragma unroll
+            for (int c = 0; c < MAX_CONSUMERS; ++c) {
+                if (m_c[c] == -INFINITY) continue;      // this consumer had no block in the run (or is not there)
+                const float wt = fast_exp2(m_c[c] - M);
+                L = fmaf(wt, l_c[c], L);
+                a0 = fmaf(wt, v_c[c].x, a0);
+                a1 = fmaf(wt, v_c[c].y, a1);
             }
             if (whole) {
                 const float inv = L > 0.f ? 1.f / L : 0.f;
@@ -350,6 +393,35 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
             }
         }
     };
+
+    if (COMBINER && warp == C + 1) {
+        // ================= combiner =================
+        // Walks the range run by run like the consumers; when all of them have handed in their state of a run
+        // it combines them (the segment's rows, or its partial) and gives the scratch buffer back.  The
+        // consumers never stop for it: they would all stop at the same blocks, and with them the SM's copies.
+        Cursor cc = {0, 0, 0, 1};
+        if (n > 0) cc = locate(prefix, p.B, p.Hkv, x_first);
+        bool ok = true;
+        for (int k = 0, run = 0; k < n && ok; ++run) {
+            const int b = cc.b, h = cc.h, pages = cc.pages;
+            const int to_edge = reverse ? cc.pg + 1 : pages - cc.pg;
+            const int len = to_edge < n - k ? to_edge : n - k;
+            const int slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
+            if (k + len >= n) break;                   // the range's last run is combined by the consumers, all together
+            ok = wait_or_quit(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1), gave_up);
+            if (!ok) break;
+            combine(run, b, h, len == pages, slot, lane, 32);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(scratch_free + 8 * (run & 1));
+            k += len;
+            if (k < n) {
+                cc.pg = reverse ? cc.pg - (len - 1) : cc.pg + (len - 1);
+                step(cc, prefix, p.Hkv, reverse);
+            }
+        }
+        if (!ok && lane == 0 && !gave_up[0]) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
+        return;
+    }
 
     Cursor cons = {0, 0, 0, 1};
     if (n > 0) cons = locate(prefix, p.B, p.Hkv, x_first);
@@ -395,11 +467,16 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
                 held = claim();
             }
             if (failed) break;
-            // the run before this one has long been complete: combine it, then hand in this run's state
+            // Nobody goes on to run r+1 before everybody has handed in run r-1 (long the case, normally).  The
+            // consumers must stay within a run of each other: one without a block in a run neither waits for that
+            // run's query rows nor sees that phase of their barrier, and the count of rows taken, by which the
+            // producer refills a buffer, is only right while nobody counts two runs ahead.
             if (run > 0) {
                 if (!wait_or_quit(run_done + 8 * (qb ^ 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up)) { fail(); break; }
-                combine(run - 1, prev_b, prev_h, prev_whole, prev_slot);
+                if (!COMBINER) combine(run - 1, prev_b, prev_h, prev_whole, prev_slot, (int)threadIdx.x, C * 32);    // ... and combine it here
             }
+            // with a combining warp: the scratch buffer of this run's parity is free once run - 2 has been combined
+            if (COMBINER && run >= 2 && !wait_or_quit(scratch_free + 8 * qb, (uint32_t)(((run >> 1) - 1) & 1), gave_up)) { fail(); break; }
             if (has_blocks) st.finish(mine, mine + G * D, 0, G, lane);
             else if (lane < G) mine[G * D + 2 * lane] = -INFINITY;             // no block of this run: nothing to contribute
         }
@@ -416,9 +493,9 @@ __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + 1) * 32, 1) decode
             step(cons, prefix, p.Hkv, reverse);
         }
     }
-    if (!failed && run > 0) {
+    if (!failed && run > 0) {                          // the last run: every consumer has nothing else left to do
         if (wait_or_quit(run_done + 8 * ((run - 1) & 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up))
-            combine(run - 1, prev_b, prev_h, prev_whole, prev_slot);
+            combine(run - 1, prev_b, prev_h, prev_whole, prev_slot, (int)threadIdx.x, C * 32);
         else
             fail();
     }
@@ -440,7 +517,7 @@ cudaError_t launch_cta_t(const DecodeParams &p, int G, int grid, int consumers, 
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)((consumers + 1) * 32));
+    cfg.blockDim = dim3((unsigned)((consumers + (State::CTA_COMBINER ? 2 : 1)) * 32));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -462,7 +539,7 @@ size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, boo
     // 128 bytes of slack for aligning the ring base; barriers: full, empty per stage, two run barriers; two words
     // ... the query rows of two runs, their barriers, and the issued-block word of every stage
     return 128 + table_bytes(B) + (size_t)stages * blk + scratch + 2 * (size_t)G * D * 2 + 16 * (size_t)stages + 32 + 16 +
-           4 * (size_t)stages + 16;
+           4 * (size_t)stages + 16 + 8 + 16;           // (... and the two scratch-free barriers behind them, 8-byte aligned)
 }
 
 cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,

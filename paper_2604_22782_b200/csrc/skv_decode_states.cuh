@@ -25,6 +25,8 @@ template <int D>
 struct TensorCoreState {
     static constexpr int BLOCK = block_bytes(D);   // bytes of one (page, kv head) block
     static constexpr int MAX_CTA_CONSUMERS = 8;    // consumer warps of the CTA-per-range kernel that the registers allow
+    static constexpr bool CTA_COMBINER = true;     // ... and a warp of its own that combines the consumers' states
+    static constexpr int CTA_MAX_REGS = 160;       // 10 warps of it and a CTA of the merge kernel (64 x 208) fit one SM
     static constexpr int KS = D / 16;   // k-steps of QK^T, and pairs of 8-dim tiles of PV
     uint32_t qa[KS][2];
     float o[D / 8][4];
@@ -135,6 +137,8 @@ template <int D>
 struct CudaCoreState {
     static constexpr int BLOCK = block_bytes(D);
     static constexpr int MAX_CTA_CONSUMERS = D > 64 ? 7 : 8;   // (64 query and 64 output values per lane at head_dim 128)
+    static constexpr bool CTA_COMBINER = D <= 64;  // (at head_dim 128 the registers leave no room for a tenth warp)
+    static constexpr int CTA_MAX_REGS = D <= 64 ? 160 : 200;
     static constexpr int HC = D / 16;   // 16-byte chunks per dim half
     float q[D / 2];
     float o[D / 2];
@@ -262,6 +266,8 @@ template <int D>
 struct Fp8State {
     static constexpr int BLOCK = fp8_block_bytes(D);
     static constexpr int MAX_CTA_CONSUMERS = 8;
+    static constexpr bool CTA_COMBINER = true;
+    static constexpr int CTA_MAX_REGS = 160;
     static constexpr int KS = D / 16;
     static constexpr int DT = D / 4;    // dims per thread of a quad
     uint32_t qa[KS][2];                 // f16x2: dims DT*tig + 4ks + {0,1} and + {2,3} of Q / qmax
