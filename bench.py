@@ -260,6 +260,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the sharing-ratio sweep (owner fractions 1, 1/2, 1/4, 1/8)")
     ap.add_argument("--only", default="", help="comma-separated legs to run beside the headline leg "
                     "(up_front, roofline, single_call, e2e, sweep, prefill, fp8, small_batch); default: all")
+    ap.add_argument("--merge", type=int, default=-1, help="skv_set_decode_merge: 0 auto, 1 merge kernel, 2 inside the split-K kernel")
     ap.add_argument("--graph", type=int, default=1, help="1: the per-layer loop is captured into a CUDA graph and "
                     "replayed (GPU-bound timing); 0: issued from Python every step")
     ap.add_argument("--region-ms", type=float, default=1000.0, help="GPU work per leg over which the median is taken")
@@ -291,7 +292,8 @@ def main():
               tuning=[int(x) for x in args.tuning.split(",")] if args.tuning else None,
               overlap=args.overlap if args.overlap >= 0 else None,
               l2_keep=args.l2_keep if args.l2_keep >= 0 else None,
-              worker=tuple(int(x) for x in args.worker.split(",")) if args.worker else None)
+              worker=tuple(int(x) for x in args.worker.split(",")) if args.worker else None,
+              merge=args.merge if args.merge >= 0 else None)
     l2_keep = args.l2_keep if args.l2_keep >= 0 else DEFAULT_L2_KEEP
     harness.prefill(dw, upto_offset=-1)
     t = harness.step_tensors(dw)

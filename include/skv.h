@@ -444,6 +444,20 @@ int skv_set_decode_worker(skv_cache *cache, int mode, int consumers, int stages,
  * identical. */
 int skv_set_decode_early_fetch(skv_cache *cache, int enabled);
 
+/* Who combines the partials of a stand-alone attention call (skv_decode_attn,
+ * skv_decode_attn_static).  mode 1: the merge kernel, launched after every split-K
+ * launch.  mode 2: the CTA-per-range kernel itself, wherever it runs and its variant
+ * has the warp for it (not: one query head per kv head at head_dim 128; not with
+ * more than one CTA per SM; not the tcgen05 FP8 kernel): a segment cut by range
+ * ends is finished by handing its partial from range to range through the
+ * workspace, each hand-over marked by a tag the next CTA waits for (bounded;
+ * SKV_ERR_TIMEOUT in the status word when it runs out), and no merge launch
+ * follows.  That is quick when few segments are cut more than once and slow when a
+ * segment spans many ranges.  mode 0 (default): mode 2 when the call has at least
+ * as many (sequence, kv head) segments as CTAs, else mode 1.  Results agree within
+ * the rounding of a different summation order.  SKV_ERR_ARG for other modes. */
+int skv_set_decode_merge(skv_cache *cache, int mode);
+
 /* L2 reuse between consecutive layers that read the same owner (the paper's
  * depth-wise sharing makes them stream identical pages): with keep_percent > 0
  * such layers walk every worker's block range in alternating directions, and a

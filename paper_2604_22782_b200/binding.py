@@ -80,6 +80,7 @@ lib.skv_set_decode_overlap.argtypes = [_vp, _int]
 lib.skv_set_decode_l2_reuse.argtypes = [_vp, _int]
 lib.skv_set_decode_early_fetch.argtypes = [_vp, _int]
 lib.skv_set_decode_worker.argtypes = [_vp, _int, _int, _int, _int]
+lib.skv_set_decode_merge.argtypes = [_vp, _int]
 lib.skv_set_host_step.argtypes = [_vp, _int, _int]
 lib.skv_set_trace_buffer.argtypes = [_vp, _vp, _sz]
 lib.skv_decode_worker_count.argtypes = [_vp]
@@ -467,6 +468,9 @@ class SkvCache:
 
     def skv_set_decode_early_fetch(self, enabled: int) -> None:
         _check(lib.skv_set_decode_early_fetch(self._h, enabled), "skv_set_decode_early_fetch")
+
+    def skv_set_decode_merge(self, mode: int) -> None:
+        _check(lib.skv_set_decode_merge(self._h, mode), "skv_set_decode_merge")
 
     def skv_set_decode_l2_reuse(self, keep_percent: int) -> None:
         _check(lib.skv_set_decode_l2_reuse(self._h, keep_percent), "skv_set_decode_l2_reuse")

@@ -9,6 +9,8 @@
 #include <string.h>
 #include <vector>
 
+#include <atomic>
+#include <chrono>
 #include <mutex>
 
 using namespace skv;
@@ -67,6 +69,9 @@ struct skv_cache {
     int cta_stages = 0;              // its ring depth; 0 = as deep as shared memory allows, up to 20 per SM
     int cta_per_sm = 1;              // its CTAs resident per SM
     bool cta_in_turn = true;         // its consumers take the blocks in turn (reproducible) instead of first come first served
+    int merge_mode = 0;              // 0 auto, 1 a merge launch after every split-K launch, 2 merged by the CTA-per-range
+                                     // kernel itself wherever that kernel can
+    unsigned long long epoch_nonce = 0, epoch_count = 0;   // tags of in-kernel merging: never the same value twice
     std::vector<uint8_t> walk_reverse;   // per layer, for l2_keep_pct > 0: walk the block ranges backwards
     std::vector<uint8_t> walk_keep;      // per layer: the next layer reads the same owner
     int64_t launches = 0;
@@ -122,7 +127,7 @@ size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // GPU; each buffer is  page-count prefix | partial (max,sum) | partial outputs.  Nothing in it has to be
 // initialised: every slot the merge kernel reads was written by the split-K launch before it.
 struct WorkspaceLayout {
-    size_t prefix_off, ml_off, o_off, buf_bytes, total;
+    size_t prefix_off, ml_off, o_off, tag_off, buf_bytes, total;
     int64_t n_slots;
 };
 
@@ -135,7 +140,8 @@ WorkspaceLayout workspace_layout(const skv_cache *c, int batch, int q_heads, int
     w.prefix_off = 0;
     w.ml_off = w.prefix_off + round_up((size_t)(batch + 1) * sizeof(int32_t), 256);
     w.o_off = w.ml_off + round_up((size_t)w.n_slots * G * 2 * sizeof(float), 256);
-    w.buf_bytes = w.o_off + round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
+    w.tag_off = w.o_off + round_up((size_t)w.n_slots * G * c->head_dim * sizeof(float), 256);
+    w.buf_bytes = w.tag_off + round_up((size_t)w.n_slots * sizeof(unsigned long long), 256);    // one tag per slot
     w.total = 2 * w.buf_bytes;
     return w;
 }
@@ -307,6 +313,12 @@ int create_impl(skv_cache **out, int n_layers, const int32_t *r, int kv_heads, i
     }
     skv_cache *c = new (std::nothrow) skv_cache;
     if (!c) return SKV_ERR_ARG;
+    {   // a number of the handle's own for the tags of in-kernel merging: two handles may take turns on one workspace
+        static std::atomic<unsigned long long> handles{0};
+        const unsigned long long t = (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
+        c->epoch_nonce = ((t * 0x9E3779B97F4A7C15ull) >> 32) ^ (++handles * 0x85EBCA6Bull) ^ (unsigned long long)(uintptr_t)c;
+        c->epoch_nonce &= 0xFFFFFFFFull;
+    }
     c->n_layers = n_layers;
     c->kv_heads = kv_heads;
     c->head_dim = head_dim;
@@ -521,6 +533,7 @@ struct SplitkPlan {
     int n_workers = 0;       // ranges the block list was cut into
     int unit_tokens = PAGE;  // tokens per unit of the list
     int finished_single = 0; // segments inside one range were finished by the split-K launch itself
+    int merged = 0;          // ... and so were all others: no merge launch is needed
 };
 
 // Launches the split-K kernel on buffer `buf` (0 or 1) of the workspace.  `chained` = the call follows
@@ -579,6 +592,15 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.scale_log2 = sc * 1.4426950408889634f;
     p.flags = chained ? DECODE_LATE_WAIT : (c->early_fetch && c->tune.pdl) ? DECODE_EARLY_FETCH : 0;
     if (cta && c->cta_in_turn) p.flags |= DECODE_CLAIM_IN_TURN;
+    // Merging inside the kernel hands partials from CTA to CTA along the block list, which is only quick when
+    // few segments are cut more than once: by default where there are at least as many segments as ranges.
+    // Every CTA must be resident at once (one per SM), because a CTA waits for its neighbour's partial.
+    const int kernel = c->fp8 ? 2 : tensor_core ? 1 : 0;
+    const bool in_kernel_merge = cta && decode_cta_can_merge(c->head_dim, kernel) && c->cta_per_sm == 1 && c->merge_mode != 1 &&
+                                 (c->merge_mode == 2 || (int64_t)batch * c->kv_heads >= (int64_t)W);
+    if (in_kernel_merge) p.flags |= DECODE_MERGE_IN_KERNEL;
+    p.tags = reinterpret_cast<unsigned long long *>(ws + wl.tag_off);
+    p.epoch = (c->epoch_nonce << 32) | (++c->epoch_count & 0xFFFFFFFFull);
     p.keep_pct = 0;
     // what one call streams fits in L2 beside everything else when it is under about a third of it
     p.l2_fit_blocks = (int64_t)(c->l2_bytes / 3) / (int64_t)(c->fp8 ? fp8_block_bytes(c->head_dim) : block_bytes(c->head_dim));
@@ -589,7 +611,6 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.status = c->status_word();
     const size_t trace_need = (size_t)W * (cta ? c->cta_consumers : 1) * 32;
     p.trace = (c->trace && c->trace_bytes >= trace_need) ? c->trace : nullptr;
-    const int kernel = c->fp8 ? 2 : tensor_core ? 1 : 0;
     const cudaError_t le =
         umma  ? launch_decode_fp8_umma(p, c->head_dim, G, W, c->tune.pdl != 0, st)
         : cta ? launch_decode_cta(p, c->head_dim, G, kernel, W, c->cta_consumers, cta_S, c->tune.pdl != 0, st)
@@ -605,6 +626,7 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
         plan->n_workers = W;
         plan->unit_tokens = umma ? decode_fp8_umma_tile_tokens() : PAGE;
         plan->finished_single = cta ? 1 : 0;
+        plan->merged = in_kernel_merge ? 1 : 0;
     }
     return SKV_OK;
 }
@@ -672,6 +694,7 @@ int skv_decode_attn(skv_cache *c, int layer, const void *Q, const int32_t *page_
     int rc = launch_splitk(c, layer, Q, page_table, seq_lens, batch, q_heads, pt_stride, scale, workspace,
                            workspace_bytes, stream, &plan, out);
     if (rc) return rc;
+    if (plan.merged) return SKV_OK;
     return launch_merge_on(c, out, batch, q_heads, workspace, workspace_bytes, stream, 0, &plan, seq_lens, pt_stride);
 }
 
@@ -1131,6 +1154,13 @@ int skv_set_decode_worker(skv_cache *c, int mode, int consumers, int stages, int
     if (consumers) c->cta_consumers = consumers;
     c->cta_stages = stages;
     if (ctas_per_sm) c->cta_per_sm = ctas_per_sm;
+    return SKV_OK;
+}
+
+int skv_set_decode_merge(skv_cache *c, int mode)
+{
+    if (!c || mode < 0 || mode > 2) return SKV_ERR_ARG;
+    c->merge_mode = mode;
     return SKV_OK;
 }
 

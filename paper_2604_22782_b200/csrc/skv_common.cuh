@@ -104,6 +104,9 @@ constexpr int DECODE_EARLY_FETCH = 4;  // the lengths, the page table and all ca
 constexpr int DECODE_CLAIM_IN_TURN = 8; // CTA-per-range kernel: block j of a range goes to consumer j mod C instead
                                       // of to whichever consumer is free first
 
+constexpr int DECODE_MERGE_IN_KERNEL = 16; // CTA-per-range kernel: segments cut by range ends are finished by the CTAs
+                                          // themselves, handing partials from range to range (no merge launch follows)
+
 struct DecodeParams {
     const uint8_t *layer_base;  // first page of the owner layer that is read
     int64_t page_stride;
@@ -124,6 +127,8 @@ struct DecodeParams {
                                 // the next layer that reads the same owner: all of it is loaded with normal priority
     int *status;
     unsigned long long *trace;  // optional [n_workers][4]: sm id, entry ns, first-page ns, exit ns
+    unsigned long long *tags;   // [n_slots]: `epoch` once the partial at that slot is complete (DECODE_MERGE_IN_KERNEL)
+    unsigned long long epoch;   // a value no earlier call on this workspace has used
 };
 
 struct MergeParams {
@@ -192,6 +197,7 @@ cudaError_t launch_decode_splitk(const DecodeParams &p, int D, int G, int kernel
 cudaError_t launch_merge(const MergeParams &p, bool pdl, cudaStream_t s);
 // the CTA-per-range split-K kernel (skv_decode_cta.cu): grid = worker count, consumers + 1 warps per CTA
 size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, bool fp8);
+bool decode_cta_can_merge(int D, int kernel);   // the variant (kernel: 0 CUDA cores, 1 tensor cores, 2 FP8 pages) can finish cut segments itself
 cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,
                               bool pdl, cudaStream_t s);
 // FP8 pages of the sequences' pages -> bf16 pages in a scratch area (skv_dequant.cu); grid covers max_pages_per_seq

@@ -122,9 +122,11 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 // at the end of run r: wait for run r-1 to be complete and combine it, THEN write the state of run r and
 // arrive for run r, so that a consumer that writes scratch buffer r&1 has passed the barrier of run r-1,
 // which every consumer arrives at only after it has combined run r-2, the last reader of that buffer.
-template <int D, class State>
+// INMERGE: the instance that finishes cut segments itself (DECODE_MERGE_IN_KERNEL).  It is a kernel of its own
+// because it may use more registers: no CTA of the merge kernel has to fit on the SM beside it.
+template <int D, class State, bool INMERGE>
 __global__ void __launch_bounds__((State::MAX_CTA_CONSUMERS + (State::CTA_COMBINER ? 2 : 1)) * 32, 1)
-__maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
+__maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BLOCK = State::BLOCK;
@@ -142,7 +144,8 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
     const size_t scratch_off = ring_off + (size_t)S * BLOCK;
     const int part_floats = cta_part_floats(G, D);     // one consumer's state: out [G][D], then (max, sum) [G][2]
     float *scratch = reinterpret_cast<float *>(smem_raw + scratch_off);
-    const size_t q_off = scratch_off + (((size_t)2 * C * part_floats * 4 + 15) & ~(size_t)15);
+    const int CS = C + 1;                              // states per scratch buffer: the consumers' and one from the next range
+    const size_t q_off = scratch_off + (((size_t)2 * CS * part_floats * 4 + 15) & ~(size_t)15);
     const int q_bytes = G * D * 2;                     // the query rows of one kv head: a multiple of 128 bytes
     const uint16_t *q_rows = reinterpret_cast<const uint16_t *>(smem_raw + q_off);
     const size_t bars_off = q_off + 2 * (size_t)q_bytes;
@@ -153,11 +156,12 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
     volatile int *q_taken = gave_up + 2;                // [2]: consumers that have taken their copy of a buffer's rows, ever
     const uint32_t issued_at = q_full + 16 + 16;        // int [S]
     const uint32_t scratch_free = (issued_at + 4u * (uint32_t)S + 7u) & ~7u;   // two: scratch buffer r&1 has been combined
+    const uint32_t nb_ready = scratch_free + 16;        // the neighbouring range's partial is in the scratch (in-kernel merging)
 
     {   // the layout above must fit the shared memory the launch was given (else: flag it and do nothing)
         uint32_t given;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(given));
-        if (scratch_free - base + 16u > given) {
+        if (nb_ready - base + 8u > given) {
             if (threadIdx.x == 0) atomicOr(p.status, STATUS_BOUNDS);
             return;
         }
@@ -173,6 +177,7 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
             mbar_init(scratch_free + 8 * i, 1);
             q_taken[i] = 0;
         }
+        mbar_init(nb_ready, 1);
         gave_up[0] = 0;
         *next_claim = 0;
         for (int s = 0; s < S; ++s) publish_issued(issued_at + 4 * s, -1);
@@ -184,7 +189,11 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
     if (warp == 0) scan_lengths(p.seq_lens, p.B, PAGE, (int64_t)p.pt_stride * PAGE, p.status, prefix, lens, lane);
     __syncthreads();
 
-    const int64_t W = gridDim.x, w = blockIdx.x;
+    // Merging inside the kernel: a CTA may wait for the partial of the range after its own (forward walks) or
+    // before it (backward walks); the ranges are dealt so that this is always a CTA with a lower index, which
+    // the hardware has started no later than this one.
+    constexpr bool inmerge = INMERGE && COMBINER;
+    const int64_t W = gridDim.x, w = (inmerge && !reverse) ? (int64_t)gridDim.x - 1 - blockIdx.x : blockIdx.x;
     const int64_t T = (int64_t)prefix[p.B] * p.Hkv;
     int64_t x0 = 0;
     int n = 0;
@@ -193,6 +202,25 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
         n = (int)(worker_begin(w + 1, T, W) - x0);
     }
     const int64_t x_first = reverse ? x0 + n - 1 : x0;
+    // A run that is only a piece of its segment (the range ends cut it).  Without in-kernel merging its partial
+    // goes to `slot` for the merge kernel.  With it, partials travel along the block list against the walk: the
+    // piece its CTA reaches first (the SOURCE: the segment's last piece in forward walks, its first in backward
+    // walks) only leaves its partial; every other piece is the last run of its CTA, takes the partial at
+    // `src_slot` (its neighbour's, which already holds everything beyond), adds its own and either leaves the sum
+    // at `slot` or, as the FINAL piece, writes the segment's rows.  a = the run's lowest position in the list.
+    struct Piece { bool crossing, source, final; int slot, src_slot; };
+    auto piece_of = [&](int b, int h, int pages, int64_t a, int len) -> Piece {
+        Piece q;
+        const int64_t seg = (int64_t)b * p.Hkv + h, s0 = (int64_t)prefix[b] * p.Hkv + (int64_t)h * pages;
+        const bool below = a > s0, above = a + len < s0 + pages;      // the segment has blocks before / after this run
+        q.crossing = len != pages;
+        q.source = reverse ? !below : !above;
+        q.final = reverse ? !above : !below;
+        q.slot = partial_slot(T, W, w, a, seg);
+        q.src_slot = q.slot + (reverse ? -1 : 1);
+        return q;
+    };
+    const int64_t n_slots = W + (int64_t)p.B * p.Hkv;
 
     if (warp == C) {
         // ================= producer =================
@@ -352,19 +380,21 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
     // the states of run `r` (all consumers', in scratch buffer r&1) -> the segment's rows, or its partial at `slot`
     // the states of run `r` (all consumers', in scratch buffer r&1) -> the segment's rows, or its partial at `slot`;
     // by the threads first, first + step, ... of a group of `step` threads, one pair of outputs at a time
-    auto combine = [&](int r, int b, int h, bool whole, int slot, int first, int step) {
-        const float *buf = scratch + (size_t)(r & 1) * C * part_floats;
+    // (n_states: the consumers' C, or C + 1 with the neighbouring range's partial behind them; rows: write the
+    // segment's rows, normalised, instead of a partial)
+    auto combine = [&](int r, int b, int h, bool rows, int slot, int n_states, int first, int step) {
+        const float *buf = scratch + (size_t)(r & 1) * CS * part_floats;
         for (int e2 = first; e2 < G * D / 2; e2 += step) {
             const int g = (2 * e2) / D;
             // every consumer's (max, sum) of the head and its pair of outputs: all loads first
-            float m_c[MAX_CONSUMERS], l_c[MAX_CONSUMERS];
-            float2 v_c[MAX_CONSUMERS];
+            float m_c[MAX_CONSUMERS + 1], l_c[MAX_CONSUMERS + 1];
+            float2 v_c[MAX_CONSUMERS + 1];
 #pragma unroll
-            for (int c = 0; c < MAX_CONSUMERS; ++c) {
+            for (int c = 0; c < MAX_CONSUMERS + 1; ++c) {
                 m_c[c] = -INFINITY;
                 l_c[c] = 0.f;
                 v_c[c] = make_float2(0.f, 0.f);
-                if (c < C) {
+                if (c < n_states) {
                     const float *sc = buf + c * part_floats;
                     m_c[c] = sc[G * D + 2 * g];
                     l_c[c] = sc[G * D + 2 * g + 1];
@@ -373,17 +403,17 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
             }
             float M = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < MAX_CONSUMERS; ++c) M = fmaxf(M, m_c[c]);
+            for (int c = 0; c < MAX_CONSUMERS + 1; ++c) M = fmaxf(M, m_c[c]);
             float L = 0.f, a0 = 0.f, a1 = 0.f;
 #pragma unroll
-            for (int c = 0; c < MAX_CONSUMERS; ++c) {
+            for (int c = 0; c < MAX_CONSUMERS + 1; ++c) {
                 if (m_c[c] == -INFINITY) continue;      // this consumer had no block in the run (or is not there)
                 const float wt = fast_exp2(m_c[c] - M);
                 L = fmaf(wt, l_c[c], L);
                 a0 = fmaf(wt, v_c[c].x, a0);
                 a1 = fmaf(wt, v_c[c].y, a1);
             }
-            if (whole) {
+            if (rows) {
                 const float inv = L > 0.f ? 1.f / L : 0.f;
                 uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + ((int64_t)b * p.Hq + (int64_t)h * G) * D);
                 dst[e2] = pack_bf16x2(a0 * inv, a1 * inv);
@@ -399,6 +429,41 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
         // Walks the range run by run like the consumers; when all of them have handed in their state of a run
         // it combines them (the segment's rows, or its partial) and gives the scratch buffer back.  The
         // consumers never stop for it: they would all stop at the same blocks, and with them the SM's copies.
+        if (inmerge && blockIdx.x == 0)                // rows of empty sequences: zeros (no merge kernel will write them)
+            for (int b = 0; b < p.B; ++b)
+                if (lens[b] == 0) {
+                    uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + (int64_t)b * p.Hq * D);
+                    for (int i = lane; i < p.Hq * D / 2; i += 32) dst[i] = 0u;
+                }
+        // In-kernel merging, a run (the range's last) that takes its neighbour's partial: bring that partial into
+        // the scratch, behind the consumers' states, as soon as its tag says that it is complete -- which it has
+        // usually been for a long time (the neighbour reached that piece first), and the run has only begun.
+        auto fetch_neighbour = [&](const Piece &q, int run) -> bool {
+            bool ok = q.src_slot >= 0 && q.src_slot < n_slots;
+            if (!ok && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
+            uint64_t t0 = 0;
+            for (int it = 0; ok; ++it) {
+                unsigned long long tag;
+                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(tag) : "l"(p.tags + q.src_slot) : "memory");
+                if (tag == p.epoch) break;
+                __nanosleep(64);
+                if ((it & 255) == 255) {
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    if (gave_up[0] || now - t0 > 2000000000ull) ok = false;
+                }
+            }
+            ok = __all_sync(FULL, ok);
+            if (!ok) return false;
+            float *dst = scratch + ((size_t)(run & 1) * CS + C) * part_floats;
+            const float *so = p.part_o + (int64_t)q.src_slot * G * D, *sm = p.part_ml + (int64_t)q.src_slot * G * 2;
+            for (int i = lane * 4; i < G * D; i += 128)
+                *reinterpret_cast<float4 *>(dst + i) = __ldcg(reinterpret_cast<const float4 *>(so + i));
+            for (int i = lane; i < 2 * G; i += 32) dst[G * D + i] = __ldcg(sm + i);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(nb_ready);
+            return true;
+        };
         Cursor cc = {0, 0, 0, 1};
         if (n > 0) cc = locate(prefix, p.B, p.Hkv, x_first);
         bool ok = true;
@@ -406,12 +471,23 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
             const int b = cc.b, h = cc.h, pages = cc.pages;
             const int to_edge = reverse ? cc.pg + 1 : pages - cc.pg;
             const int len = to_edge < n - k ? to_edge : n - k;
-            const int slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
-            if (k + len >= n) break;                   // the range's last run is combined by the consumers, all together
+            const Piece q = piece_of(b, h, pages, reverse ? x0 + n - k - len : x0 + k, len);
+            const bool publish = inmerge && q.crossing && !q.final;      // somebody waits for this run's partial
+            const bool takes = inmerge && q.crossing && !q.source;       // (only the range's last run can)
+            if (takes) ok = fetch_neighbour(q, run);
+            if (!ok) break;
+            // the range's last run is combined by the consumers, all together, unless its partial has to be handed on
+            // (rare: a range that holds a middle piece of a long segment), which one warp does more simply
+            if (k + len >= n && !publish) break;
             ok = wait_or_quit(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1), gave_up);
             if (!ok) break;
-            combine(run, b, h, len == pages, slot, lane, 32);
+            const int n_states = takes ? C + 1 : C;
+            combine(run, b, h, !q.crossing, q.slot, n_states, lane, 32);
             __syncwarp();
+            if (publish && lane == 0) {
+                __threadfence();                        // the partial before its tag, for whoever reads the tag
+                asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.tags + q.slot), "l"(p.epoch) : "memory");
+            }
             if (lane == 0) mbar_arrive(scratch_free + 8 * (run & 1));
             k += len;
             if (k < n) {
@@ -428,8 +504,8 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
     uint64_t t_first = 0;
     int k = 0, run = 0;
     int held = -1;                                     // a block of the range this consumer has claimed and not done yet
-    int prev_b = 0, prev_h = 0, prev_slot = 0;         // the run before this one, not yet combined
-    bool prev_whole = false, failed = false;
+    int prev_b = 0, prev_h = 0, prev_slot = 0, prev_states = C;   // the run before this one, not yet combined
+    bool prev_rows = false, prev_skip = false, failed = false;
     auto fail = [&]() {
         if (lane == 0 && !gave_up[0]) { atomicOr(p.status, STATUS_TIMEOUT); gave_up[0] = 1; }
         failed = true;
@@ -440,7 +516,7 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
         const int to_edge = reverse ? cons.pg + 1 : pages - cons.pg;           // blocks left in this segment
         const int len = to_edge < n - k ? to_edge : n - k;
         const int qb = run & 1;
-        float *mine = scratch + ((size_t)qb * C + warp) * part_floats;
+        float *mine = scratch + ((size_t)qb * CS + warp) * part_floats;
         if (held < 0) held = claim();
         const bool has_blocks = held < k + len;
         {
@@ -473,7 +549,7 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
             // producer refills a buffer, is only right while nobody counts two runs ahead.
             if (run > 0) {
                 if (!wait_or_quit(run_done + 8 * (qb ^ 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up)) { fail(); break; }
-                if (!COMBINER) combine(run - 1, prev_b, prev_h, prev_whole, prev_slot, (int)threadIdx.x, C * 32);    // ... and combine it here
+                if (!COMBINER) combine(run - 1, prev_b, prev_h, prev_rows, prev_slot, C, (int)threadIdx.x, C * 32);    // ... and combine it here
             }
             // with a combining warp: the scratch buffer of this run's parity is free once run - 2 has been combined
             if (COMBINER && run >= 2 && !wait_or_quit(scratch_free + 8 * qb, (uint32_t)(((run >> 1) - 1) & 1), gave_up)) { fail(); break; }
@@ -482,10 +558,13 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(run_done + 8 * qb);
+        const Piece q = piece_of(b, h, pages, reverse ? x0 + n - k - len : x0 + k, len);
         prev_b = b;
         prev_h = h;
-        prev_whole = len == pages;                                             // the segment lies inside this range
-        prev_slot = partial_slot(T, W, w, x0 + (reverse ? n - 1 - k : k), (int64_t)b * p.Hkv + h);
+        prev_slot = q.slot;
+        prev_rows = !q.crossing || (inmerge && q.final);                       // the segment's rows come out of this run
+        prev_states = (inmerge && q.crossing && !q.source) ? C + 1 : C;        // ... with the neighbouring range's partial
+        prev_skip = inmerge && q.crossing && !q.final;                         // (a partial to hand on: the combining warp's)
         k += len;
         ++run;
         if (k < n) {                                   // first block of the next run
@@ -493,9 +572,10 @@ __maxnreg__(State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams p, int G, int S)
             step(cons, prefix, p.Hkv, reverse);
         }
     }
-    if (!failed && run > 0) {                          // the last run: every consumer has nothing else left to do
-        if (wait_or_quit(run_done + 8 * ((run - 1) & 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up))
-            combine(run - 1, prev_b, prev_h, prev_whole, prev_slot, (int)threadIdx.x, C * 32);
+    if (!failed && run > 0 && !prev_skip) {            // the last run: every consumer has nothing else left to do
+        if (wait_or_quit(run_done + 8 * ((run - 1) & 1), (uint32_t)(((run - 1) >> 1) & 1), gave_up) &&
+            (prev_states == C || wait_or_quit(nb_ready, 0u, gave_up)))
+            combine(run - 1, prev_b, prev_h, prev_rows, prev_slot, prev_states, (int)threadIdx.x, C * 32);
         else
             fail();
     }
@@ -512,7 +592,8 @@ cudaError_t launch_cta_t(const DecodeParams &p, int G, int grid, int consumers, 
 {
     if (consumers > State::MAX_CTA_CONSUMERS) consumers = State::MAX_CTA_CONSUMERS;      // (what its registers allow)
     const size_t smem = decode_cta_smem_bytes(D, p.B, G, consumers, stages, State::BLOCK != block_bytes(D));
-    auto kern = decode_cta_kernel<D, State>;
+    const bool inmerge = State::CTA_COMBINER && (p.flags & DECODE_MERGE_IN_KERNEL) != 0;
+    auto kern = inmerge ? decode_cta_kernel<D, State, State::CTA_COMBINER> : decode_cta_kernel<D, State, false>;
     cudaError_t e = ensure_dynamic_smem(kern, smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -530,16 +611,24 @@ cudaError_t launch_cta_t(const DecodeParams &p, int G, int grid, int consumers, 
 
 }  // namespace
 
+bool decode_cta_can_merge(int D, int kernel)
+{
+    if (D == 128) return kernel == 2 ? Fp8State<128>::CTA_COMBINER : kernel == 1 ? TensorCoreState<128>::CTA_COMBINER : CudaCoreState<128>::CTA_COMBINER;
+    if (D == 64) return kernel == 2 ? Fp8State<64>::CTA_COMBINER : kernel == 1 ? TensorCoreState<64>::CTA_COMBINER : CudaCoreState<64>::CTA_COMBINER;
+    return false;
+}
+
 size_t decode_cta_smem_bytes(int D, int B, int G, int consumers, int stages, bool fp8)
 {
     if (D != 64 && D != 128) return 0;
     if (consumers < 1 || consumers > MAX_CONSUMERS || stages < 2) return 0;
     const size_t blk = fp8 ? fp8_block_bytes(D) : block_bytes(D);
-    const size_t scratch = (((size_t)2 * consumers * cta_part_floats(G, D) * 4) + 15) & ~(size_t)15;
+    const size_t scratch = (((size_t)2 * (consumers + 1) * cta_part_floats(G, D) * 4) + 15) & ~(size_t)15;
     // 128 bytes of slack for aligning the ring base; barriers: full, empty per stage, two run barriers; two words
     // ... the query rows of two runs, their barriers, and the issued-block word of every stage
     return 128 + table_bytes(B) + (size_t)stages * blk + scratch + 2 * (size_t)G * D * 2 + 16 * (size_t)stages + 32 + 16 +
-           4 * (size_t)stages + 16 + 8 + 16;           // (... and the two scratch-free barriers behind them, 8-byte aligned)
+           4 * (size_t)stages + 16 + 8 + 16 + 8;       // (... the two scratch-free barriers behind them, 8-byte aligned, and
+                                                       // the barrier of the neighbouring range's partial)
 }
 
 cudaError_t launch_decode_cta(const DecodeParams &p, int D, int G, int kernel, int grid, int consumers, int stages,

@@ -37,7 +37,8 @@ class DeviceWorkload:
     def owners(self) -> List[int]:
         return [l for l in range(self.w.n_layers) if self.r[l] == l]
 
-    def retune(self, variant=None, tuning=None, overlap=None, l2_keep=None, early_fetch=None, worker=None) -> None:
+    def retune(self, variant=None, tuning=None, overlap=None, l2_keep=None, early_fetch=None, worker=None,
+               merge=None) -> None:
         """Change kernel variant / launch shape / overlap / L2 reuse / early fetch, then size the workspace again."""
         if variant is not None:
             self.cache.skv_set_decode_variant(variant)
@@ -51,6 +52,8 @@ class DeviceWorkload:
             self.cache.skv_set_decode_early_fetch(early_fetch)
         if worker is not None:                       # mode, or (mode, consumers, stages, CTAs per SM)
             self.cache.skv_set_decode_worker(*((worker,) if isinstance(worker, int) else worker))
+        if merge is not None:                        # 0 auto, 1 merge kernel, 2 inside the CTA-per-range kernel
+            self.cache.skv_set_decode_merge(merge)
         need = self.cache.skv_decode_workspace_bytes(self.batch, self.w.q_heads)
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)

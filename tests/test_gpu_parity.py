@@ -51,14 +51,14 @@ def _decode_layer(dw, layer, Q=None, scale=0.0):
 
 
 def _full_step_check(w, lens=None, r=None, variant=0, tuning=None, poison=False, permute=None, check_cache=True,
-                     overlap=None, l2_keep=None, early_fetch=None, worker=None):
+                     overlap=None, l2_keep=None, early_fetch=None, worker=None, merge=None):
     """One decode step of every layer: prefill n-1 tokens, append the last one, attend; compare all."""
     harness, dw = _make(w, lens=lens, r=r, permute=permute)
     if poison:   # every byte of the page area becomes a bf16 NaN pattern (0x7FC1)
         dw.pool_view = dw.cache.pool[256:].view(torch.int16)
         dw.pool_view.fill_(0x7FC1)
     dw.retune(variant=variant or None, tuning=tuning, overlap=overlap, l2_keep=l2_keep, early_fetch=early_fetch,
-              worker=worker)
+              worker=worker, merge=merge)
     B = dw.batch
     harness.prefill(dw, upto_offset=-1)
     seqs = list(range(B))
@@ -149,6 +149,39 @@ def test_cta_worker_shapes(variant, Hq, Hkv, D):
                           ((2, 4, 0, 2), 1), ((2, 4, 6, 2), 0), ((2, 2, 4, 4), 1), ((2, 8, 0, 1), 0),
                           (1, 0), (1, 1)):
         _full_step_check(w, lens=lens, variant=variant, check_cache=False, worker=worker, early_fetch=early)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (16, 2, 64), (3, 1, 128)])
+def test_merge_inside_the_cta_kernel(Hq, Hkv, D):
+    """skv_set_decode_merge(2): segments cut by range ends are finished by the CTAs themselves, partials handed from
+    range to range.  Few long segments (one spans dozens of ranges: a long chain of hand-overs), forward and
+    backward walks (layers 0 and 1 read one owner), an empty sequence (its rows must be zeros), with and without
+    early fetch, other consumer counts and ring depths; then a block list shorter than the number of CTAs (every
+    range a single block); the calls of one handle reuse one workspace, so tags of earlier calls are in it."""
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15, 0, 4100, 17, 16], dtype=torch.int32)
+    w = W.Workload("cta_merge", 3, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=71)
+    for worker, early in (((2, 8, 0), 0), ((2, 8, 0), 1), ((2, 3, 5), 1), ((2, 7, 4), 0), ((3, 6, 4), 1)):
+        _full_step_check(w, lens=lens, check_cache=False, worker=worker, early_fetch=early, merge=2)
+    short = torch.tensor([40, 17, 3, 0, 49], dtype=torch.int32)
+    w2 = W.Workload("cta_merge_short", 3, Hq, Hkv, D, 16, short.numel(), 0, 0, "explicit", explicit_r=(0, 0, 2), seed=72)
+    for early in (0, 1):
+        _full_step_check(w2, lens=short, check_cache=False, worker=(2, 8, 0), early_fetch=early, merge=2)
+    # (one launch per call then, not two)
+    from paper_2604_22782_b200 import harness
+    dw = harness.setup(w2, lens=short)
+    dw.retune(merge=2)
+    harness.prefill(dw, upto_offset=0)
+    before = dw.cache.skv_launch_count()
+    _decode_layer(dw, 0)
+    assert dw.cache.skv_launch_count() == before + 1
+    dw.retune(merge=1)
+    _decode_layer(dw, 0)
+    assert dw.cache.skv_launch_count() == before + 3
+    # many short sequences: more segments than CTAs, the default picks in-kernel merging by itself
+    many = torch.randint(1, 300, (200,), generator=torch.Generator().manual_seed(5), dtype=torch.int32)
+    w3 = W.Workload("cta_merge_many", 2, Hq, Hkv, D, 16, many.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=73)
+    _full_step_check(w3, lens=many, check_cache=False, early_fetch=1)
+    _full_step_check(w3, lens=many, check_cache=False, early_fetch=0, merge=1)
 
 
 def test_cta_worker_long_segments_and_reverse_walks():
