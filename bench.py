@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel of a stand-alone attention
 # call (decode_cta_kernel), mean of the two launches of the ncu capture summarised in
 # profiles/decode_cta_llama3_8b.md (taken on the two-layer form of the workload, which issues the same call)
-NCU_TRAFFIC_BYTES = {"llama3_8b": 343256000, "llama3_8b_2layers": 343256000}
+NCU_TRAFFIC_BYTES = {"llama3_8b": 345140000, "llama3_8b_2layers": 345140000}
 DEFAULT_L2_KEEP = 35     # the library's default share of each block range kept in L2 for the next layer
 
 
@@ -260,6 +260,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the sharing-ratio sweep (owner fractions 1, 1/2, 1/4, 1/8)")
     ap.add_argument("--only", default="", help="comma-separated legs to run beside the headline leg "
                     "(up_front, roofline, single_call, e2e, sweep, prefill, fp8, small_batch); default: all")
+    ap.add_argument("--batch", type=int, default=0, help="another number of sequences for the workload (a probe, not the benchmark)")
     ap.add_argument("--merge", type=int, default=-1, help="skv_set_decode_merge: 0 auto, 1 merge kernel, 2 inside the split-K kernel")
     ap.add_argument("--graph", type=int, default=1, help="1: the per-layer loop is captured into a CUDA graph and "
                     "replayed (GPU-bound timing); 0: issued from Python every step")
@@ -267,6 +268,9 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = W.get_workload(args.workload)
+    if args.batch > 0:
+        import dataclasses
+        w = dataclasses.replace(w, name=f"{w.name}_b{args.batch}", batch=args.batch)
     if args.impl == "reference":
         return run_reference(args, w)
     only = set(x for x in args.only.split(",") if x)

@@ -454,7 +454,7 @@ int skv_set_decode_early_fetch(skv_cache *cache, int enabled);
  * SKV_ERR_TIMEOUT in the status word when it runs out), and no merge launch
  * follows.  That is quick when few segments are cut more than once and slow when a
  * segment spans many ranges.  mode 0 (default): mode 2 when the call has at least
- * as many (sequence, kv head) segments as CTAs, else mode 1.  Results agree within
+ * two thirds as many (sequence, kv head) segments as CTAs, else mode 1.  Results agree within
  * the rounding of a different summation order.  SKV_ERR_ARG for other modes. */
 int skv_set_decode_merge(skv_cache *cache, int mode);
 

@@ -593,11 +593,12 @@ int launch_splitk(skv_cache *c, int layer, const void *Q, const int32_t *page_ta
     p.flags = chained ? DECODE_LATE_WAIT : (c->early_fetch && c->tune.pdl) ? DECODE_EARLY_FETCH : 0;
     if (cta && c->cta_in_turn) p.flags |= DECODE_CLAIM_IN_TURN;
     // Merging inside the kernel hands partials from CTA to CTA along the block list, which is only quick when
-    // few segments are cut more than once: by default where there are at least as many segments as ranges.
+    // few segments are cut more than once (a hand-over costs about 3 us, a merge launch 3 to 8): by default
+    // where there are at least two thirds as many segments as ranges (measured break-even: half as many).
     // Every CTA must be resident at once (one per SM), because a CTA waits for its neighbour's partial.
     const int kernel = c->fp8 ? 2 : tensor_core ? 1 : 0;
     const bool in_kernel_merge = cta && decode_cta_can_merge(c->head_dim, kernel) && c->cta_per_sm == 1 && c->merge_mode != 1 &&
-                                 (c->merge_mode == 2 || (int64_t)batch * c->kv_heads >= (int64_t)W);
+                                 (c->merge_mode == 2 || 3 * (int64_t)batch * c->kv_heads >= 2 * (int64_t)W);
     if (in_kernel_merge) p.flags |= DECODE_MERGE_IN_KERNEL;
     p.tags = reinterpret_cast<unsigned long long *>(ws + wl.tag_off);
     p.epoch = (c->epoch_nonce << 32) | (++c->epoch_count & 0xFFFFFFFFull);
