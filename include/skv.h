@@ -451,8 +451,8 @@ int skv_set_decode_early_fetch(skv_cache *cache, int enabled);
  * more than one CTA per SM; not the tcgen05 FP8 kernel): a segment cut by range
  * ends is finished by handing its partial from range to range through the
  * workspace, each hand-over marked by a tag the next CTA waits for (bounded;
- * SKV_ERR_TIMEOUT in the status word when it runs out), and no merge launch
- * follows.  That is quick when few segments are cut more than once and slow when a
+ * SKV_ERR_TIMEOUT in the status word when it runs out) and clears, and no merge
+ * launch follows.  That is quick when few segments are cut more than once and slow when a
  * segment spans many ranges.  mode 0 (default): mode 2 when the call has at least
  * two thirds as many (sequence, kv head) segments as CTAs, else mode 1.  Results agree within
  * the rounding of a different summation order.  SKV_ERR_ARG for other modes. */

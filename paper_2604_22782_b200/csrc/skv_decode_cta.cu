@@ -461,7 +461,13 @@ __maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams 
                 *reinterpret_cast<float4 *>(dst + i) = __ldcg(reinterpret_cast<const float4 *>(so + i));
             for (int i = lane; i < 2 * G; i += 32) dst[G * D + i] = __ldcg(sm + i);
             __syncwarp();
-            if (lane == 0) mbar_arrive(nb_ready);
+            if (lane == 0) {
+                // The tag has done its work: clear it.  A launch that is replayed from a CUDA graph carries the
+                // same epoch every time, so a tag left standing would pass for this launch's in the next replay.
+                // (Every tag has exactly one reader, this one; the slot is not written again before the kernel ends.)
+                asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p.tags + q.src_slot), "l"(0ull) : "memory");
+                mbar_arrive(nb_ready);
+            }
             return true;
         };
         Cursor cc = {0, 0, 0, 1};

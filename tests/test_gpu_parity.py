@@ -184,6 +184,39 @@ def test_merge_inside_the_cta_kernel(Hq, Hkv, D):
     _full_step_check(w3, lens=many, check_cache=False, early_fetch=0, merge=1)
 
 
+def test_merge_inside_the_kernel_replayed_from_a_graph():
+    """A call captured into a CUDA graph carries the same tag value in every replay: the tags of one replay must
+    not pass for those of the next.  The query changes between replays; every replay is checked against the oracle."""
+    from paper_2604_22782_b200 import harness
+    lens = torch.tensor([700, 33, 1, 256, 1023, 90, 15, 0, 4100, 17, 16], dtype=torch.int32)
+    w = W.Workload("cta_graph", 2, 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=74)
+    dw = harness.setup(w, lens=lens)
+    dw.retune(merge=2, early_fetch=1)
+    harness.prefill(dw, upto_offset=0)
+    o = _oracle_for(dw, list(range(dw.batch)), range(w.n_layers), upto_offset=0)
+    Q = harness.step_inputs(dw, 1)["Q"].clone()
+    out = torch.empty_like(Q)
+    side = torch.cuda.Stream(device=dw.device)
+    side.wait_stream(torch.cuda.current_stream(dw.device))
+    with torch.cuda.stream(side):
+        dw.cache.skv_decode_attn(1, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+    torch.cuda.current_stream(dw.device).wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        dw.cache.skv_decode_attn(1, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+    gen = torch.Generator(device="cpu").manual_seed(9)
+    for rep in range(4):
+        Q.copy_((torch.randn(Q.shape, generator=gen) * (0.5 + rep)).to(torch.bfloat16))
+        out.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        ref = o.decode_attn(1, Q.cpu(), dw.lens_cpu)
+        ok, err = _within_tol(out, ref)
+        assert ok, f"replay {rep}: max abs err {err}"
+    assert dw.cache.skv_get_status() == 0
+
+
 def test_cta_worker_long_segments_and_reverse_walks():
     """Segments much longer than a range (every CTA holds a piece of one segment and writes a partial), walked
     forwards and backwards with part of the stream kept in L2."""
