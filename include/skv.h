@@ -193,7 +193,8 @@ int skv_gather_fp8(skv_cache *cache, int layer, const int64_t *slot_ids, int64_t
  * under the CURRENT launch shape (ask again after skv_set_decode_tuning or
  * skv_set_decode_variant).
  * Independent of sequence lengths.  It holds, twice (two calls of a chain may
- * overlap), the split partials and a page-count prefix. */
+ * overlap), the split partials, one 8-byte tag per partial and a page-count
+ * prefix. */
 int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, size_t *out_bytes);
 
 /* Eq. (3.1) for one layer and one new token per sequence:
@@ -212,7 +213,7 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
  *   scale       <= 0 selects 1/sqrt(head_dim)
  *   workspace   device, 256-byte aligned, >= skv_decode_workspace_bytes; needs
  *               no initialisation and may be shared by calls on one stream.
- * Two launches.  Split-K (flash-decoding): the (sequence, kv head, page) blocks
+ * One or two launches.  Split-K (flash-decoding): the (sequence, kv head, page) blocks
  * of the call form one list that is cut into equal contiguous ranges, one per
  * worker, whatever the mix of lengths; a worker streams its range through
  * shared memory and leaves, for each (sequence, kv head) its range touches, an
@@ -220,8 +221,9 @@ int skv_decode_workspace_bytes(const skv_cache *cache, int batch, int q_heads, s
  * combines its partials by log-sum-exp and writes the bf16 rows.  The worker is
  * a CTA per SM whose warps share one ring of stages and combine their states in
  * shared memory -- it then finishes every (sequence, kv head) that lies inside
- * its range itself and the merge launch has only the others left -- or a single
- * warp (skv_set_decode_worker).  Slots past seq_lens[b] in the last page contribute nothing
+ * its range itself and the merge launch has only the others left, or, where
+ * skv_set_decode_merge lets it, finishes those too and no merge launch follows
+ * -- or a single warp (skv_set_decode_worker).  Slots past seq_lens[b] in the last page contribute nothing
  * whatever they contain.  No host synchronisation; sequence lengths are read
  * on the device.  The split-K launch waits for the work before it in the
  * stream before it reads anything; with skv_set_decode_overlap on, the merge

@@ -153,6 +153,29 @@ def test_accounting_only_handle_refuses_to_launch():
     assert e.value.status == B.SKV_ERR_UNSUPPORTED
 
 
+def test_settings_reject_values_outside_their_range():
+    """The launch-shape and merge settings take effect on the host only: bad values are SKV_ERR_ARG."""
+    c = skv.SkvCache([0, 0], 2, 64, 16, 4, accounting_only=True)
+    for mode in (0, 1, 2):
+        c.skv_set_decode_merge(mode)
+    for bad in (-1, 3):
+        with pytest.raises(skv.SkvError) as e:
+            c.skv_set_decode_merge(bad)
+        assert e.value.status == B.SKV_ERR_ARG
+    c.skv_set_decode_worker(2, 8, 16, 1)
+    for bad in ((4, 8, 16, 1), (2, 9, 16, 1), (2, 8, 1, 1), (2, 8, 27, 1), (2, 8, 16, 5)):
+        with pytest.raises(skv.SkvError) as e:
+            c.skv_set_decode_worker(*bad)
+        assert e.value.status == B.SKV_ERR_ARG
+    for bad in (-1, 2):
+        with pytest.raises(skv.SkvError) as e:
+            c.skv_set_decode_early_fetch(bad)
+        assert e.value.status == B.SKV_ERR_ARG
+    # the workspace holds one 8-byte tag per partial slot next to the partials themselves
+    small, large = c.skv_decode_workspace_bytes(4, 4), c.skv_decode_workspace_bytes(8, 4)
+    assert large > small > 0
+
+
 def test_work_partition_is_a_balanced_exact_cover():
     rnd = random.Random(1)
     cases = [(1, 1), (1, 7), (5, 7), (7, 7), (40960, 1184), (1183, 1184), (1185, 1184), (524288, 2368)]
