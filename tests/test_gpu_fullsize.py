@@ -219,3 +219,45 @@ def test_sharing_sweep_cache_bytes_scale_exactly():
     pages = int(((lens.to(torch.int64) + 15) // 16).sum())
     sizes = [skv_cache_pool_bytes(W.routing_map(W.sweep_workload(g)), 8, 128, 16, pages) - 256 for g in (1, 2, 4, 8)]
     assert [s * g for s, g in zip(sizes, (1, 2, 4, 8))] == [sizes[0]] * 4
+
+
+@pytest.mark.parametrize("group", [1, 2, 4, 8])
+def test_largest_batch_of_a_kv_budget_is_a_cache_that_can_be_created(group):
+    """The sweep's "largest batch in a 120e9-byte KV budget" (worst-case length 2048 = 128 pages per sequence) is a
+    closed form in bench.py; here the same arithmetic is checked against a real cache: a pool of exactly the bytes
+    the library asks for at that batch fits the budget, one sequence more does not, the cache is created on it and
+    its last page can be written and read back.  At a tenth of the budget for every ratio (12e9 bytes), and at the
+    whole 120e9 bytes for the owner fraction 1/8 when the GPU has the room."""
+    from paper_2604_22782_b200 import binding as skv
+    w = W.sweep_workload(group)
+    r = W.routing_map(w)
+    pages_per_seq = (w.len_hi + w.page_size - 1) // w.page_size
+    one_seq = skv.skv_cache_pool_bytes(r, w.kv_heads, w.head_dim, w.page_size, pages_per_seq) - 256
+    assert one_seq == (32 // group) * pages_per_seq * w.kv_heads * 2 * 16 * w.head_dim * 2
+    budgets = [12e9]
+    free, _ = torch.cuda.mem_get_info()
+    if group == 8 and free > 150e9:
+        budgets.append(120e9)
+    for budget in budgets:
+        max_batch = int(budget // one_seq)
+        need = skv.skv_cache_pool_bytes(r, w.kv_heads, w.head_dim, w.page_size, max_batch * pages_per_seq)
+        assert need - 256 <= budget < need - 256 + one_seq
+        if budget == 120e9:
+            assert max_batch == {1: 447, 2: 894, 4: 1788, 8: 3576}[group]      # the figures the benchmark prints
+        pool = torch.empty(need, dtype=torch.uint8, device="cuda")
+        cache = skv.SkvCache(r, w.kv_heads, w.head_dim, w.page_size, max_batch * pages_per_seq, device_pool=pool)
+        assert cache.skv_cache_stats()["kv_bytes"] == need - 256
+        # the very last slot of the very last page, on the last owner layer
+        last_owner = max(l for l in range(w.n_layers) if r[l] == l)
+        slot = torch.tensor([max_batch * pages_per_seq * w.page_size - 1], dtype=torch.int64, device="cuda")
+        K = torch.randn((1, w.kv_heads, w.head_dim), device="cuda").to(torch.bfloat16)
+        V = torch.randn((1, w.kv_heads, w.head_dim), device="cuda").to(torch.bfloat16)
+        cache.skv_append(last_owner, K, V, slot)
+        Kg, Vg = torch.zeros_like(K), torch.zeros_like(V)
+        cache.skv_gather(last_owner, slot, Kg, Vg)
+        torch.cuda.synchronize()
+        assert torch.equal(Kg.view(torch.int16), K.view(torch.int16)) and torch.equal(Vg.view(torch.int16), V.view(torch.int16))
+        assert cache.skv_get_status() == 0
+        cache.close()
+        del cache, pool
+        torch.cuda.empty_cache()
