@@ -71,6 +71,29 @@ def test_cache_codes_and_decode_outputs(Hq, Hkv, D, variant):
     assert st["page_bytes"] == Hkv * (2 * 16 * D + 128)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,variant", [(6, 2, 64, 0), (8, 2, 128, 2)])
+def test_decode_merged_inside_the_cta_kernel(Hq, Hkv, D, variant):
+    """FP8 pages through the CTA-per-range kernel (head_dim 64, or the mma.sync variant at head_dim 128) with the
+    segments cut by range ends finished inside the kernel (skv_set_decode_merge(2)), early fetch on and off."""
+    lens = torch.tensor([1, 5, 16, 17, 31, 33, 47, 100, 3, 700, 2049, 129, 256, 112, 0, 4100], dtype=torch.int32)
+    w = W.Workload("fp8_merge", 2, Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=(0, 0), seed=98, kv_std=1.7)
+    harness, dw = _setup(w, lens, poison=True)
+    o, stored, si, pos = _oracle(dw, range(2))
+    for early in (0, 1):
+        dw.retune(variant=variant, merge=2, early_fetch=early)
+        for l in range(2):
+            Q = harness.step_inputs(dw, l)["Q"]
+            out = torch.full((dw.batch, Hq, D), float("nan"), dtype=torch.bfloat16, device=dw.device)
+            before = dw.cache.skv_launch_count()
+            dw.cache.skv_decode_attn(l, Q, dw.page_table, dw.seq_lens, out, dw.workspace)
+            torch.cuda.synchronize()
+            assert dw.cache.skv_launch_count() == before + 1          # no merge launch
+            ref = o.decode_attn(l, Q.cpu(), dw.lens_cpu)
+            err = (out.cpu().double() - ref).abs()
+            assert bool((err <= ATOL + RTOL * ref.abs()).all()), f"layer {l} early {early}: max abs err {err.max().item()}"
+    assert dw.cache.skv_get_status() == 0
+
+
 def test_rows_of_very_different_magnitude():
     """Per-row scales spanning 2^-20 .. 2^12 in one sequence: the scales are applied outside the f16
     contractions, so neither overflow nor flush-to-zero may show.  With such a spread an output element
