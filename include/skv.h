@@ -442,8 +442,14 @@ int skv_set_decode_worker(skv_cache *cache, int mode, int consumers, int stages,
  * The caller's promise when switching it on: the kernel directly before each such
  * call in its stream writes neither seq_lens nor page_table nor any cached token
  * other than tokens in the last page of a sequence (skv_append of the step's new
- * token is such a kernel; so is any kernel that only produces Q).  Results are
- * identical. */
+ * token is such a kernel; so is any kernel that only produces Q).  If that kernel
+ * was itself launched with the programmatic stream-serialisation attribute and
+ * releases its dependents before it has waited for the kernel before it (as
+ * skv_append's decode-step kernel does), the promise covers that earlier kernel
+ * too, and so on up the chain: with a decoder whose own kernels between two
+ * attention calls behave like that, the next layer's attention kernel moves into
+ * the SMs that this layer's leaves and fills its ring while the rest still work.
+ * Results are identical. */
 int skv_set_decode_early_fetch(skv_cache *cache, int enabled);
 
 /* Who combines the partials of a stand-alone attention call (skv_decode_attn,

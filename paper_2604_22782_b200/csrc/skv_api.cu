@@ -447,7 +447,7 @@ int skv_append(skv_cache *c, int layer, const void *K, const void *V, const int6
         q.Hkv = c->kv_heads;
         q.D = c->head_dim;
         q.status = c->status_word();
-        if (launch_append_fp8(q, 1, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+        if (launch_append_fp8(q, 1, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
         c->launches += 1;
         return SKV_OK;
     }
@@ -463,7 +463,7 @@ int skv_append(skv_cache *c, int layer, const void *K, const void *V, const int6
     p.Hkv = c->kv_heads;
     p.D = c->head_dim;
     p.status = c->status_word();
-    if (launch_append(p, 1, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
+    if (launch_append(p, 1, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SKV_ERR_CUDA;
     c->launches += 1;
     return SKV_OK;
 }
@@ -725,7 +725,7 @@ int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot
         q.Hkv = c->kv_heads;
         q.D = c->head_dim;
         q.status = c->status_word();
-        if (launch_append_fp8(q, n_upd, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        if (launch_append_fp8(q, n_upd, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
             (void)cudaGetLastError();
             return SKV_ERR_CUDA;
         }
@@ -744,7 +744,7 @@ int step_updates(skv_cache *c, const void *K, const void *V, const int64_t *slot
     ap.Hkv = c->kv_heads;
     ap.D = c->head_dim;
     ap.status = c->status_word();
-    if (launch_append(ap, n_upd, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    if (launch_append(ap, n_upd, c->tune.pdl != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return SKV_ERR_CUDA;
     }

@@ -38,6 +38,8 @@ __device__ __forceinline__ CopyCoord coord_of(int64_t n_tok, int Hkv, int CH)
 __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
 {
     pdl_trigger();      // an attention launch right after this one may set itself up while the rows are copied
+    pdl_wait();         // (launched ahead of the end of the kernel before it: the rows and the slot map may be that
+                        // kernel's, and whoever waits for this kernel's end must be able to take the other's for granted)
     const int CH = p.D / CHUNK_ELEMS;
     const CopyCoord k = coord_of(p.n_tokens, p.Hkv, CH);
     if (!k.in_range) return;
@@ -424,6 +426,7 @@ __device__ __forceinline__ void append_fp8_token(const AppendFp8Params &p, int64
 __global__ void __launch_bounds__(COPY_THREADS) append_fp8_kernel(AppendFp8Params p)
 {
     pdl_trigger();
+    pdl_wait();         // (as in append_kernel)
     const int lane = threadIdx.x & 31;
     // (rows counted head-major and an odd number of warps in the grid: a warp then meets every position inside
     // a page in turn, instead of always the pages' first rows or never one)
@@ -551,7 +554,7 @@ int64_t copy_blocks(int64_t n, int Hkv, int D)
 }  // namespace
 
 // n_layers consecutive owner layers (grid.z) take rows from K/V [n_layers][n_tokens][Hkv][D] with one slot map
-cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s)
+cudaError_t launch_append(const AppendParams &p, int n_layers, bool pdl, cudaStream_t s)
 {
     const int64_t blocks = copy_blocks(p.n_tokens, p.Hkv, p.D);
     if (blocks == 0) return cudaSuccess;
@@ -564,8 +567,18 @@ cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s)
         append_pages_kernel<<<dim3((unsigned)ctas, 2, (unsigned)n_layers), PAGE_WARPS * 32, 0, s>>>(p);
         return cudaGetLastError();
     }
-    append_kernel<<<dim3((unsigned)blocks, 2, (unsigned)n_layers), COPY_THREADS, 0, s>>>(p);
-    return cudaGetLastError();
+    // A decode step's rows: with the attribute the launch may be brought forward to where the kernel before it
+    // releases its dependents (the kernel waits for that kernel's end itself before it touches anything).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 2, (unsigned)n_layers);
+    cfg.blockDim = dim3(COPY_THREADS);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, append_kernel, p);
 }
 
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t s)
@@ -581,7 +594,7 @@ cudaError_t launch_gather(const GatherParams &p, cudaStream_t s)
 
 namespace skv {
 
-cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s)
+cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, bool pdl, cudaStream_t s)
 {
     if (p.n_tokens == 0) return cudaSuccess;
     if (n_layers < 1 || n_layers > 65535) return cudaErrorInvalidConfiguration;
@@ -593,7 +606,18 @@ cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream
     const dim3 grid((unsigned)blocks, 2, (unsigned)n_layers);
     if (groups && p.D == 128) append_fp8_groups_kernel<true><<<grid, 224, 0, s>>>(p);
     else if (groups) append_fp8_groups_kernel<false><<<grid, 224, 0, s>>>(p);
-    else append_fp8_kernel<<<grid, 224, 0, s>>>(p);
+    else {                                                // a decode step's rows (launched as append_kernel is)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(224);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, append_fp8_kernel, p);
+    }
     return cudaGetLastError();
 }
 

@@ -179,7 +179,7 @@ struct DecodeTuning {
 };
 
 // host launchers (each returns a cudaError_t from the launch)
-cudaError_t launch_append(const AppendParams &p, int n_layers, cudaStream_t s);
+cudaError_t launch_append(const AppendParams &p, int n_layers, bool pdl, cudaStream_t s);
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t s);
 // decode attention over FP8 pages on tcgen05 (skv_decode_fp8_umma.cu): a worker is a CTA, grid = worker count
 bool decode_fp8_umma_supported(int D, int G);
@@ -187,7 +187,7 @@ int decode_fp8_umma_ctas_per_sm();
 int decode_fp8_umma_tile_tokens();           // tokens per unit of its flattened list
 size_t decode_fp8_umma_smem_bytes(int D, int B);
 cudaError_t launch_decode_fp8_umma(const DecodeParams &p, int D, int G, int grid, bool pdl, cudaStream_t s);
-cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, cudaStream_t s);
+cudaError_t launch_append_fp8(const AppendFp8Params &p, int n_layers, bool pdl, cudaStream_t s);
 cudaError_t launch_gather_fp8(const GatherFp8Params &p, cudaStream_t s);
 // smem bytes the split-K kernel needs for this shape, or 0 if unsupported
 size_t decode_smem_bytes(int D, int B, int warps, int stages, bool fp8);
