@@ -435,40 +435,83 @@ __maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams 
                     uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + (int64_t)b * p.Hq * D);
                     for (int i = lane; i < p.Hq * D / 2; i += 32) dst[i] = 0u;
                 }
-        // In-kernel merging, a run (the range's last) that takes its neighbour's partial: bring that partial into
-        // the scratch, behind the consumers' states, as soon as its tag says that it is complete -- which it has
-        // usually been for a long time (the neighbour reached that piece first), and the run has only begun.
-        auto fetch_neighbour = [&](const Piece &q, int run) -> bool {
-            bool ok = q.src_slot >= 0 && q.src_slot < n_slots;
-            if (!ok && lane == 0) atomicOr(p.status, STATUS_BOUNDS);
-            uint64_t t0 = 0;
-            for (int it = 0; ok; ++it) {
-                unsigned long long tag;
-                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(tag) : "l"(p.tags + q.src_slot) : "memory");
-                if (tag == p.epoch) break;
-                __nanosleep(64);
-                if ((it & 255) == 255) {
-                    const uint64_t now = global_timer_ns();
-                    if (t0 == 0) t0 = now;
-                    if (gave_up[0] || now - t0 > 2000000000ull) ok = false;
-                }
+        // In-kernel merging: the range's last run may take its neighbour's partial.  Which run that is, and from
+        // which slot, is known before the walk begins, and the neighbour reached that piece FIRST, so its partial
+        // is usually there long before this CTA comes to its last run.  The warp looks at the slot's tag whenever
+        // it waits for the consumers anyway and brings the partial into the scratch, behind the consumers' states
+        // (of both run parities: which one the last run has is not known yet), as soon as the tag says that it is
+        // complete.  Left to the last run itself, the tag's and the partial's round trips to L2 were in the open
+        // whenever that run was only a few blocks long (+2 to +4 us for such a CTA, and the launch ends with them).
+        Piece lastq = {false, false, false, 0, 0};
+        bool takes_last = false, fetched = false;
+        if (inmerge && n > 0) {
+            const Cursor lc = locate(prefix, p.B, p.Hkv, reverse ? x0 : x0 + n - 1);
+            const int64_t s0 = (int64_t)prefix[lc.b] * p.Hkv + (int64_t)lc.h * lc.pages;
+            const int64_t a = s0 > x0 ? s0 : x0, e = s0 + lc.pages < x0 + n ? s0 + lc.pages : x0 + n;
+            lastq = piece_of(lc.b, lc.h, lc.pages, a, (int)(e - a));
+            takes_last = lastq.crossing && !lastq.source;
+            if (takes_last && (lastq.src_slot < 0 || lastq.src_slot >= n_slots)) {
+                if (lane == 0) { atomicOr(p.status, STATUS_BOUNDS); gave_up[0] = 1; }
+                return;
             }
-            ok = __all_sync(FULL, ok);
-            if (!ok) return false;
-            float *dst = scratch + ((size_t)(run & 1) * CS + C) * part_floats;
-            const float *so = p.part_o + (int64_t)q.src_slot * G * D, *sm = p.part_ml + (int64_t)q.src_slot * G * 2;
-            for (int i = lane * 4; i < G * D; i += 128)
-                *reinterpret_cast<float4 *>(dst + i) = __ldcg(reinterpret_cast<const float4 *>(so + i));
-            for (int i = lane; i < 2 * G; i += 32) dst[G * D + i] = __ldcg(sm + i);
+        }
+        // one look at the tag; the partial, if it is there
+        auto try_fetch = [&]() -> bool {
+            unsigned long long tag;
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(tag) : "l"(p.tags + lastq.src_slot) : "memory");
+            if (!__all_sync(FULL, tag == p.epoch)) return false;
+            float *dst0 = scratch + (size_t)C * part_floats, *dst1 = dst0 + (size_t)CS * part_floats;
+            const float *so = p.part_o + (int64_t)lastq.src_slot * G * D, *sm = p.part_ml + (int64_t)lastq.src_slot * G * 2;
+            for (int i = lane * 4; i < G * D; i += 128) {
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(so + i));
+                *reinterpret_cast<float4 *>(dst0 + i) = v;
+                *reinterpret_cast<float4 *>(dst1 + i) = v;
+            }
+            for (int i = lane; i < 2 * G; i += 32) {
+                const float v = __ldcg(sm + i);
+                dst0[G * D + i] = v;
+                dst1[G * D + i] = v;
+            }
             __syncwarp();
             if (lane == 0) {
                 // The tag has done its work: clear it.  A launch that is replayed from a CUDA graph carries the
                 // same epoch every time, so a tag left standing would pass for this launch's in the next replay.
                 // (Every tag has exactly one reader, this one; the slot is not written again before the kernel ends.)
-                asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p.tags + q.src_slot), "l"(0ull) : "memory");
+                asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p.tags + lastq.src_slot), "l"(0ull) : "memory");
                 mbar_arrive(nb_ready);
             }
             return true;
+        };
+        // ... until it is there (bounded)
+        auto fetch_neighbour = [&]() -> bool {
+            uint64_t t0 = 0;
+            for (int it = 0;; ++it) {
+                if (try_fetch()) return true;
+                __nanosleep(64);
+                if ((it & 255) == 255) {
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    const bool quit = gave_up[0] || now - t0 > 2000000000ull;
+                    if (__any_sync(FULL, quit)) return false;
+                }
+            }
+        };
+        // the wait for a run's states, with a look at the tag every microsecond while the partial is still out
+        auto wait_run = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (mbar_try_wait(bar, parity)) return true;
+            uint64_t t0 = 0;
+            while (takes_last && !fetched) {
+                for (int i = 0; i < 16 && !fetched; ++i) {
+                    const bool done = mbar_try_wait_for(bar, parity, 1000u);
+                    if (__all_sync(FULL, done)) return true;
+                    fetched = try_fetch();
+                }
+                const uint64_t now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                const bool quit = gave_up[0] || now - t0 > 2000000000ull;
+                if (__any_sync(FULL, quit)) return false;
+            }
+            return wait_or_quit(bar, parity, gave_up);
         };
         Cursor cc = {0, 0, 0, 1};
         if (n > 0) cc = locate(prefix, p.B, p.Hkv, x_first);
@@ -480,12 +523,14 @@ __maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams 
             const Piece q = piece_of(b, h, pages, reverse ? x0 + n - k - len : x0 + k, len);
             const bool publish = inmerge && q.crossing && !q.final;      // somebody waits for this run's partial
             const bool takes = inmerge && q.crossing && !q.source;       // (only the range's last run can)
-            if (takes) ok = fetch_neighbour(q, run);
-            if (!ok) break;
             // the range's last run is combined by the consumers, all together, unless its partial has to be handed on
             // (rare: a range that holds a middle piece of a long segment), which one warp does more simply
-            if (k + len >= n && !publish) break;
-            ok = wait_or_quit(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1), gave_up);
+            if (k + len >= n && !publish) {
+                if (takes && !fetched) ok = fetched = fetch_neighbour();   // (takes: this is the last run, q is lastq)
+                break;
+            }
+            ok = wait_run(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1));
+            if (ok && takes && !fetched) ok = fetched = fetch_neighbour();
             if (!ok) break;
             const int n_states = takes ? C + 1 : C;
             combine(run, b, h, !q.crossing, q.slot, n_states, lane, 32);
