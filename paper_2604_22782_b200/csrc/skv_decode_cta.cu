@@ -45,6 +45,20 @@ __device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity,
     return ok != 0;
 }
 
+// A look at the barrier that never suspends the thread.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // wait with a time limit that also gives up soon after another warp of the CTA has
 __device__ __forceinline__ bool wait_or_quit(uint32_t bar, uint32_t parity, volatile int *gave_up)
 {
@@ -496,22 +510,24 @@ __maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams 
                 }
             }
         };
-        // the wait for a run's states, with a look at the tag every microsecond while the partial is still out
+        // The wait for a run's states.  This warp polls (a look that never suspends, then a short sleep) instead
+        // of letting the hardware suspend it: a suspended wait with a hint of 1 us came back only every 5 to 8 us,
+        // too rarely for the looks at the tag in between.  One warp per SM that looks about once a microsecond
+        // takes nothing from the consumers.
         auto wait_run = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (mbar_try_wait(bar, parity)) return true;
             uint64_t t0 = 0;
-            while (takes_last && !fetched) {
-                for (int i = 0; i < 16 && !fetched; ++i) {
-                    const bool done = mbar_try_wait_for(bar, parity, 1000u);
-                    if (__all_sync(FULL, done)) return true;
-                    fetched = try_fetch();
+            for (int it = 1;; ++it) {
+                const bool done = mbar_test_wait(bar, parity);
+                if (__all_sync(FULL, done)) return true;
+                if (takes_last && !fetched && (it & 1) == 0) fetched = try_fetch();
+                __nanosleep(400);
+                if ((it & 255) == 0) {
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    const bool quit = gave_up[0] || now - t0 > 2000000000ull;
+                    if (__any_sync(FULL, quit)) return false;
                 }
-                const uint64_t now = global_timer_ns();
-                if (t0 == 0) t0 = now;
-                const bool quit = gave_up[0] || now - t0 > 2000000000ull;
-                if (__any_sync(FULL, quit)) return false;
             }
-            return wait_or_quit(bar, parity, gave_up);
         };
         Cursor cc = {0, 0, 0, 1};
         if (n > 0) cc = locate(prefix, p.B, p.Hkv, x_first);
@@ -532,14 +548,15 @@ __maxnreg__(INMERGE ? 200 : State::CTA_MAX_REGS) decode_cta_kernel(DecodeParams 
             ok = wait_run(run_done + 8 * (run & 1), (uint32_t)((run >> 1) & 1));
             if (ok && takes && !fetched) ok = fetched = fetch_neighbour();
             if (!ok) break;
+            if (takes_last && !fetched) fetched = try_fetch();       // (before the work below, if it has come meanwhile)
             const int n_states = takes ? C + 1 : C;
             combine(run, b, h, !q.crossing, q.slot, n_states, lane, 32);
             __syncwarp();
+            if (lane == 0) mbar_arrive(scratch_free + 8 * (run & 1));   // (first: the fence below takes microseconds while the SM streams)
             if (publish && lane == 0) {
                 __threadfence();                        // the partial before its tag, for whoever reads the tag
                 asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.tags + q.slot), "l"(p.epoch) : "memory");
             }
-            if (lane == 0) mbar_arrive(scratch_free + 8 * (run & 1));
             k += len;
             if (k < n) {
                 cc.pg = reverse ? cc.pg - (len - 1) : cc.pg + (len - 1);
