@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the split-K kernel of a stand-alone attention
 # call (decode_cta_kernel), mean of the two launches of the ncu capture summarised in
 # profiles/decode_cta_llama3_8b.md (taken on the two-layer form of the workload, which issues the same call)
-NCU_TRAFFIC_BYTES = {"llama3_8b": 345140000, "llama3_8b_2layers": 345140000}
+NCU_TRAFFIC_BYTES = {"llama3_8b": 346880000, "llama3_8b_2layers": 346880000}
 DEFAULT_L2_KEEP = 35     # the library's default share of each block range kept in L2 for the next layer
 
 
