@@ -43,6 +43,13 @@ __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
     const int CH = p.D / CHUNK_ELEMS;
     const CopyCoord k = coord_of(p.n_tokens, p.Hkv, CH);
     if (!k.in_range) return;
+    const int which = blockIdx.y;                       // 0 = K, 1 = V
+    const int64_t layer = blockIdx.z;                   // owner layers of one launch, consecutive in the pool
+    const int64_t row_chunks = (int64_t)p.Hkv * CH;
+    const uint4 *src = (which ? p.V : p.K) + (layer * p.n_tokens + k.tok) * row_chunks + (int64_t)k.h * CH + k.c;
+    // the row's piece and the token's slot are asked for together (neither address depends on the other: one
+    // trip to memory instead of two, in a kernel that is nothing but that trip)
+    const uint4 piece = __ldg(src);
     const int64_t slot = p.slot_map[k.tok];
     if (slot < 0) return;
     if (slot >= p.n_slots) {
@@ -51,13 +58,9 @@ __global__ void __launch_bounds__(COPY_THREADS) append_kernel(AppendParams p)
     }
     const int64_t page = slot / PAGE;
     const int off = (int)(slot - page * PAGE);
-    const int which = blockIdx.y;                       // 0 = K, 1 = V
-    const int64_t layer = blockIdx.z;                   // owner layers of one launch, consecutive in the pool
-    const int64_t row_chunks = (int64_t)p.Hkv * CH;
-    const uint4 *src = (which ? p.V : p.K) + (layer * p.n_tokens + k.tok) * row_chunks + (int64_t)k.h * CH + k.c;
     uint8_t *dst = p.layer_base + layer * p.layer_stride + page * p.page_stride + (int64_t)k.h * block_bytes(p.D) +
                    (int64_t)which * half_bytes(p.D) + ((int64_t)k.c * PAGE + off) * 16;
-    *reinterpret_cast<uint4 *>(dst) = __ldg(src);
+    *reinterpret_cast<uint4 *>(dst) = piece;
 }
 
 // Large calls (a prompt): one warp per (group of 16 consecutive tokens of the call, kv head), grid.y = K or V,
