@@ -759,6 +759,10 @@ def fp8_leg(args, dev):
     ms_loop = simple_time(run, dev, args.warmup, n)
     ms = simple_time(step_up_front, dev, args.warmup, n)
     del run, keep_alive
+    step_coop = make_steps(dw, t, query_kernel=cooperating_query_kernel())[0]
+    run, _, keep_alive = as_graph(step_coop, dev) if args.graph else (step_coop, "eager", None)
+    ms_coop = simple_time(run, dev, args.warmup, n)
+    del run, keep_alive
     if cache.skv_get_status() != 0:
         raise SystemExit("device status after the FP8 leg")
     st = cache.skv_cache_stats()
@@ -766,7 +770,8 @@ def fp8_leg(args, dev):
     return {"workload": w.name, "kv_bytes_per_token": st["bytes_per_token"],
             "per_layer_loop": {"ms_per_step": ms_loop, "us_per_attn_call": ms_loop * 1e3 / w.n_layers,
                                "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms_loop * 1e-3) / 1e9,
-                               "tokens_attended_per_us": w.n_layers * tokens / (ms_loop * 1e3), "launch": how},
+                               "tokens_attended_per_us": w.n_layers * tokens / (ms_loop * 1e3), "launch": how,
+                               "us_per_attn_call_cooperating_query_kernel": ms_coop * 1e3 / w.n_layers},
             "inputs_up_front": {"ms_per_step": ms, "us_per_attn_call": ms * 1e3 / w.n_layers,
                                 "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9,
                                 "tokens_attended_per_us": w.n_layers * tokens / (ms * 1e3)}}
@@ -795,6 +800,11 @@ def sharing_sweep(args, dev):
         ms = simple_time(run, dev, args.warmup, n)                  # the step as a decoder runs it (see make_steps)
         ms_up_front = simple_time(step_up_front, dev, args.warmup, n)
         del run, keep_alive
+        # the same loop with a query kernel of the caller's that takes part in programmatic launches
+        step_coop = make_steps(dw, t, query_kernel=cooperating_query_kernel())[0]
+        run, _, keep_alive = as_graph(step_coop, dev) if args.graph else (step_coop, "eager", None)
+        ms_coop = simple_time(run, dev, args.warmup, n)
+        del run, keep_alive, step_coop
         st = cache.skv_cache_stats()
         pages = (dw.lens_cpu.to(torch.int64) + w.page_size - 1) // w.page_size
         per_seq_mean = st["n_owners"] * float(pages.double().mean()) * st["page_bytes"]
@@ -807,6 +817,9 @@ def sharing_sweep(args, dev):
             "max_batch_120e9_max_len": int(budget // per_seq_worst),
             "ms_per_step": ms, "steps_per_s": 1e3 / ms, "us_per_attn_call": ms * 1e3 / w.n_layers,
             "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms * 1e-3) / 1e9, "launch": how,
+            "cooperating_query_kernel": {"ms_per_step": ms_coop, "steps_per_s": 1e3 / ms_coop,
+                                         "us_per_attn_call": ms_coop * 1e3 / w.n_layers,
+                                         "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms_coop * 1e-3) / 1e9},
             "inputs_up_front": {"ms_per_step": ms_up_front, "steps_per_s": 1e3 / ms_up_front,
                                 "attn_gbs": w.n_layers * dw.kv_bytes_per_call() / (ms_up_front * 1e-3) / 1e9},
         })
