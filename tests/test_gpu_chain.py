@@ -38,16 +38,23 @@ def test_query_kernel_rejects_bad_arguments():
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("Hq,Hkv,D,worker", [
+    (8, 2, 128, None),       # tensor-core states, CTA per range with a combining warp
+    (4, 4, 128, None),       # one query head per kv head: CUDA-core states, no combining warp, merge launch
+    (8, 2, 64, None),        # head_dim 64
+    (8, 1, 128, None),       # eight query heads share a kv head
+    (8, 2, 128, 1),          # the warp-per-range kernel
+])
 @pytest.mark.parametrize("fp8", [False, True])
 @pytest.mark.parametrize("merge", [1, 2])
-def test_chained_programmatic_launches_match_the_oracle(merge, fp8):
+def test_chained_programmatic_launches_match_the_oracle(merge, fp8, Hq, Hkv, D, worker):
     from paper_2604_22782_b200 import harness
     hooks = _hooks_lib()
     lens = torch.tensor([16, 17, 1, 33, 4000, 250, 64, 1200, 2047, 5, 900, 3100], dtype=torch.int32)
     r = (0, 0, 2, 2, 2, 5)
-    w = W.Workload("chain", len(r), 8, 2, 128, 16, lens.numel(), 0, 0, "explicit", explicit_r=r, seed=67)
+    w = W.Workload("chain", len(r), Hq, Hkv, D, 16, lens.numel(), 0, 0, "explicit", explicit_r=r, seed=67)
     dw = harness.setup(w, lens=lens, fp8=fp8)
-    dw.retune(early_fetch=1, merge=merge)
+    dw.retune(early_fetch=1, merge=merge, worker=worker)
     harness.prefill(dw, upto_offset=-1)
     owners = [l for l in range(w.n_layers) if r[l] == l]
     if fp8:
